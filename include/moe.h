@@ -1,0 +1,210 @@
+/*
+ * moe.h - C ABI of the B200 (sm_100a) per-layer top-k Mixture-of-Experts forward pass.
+ *
+ * The operation is the MoE module of the LExI paper (arXiv 2509.02753), Section 2,
+ * paragraph "Mixture of Experts":
+ *
+ *     y = sum_{i in top-k} G(x)_i * E_i(x),      G(x) = Softmax(TopK[x . W_g]),
+ *
+ * evaluated with a number of active experts k_l that is set per layer (Algorithm 1's
+ * UpdateTopk step; Algorithm 2 returns the allocation k* = (k_1, ..., k_L)).  Each expert
+ * E_i is a bias-free SwiGLU FFN,  E(x) = W_down (silu(W_gate x) * (W_up x)),  the FFN of
+ * the models in the paper's Table 1.  An optional always-on shared expert (present in the
+ * Qwen1.5-MoE and DeepSeek-V2-Lite rows of Table 1, not described in the paper) is added
+ * after the routed sum.
+ *
+ * Conventions
+ *   - All tensors are dense, row-major, contiguous.  T tokens, d hidden size, E routed
+ *     experts, I expert intermediate size, I_s shared-expert intermediate size.
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
+ *     ordinary host memory.  Nothing in this library takes ownership of a caller pointer
+ *     or keeps it after the call returns, except where a function says so.
+ *   - Every call is asynchronous on the CUDA stream it is given (a cudaStream_t passed as
+ *     void*, NULL = the legacy default stream) unless it says "synchronises".
+ *   - One plan serves one stream at a time: calls on the same plan must not overlap on the
+ *     GPU, because they share the plan's workspace.
+ *   - Every function returns an int status: MOE_OK (0) or a negative MOE_ERR_* code.  No
+ *     exception, abort or device trap crosses this boundary.  Problems found by device
+ *     code (a bounded wait that ran out, an index outside its range) are recorded in a
+ *     device-side status word that moe_device_status() reads.
+ *   - There is no CPU fallback: without a CUDA device of compute capability 10.x every
+ *     compute entry point fails with MOE_ERR_CUDA.
+ */
+#ifndef LEXI_MOE_H_
+#define LEXI_MOE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    MOE_OK                  = 0,
+    MOE_ERR_INVALID_ARG     = -1,  /* null pointer, k out of 1..E, T out of 0..max_T, ...    */
+    MOE_ERR_SHAPE           = -2,  /* a size the kernels do not support (see moe_config_t)   */
+    MOE_ERR_ALIGN           = -3,  /* a tensor pointer that is not 16-byte aligned           */
+    MOE_ERR_WORKSPACE       = -4,  /* workspace allocation failed                            */
+    MOE_ERR_CUDA            = -5,  /* a CUDA runtime/driver call failed (no device, ...)     */
+    MOE_ERR_TIMEOUT         = -6,  /* a bounded device-side wait ran out                     */
+    MOE_ERR_NOT_IMPLEMENTED = -7,
+    MOE_ERR_DEVICE_CHECK    = -8   /* a device-side index check failed                       */
+};
+
+typedef enum { MOE_F32 = 0, MOE_BF16 = 1 } moe_dtype_t;
+
+/* How the expert FFNs are scheduled.  AUTO picks from dtype and T (see moe_layer_forward). */
+typedef enum {
+    MOE_SCHED_AUTO    = 0,
+    MOE_SCHED_SIMT    = 1,  /* CUDA-core FMA kernels; the only schedule for MOE_F32          */
+    MOE_SCHED_DECODE  = 2,  /* tcgen05, narrow weight tiles + split-K: weight streaming      */
+    MOE_SCHED_PREFILL = 3   /* tcgen05, 128x256 tiles, double-buffered TMEM accumulators     */
+} moe_schedule_t;
+
+/* Shapes fixed when the plan is made. */
+typedef struct {
+    int32_t d;             /* hidden size; multiple of 8 (multiple of 64 for bf16 tcgen05)   */
+    int32_t E;             /* routed experts, 1..128                                        */
+    int32_t I;             /* expert intermediate size; multiple of 8                        */
+    int32_t I_shared;      /* shared-expert intermediate size, 0 = no shared expert          */
+    int32_t shared_gate;   /* 0: shared output added as is; 1: times sigmoid(x . w_s)        */
+    int32_t max_T;         /* largest token count of any call, >= 1                          */
+    int32_t max_k;         /* largest k_l of any call, 1 <= max_k <= E                       */
+    int32_t dtype;         /* moe_dtype_t of x, y and all weights; router math is fp32       */
+    float   routed_scale;  /* factor on the routed sum before the shared term (1.0 usually)  */
+} moe_config_t;
+
+/* Weights of one layer: device pointers, caller-owned, read-only, 16-byte aligned. */
+typedef struct {
+    const void  *router_W;     /* [E, d]   gating matrix W_g, row e = expert e               */
+    const float *router_bias;  /* [E] fp32 added to the logits, or NULL                      */
+    const void  *W_gate;       /* [E, I, d]                                                  */
+    const void  *W_up;         /* [E, I, d]                                                  */
+    const void  *W_down;       /* [E, d, I]                                                  */
+    const void  *Ws_gate;      /* [I_s, d] or NULL when I_shared = 0                         */
+    const void  *Ws_up;        /* [I_s, d]                                                   */
+    const void  *Ws_down;      /* [d, I_s]                                                   */
+    const void  *w_s;          /* [d], needed when shared_gate = 1                           */
+} moe_layer_weights_t;
+
+typedef struct moe_plan moe_plan_t;   /* opaque; owns the workspace and the schedule state */
+
+/*
+ * moe_plan_create: validates the shapes and allocates (cudaMalloc, on the current device)
+ * the workspace for calls of up to max_T tokens and max_k active experts: router logits,
+ * top-k indices and gates, dispatch tables, the expert-ordered copy of x, the intermediate
+ * h, the per-pair expert outputs, the fp32 residual stream of the stack.
+ * Synchronises.  *out receives the plan (NULL on failure).
+ * Errors: INVALID_ARG, SHAPE, CUDA (no sm_100 device), WORKSPACE.
+ */
+int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out);
+
+/* Frees the workspace.  Synchronises the device first.  NULL is accepted. */
+int moe_plan_destroy(moe_plan_t *plan);
+
+/* Bytes of device memory the plan holds (0 for NULL). */
+uint64_t moe_plan_workspace_bytes(const moe_plan_t *plan);
+
+/* Forces a schedule for later calls (MOE_SCHED_AUTO restores the choice by shape).
+ * Errors: INVALID_ARG; SHAPE if the schedule cannot run the plan's dtype/shape. */
+int moe_plan_set_schedule(moe_plan_t *plan, int32_t schedule);
+
+/* The schedule the next call with T tokens and k_l active experts would use. */
+int moe_plan_get_schedule(const moe_plan_t *plan, int32_t T, int32_t k_l);
+
+/*
+ * moe_layer_forward: one MoE module with k_l active experts (Section 2; UpdateTopk of
+ * Algorithm 1 is the k_l argument).
+ *
+ *   x [T, d] device, read-only;  y [T, d] device, written;  y must not overlap x.
+ *   1 <= k_l <= max_k;  0 <= T <= max_T (T = 0 is a no-op).
+ *   renorm = 1: gates are the softmax over the k_l selected logits (the paper's formula);
+ *   renorm = 0: gates are the selected entries of the softmax over all E logits.
+ *   Selection is on the fp32 logits x . W_g (+ bias): larger first, equal -> lower index.
+ *
+ * Steps, all on the GPU: router (GEMM + softmax + top-k_l + renorm), dispatch (per-expert
+ * histogram, prefix scan, stable permutation, gather of x into expert order), grouped
+ * gate/up GEMM with SwiGLU, grouped down GEMM, weighted combine plus shared expert.
+ * Schedule under MOE_SCHED_AUTO: SIMT for fp32; for bf16 DECODE when T * k_l < 16 * E
+ * (fewer than 16 tokens per expert on average: weight streaming decides the time), else PREFILL.
+ * Errors: INVALID_ARG, ALIGN, CUDA.
+ */
+int moe_layer_forward(moe_plan_t *plan, const void *x, const moe_layer_weights_t *w,
+                      int32_t T, int32_t k_l, int32_t renorm, void *y, void *cuda_stream);
+
+/*
+ * moe_layer_forward_host: the same call for callers that hold x and y in HOST memory
+ * (pinned memory makes the copies asynchronous).  Copies x to the device, runs
+ * moe_layer_forward, copies y back, all on the given stream; weights stay on the device.
+ * The staging buffers belong to the plan.  Does not synchronise: wait on the stream
+ * before reading y_host.
+ */
+int moe_layer_forward_host(moe_plan_t *plan, const void *x_host, const moe_layer_weights_t *w,
+                           int32_t T, int32_t k_l, int32_t renorm, void *y_host,
+                           void *cuda_stream);
+
+/*
+ * moe_stack_forward: L MoE modules in sequence, layer l with k_vec[l] active experts -
+ * the deployment form of the allocation k* that Algorithm 2 returns:
+ *
+ *     h <- h + MoE_l(h; k_vec[l])        l = 0 .. n_layers-1
+ *
+ *   h [T, d] device, updated in place.  layers: HOST array of n_layers weight structs.
+ *   k_vec: HOST array of n_layers values, each in 1..max_k.
+ * For bf16 the running h is kept in fp32 inside the plan (each layer reads it rounded to
+ * bf16; the final h is rounded once), so rounding does not accumulate over the layers.
+ * Errors: as moe_layer_forward.
+ */
+int moe_stack_forward(moe_plan_t *plan, void *h, const moe_layer_weights_t *layers,
+                      int32_t n_layers, const int32_t *k_vec, int32_t renorm, int32_t T,
+                      void *cuda_stream);
+
+/*
+ * moe_route_from_logits (test hook): TopK + Softmax + dispatch tables from logits the
+ * caller supplies, so that routing can be compared bit for bit (Section 2's TopK[.] and
+ * Softmax).  logits [T, E] fp32 device.  Outputs, device, any may be NULL:
+ *   topk_idx [T, k_l] int32 (descending logit), topk_w [T, k_l] fp32,
+ *   counts [E] int32, offsets [E+1] int32 (exclusive scan), perm [T*k_l] int32
+ *   (perm[r] = t*k_l + j of the r-th row in expert-major order, ascending t inside an expert).
+ */
+int moe_route_from_logits(moe_plan_t *plan, const float *logits, int32_t T, int32_t k_l,
+                          int32_t renorm, int32_t *topk_idx, float *topk_w, int32_t *counts,
+                          int32_t *offsets, int32_t *perm, void *cuda_stream);
+
+/*
+ * moe_last_routing (test hook): copies the routing artefacts of the plan's most recent
+ * layer call into caller device buffers (shapes as in moe_route_from_logits, for the T and
+ * k_l of that call; logits [T, E] fp32).  Any pointer may be NULL.
+ */
+int moe_last_routing(moe_plan_t *plan, int32_t *topk_idx, float *topk_w, int32_t *counts,
+                     int32_t *offsets, int32_t *perm, float *logits, void *cuda_stream);
+
+/*
+ * moe_device_status: synchronises the stream, reads and clears the device status word.
+ * Returns MOE_OK, MOE_ERR_TIMEOUT, MOE_ERR_DEVICE_CHECK or MOE_ERR_CUDA.
+ */
+int moe_device_status(moe_plan_t *plan, void *cuda_stream);
+
+/*
+ * Stage timing (measurement aid).  While enabled, every layer call records CUDA events on its
+ * stream at the stage boundaries: router | dispatch + gather | gate/up GEMM + SwiGLU | down GEMM
+ * | combine.  moe_plan_stage_times synchronises on the recorded events, adds the elapsed
+ * milliseconds of every layer call since the last read into ms[0..4] (host, 5 floats), stores
+ * the number of calls summed in *n_calls, and forgets them.  At most 256 calls are kept between
+ * reads; later ones are not timed.  Enabling allocates the events; disabling frees them.
+ */
+enum { MOE_STAGE_ROUTER = 0, MOE_STAGE_DISPATCH = 1, MOE_STAGE_FFN1 = 2, MOE_STAGE_FFN2 = 3,
+       MOE_STAGE_COMBINE = 4, MOE_N_STAGES = 5 };
+int moe_plan_set_stage_timing(moe_plan_t *plan, int32_t enable);
+int moe_plan_stage_times(moe_plan_t *plan, float *ms, int32_t *n_calls);
+
+/* Number of kernel launches this plan has issued since it was created. */
+uint64_t moe_plan_launch_count(const moe_plan_t *plan);
+
+/* Static string for a status code. */
+const char *moe_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LEXI_MOE_H_ */

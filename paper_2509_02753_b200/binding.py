@@ -1,0 +1,297 @@
+"""Thin ctypes binding of the C ABI in ``include/moe.h``.
+
+Argument marshalling only: every step of the MoE forward pass runs in the CUDA
+kernels of ``liblexi_moe.so``.  There is no CPU or PyTorch fallback: if the
+library is missing, or a call returns an error status, a ``MoEError`` is raised.
+
+PyTorch is used for device memory (``tensor.data_ptr()``) and for the current
+CUDA stream; the functions below keep the names of the C entry points.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "liblexi_moe.so")
+
+MOE_F32, MOE_BF16 = 0, 1
+MOE_SCHED_AUTO, MOE_SCHED_SIMT, MOE_SCHED_DECODE, MOE_SCHED_PREFILL = 0, 1, 2, 3
+SCHEDULE_NAMES = {0: "auto", 1: "simt", 2: "decode", 3: "prefill"}
+
+EXPORTS = (
+    "moe_plan_create", "moe_plan_destroy", "moe_plan_workspace_bytes", "moe_plan_set_schedule",
+    "moe_plan_get_schedule", "moe_layer_forward", "moe_layer_forward_host", "moe_stack_forward",
+    "moe_route_from_logits", "moe_last_routing", "moe_device_status", "moe_plan_launch_count",
+    "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
+)
+STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
+
+
+class MoEError(RuntimeError):
+    def __init__(self, where: str, status: int):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class moe_config_t(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int32), ("E", ctypes.c_int32), ("I", ctypes.c_int32),
+                ("I_shared", ctypes.c_int32), ("shared_gate", ctypes.c_int32),
+                ("max_T", ctypes.c_int32), ("max_k", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("routed_scale", ctypes.c_float)]
+
+
+class moe_layer_weights_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("router_W", "router_bias", "W_gate", "W_up", "W_down",
+                 "Ws_gate", "Ws_up", "Ws_down", "w_s")]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads ``liblexi_moe.so`` (built by ``paper_2509_02753_b200.build``); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise MoEError(f"CUDA library not built ({LIB_PATH}); run __graft_entry__.build()", -5)
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint64
+    P = ctypes.POINTER
+    lib.moe_plan_create.argtypes = [P(moe_config_t), P(vp)]
+    lib.moe_plan_destroy.argtypes = [vp]
+    lib.moe_plan_workspace_bytes.argtypes = [vp]
+    lib.moe_plan_workspace_bytes.restype = u64
+    lib.moe_plan_launch_count.argtypes = [vp]
+    lib.moe_plan_launch_count.restype = u64
+    lib.moe_plan_set_schedule.argtypes = [vp, i32]
+    lib.moe_plan_get_schedule.argtypes = [vp, i32, i32]
+    lib.moe_layer_forward.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, vp, vp]
+    lib.moe_layer_forward_host.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, vp, vp]
+    lib.moe_stack_forward.argtypes = [vp, vp, P(moe_layer_weights_t), i32, P(i32), i32, i32, vp]
+    lib.moe_route_from_logits.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+    lib.moe_last_routing.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.moe_device_status.argtypes = [vp, vp]
+    lib.moe_plan_set_stage_timing.argtypes = [vp, i32]
+    lib.moe_plan_stage_times.argtypes = [vp, P(ctypes.c_float), P(i32)]
+    lib.moe_status_string.argtypes = [ctypes.c_int]
+    lib.moe_status_string.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name not in ("moe_plan_workspace_bytes", "moe_plan_launch_count", "moe_status_string"):
+            getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    try:
+        return load_library().moe_status_string(int(status)).decode()
+    except MoEError:
+        return "library not loaded"
+
+
+def _check(where: str, status: int) -> None:
+    if status != 0:
+        raise MoEError(where, status)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream or None
+
+
+def _dtype_code(dtype: torch.dtype) -> int:
+    if dtype == torch.float32:
+        return MOE_F32
+    if dtype == torch.bfloat16:
+        return MOE_BF16
+    raise TypeError(f"plan dtype must be float32 or bfloat16, got {dtype}")
+
+
+def make_weights(w: Dict[str, Optional[torch.Tensor]]) -> moe_layer_weights_t:
+    """Packs a dict of contiguous CUDA tensors (keys as in ``moe_layer_weights_t``)."""
+    s = moe_layer_weights_t()
+    for name, _ in moe_layer_weights_t._fields_:
+        t = w.get(name)
+        if t is not None:
+            assert t.is_cuda and t.is_contiguous(), name
+        setattr(s, name, _ptr(t))
+    return s
+
+
+# ---- the C entry points, same names ------------------------------------------------------
+
+def moe_plan_create(d: int, E: int, I: int, max_T: int, max_k: int, dtype: torch.dtype, *,
+                    I_shared: int = 0, shared_gate: bool = False, routed_scale: float = 1.0) -> int:
+    cfg = moe_config_t(d, E, I, I_shared, int(shared_gate), max_T, max_k, _dtype_code(dtype),
+                       routed_scale)
+    out = ctypes.c_void_p()
+    _check("moe_plan_create", load_library().moe_plan_create(ctypes.byref(cfg), ctypes.byref(out)))
+    return out.value
+
+
+def moe_plan_destroy(plan: int) -> None:
+    _check("moe_plan_destroy", load_library().moe_plan_destroy(plan))
+
+
+def moe_plan_workspace_bytes(plan: int) -> int:
+    return int(load_library().moe_plan_workspace_bytes(plan))
+
+
+def moe_plan_launch_count(plan: int) -> int:
+    return int(load_library().moe_plan_launch_count(plan))
+
+
+def moe_plan_set_schedule(plan: int, schedule: int) -> None:
+    _check("moe_plan_set_schedule", load_library().moe_plan_set_schedule(plan, schedule))
+
+
+def moe_plan_get_schedule(plan: int, T: int, k_l: int) -> int:
+    return int(load_library().moe_plan_get_schedule(plan, T, k_l))
+
+
+def moe_layer_forward(plan: int, x: torch.Tensor, w: moe_layer_weights_t, k_l: int, renorm: bool,
+                      y: torch.Tensor, stream=None) -> None:
+    assert x.is_cuda and y.is_cuda and x.is_contiguous() and y.is_contiguous()
+    _check("moe_layer_forward",
+           load_library().moe_layer_forward(plan, x.data_ptr(), ctypes.byref(w), x.shape[0], k_l,
+                                            int(renorm), y.data_ptr(), _stream(stream)))
+
+
+def moe_layer_forward_host(plan: int, x_host: torch.Tensor, w: moe_layer_weights_t, k_l: int,
+                           renorm: bool, y_host: torch.Tensor, stream=None) -> None:
+    assert not x_host.is_cuda and not y_host.is_cuda
+    assert x_host.is_contiguous() and y_host.is_contiguous()
+    _check("moe_layer_forward_host",
+           load_library().moe_layer_forward_host(plan, x_host.data_ptr(), ctypes.byref(w),
+                                                 x_host.shape[0], k_l, int(renorm),
+                                                 y_host.data_ptr(), _stream(stream)))
+
+
+def moe_stack_forward(plan: int, h: torch.Tensor, layers: Sequence[moe_layer_weights_t],
+                      k_vec: Sequence[int], renorm: bool, stream=None) -> None:
+    assert h.is_cuda and h.is_contiguous() and len(layers) == len(k_vec)
+    n = len(layers)
+    arr = (moe_layer_weights_t * max(n, 1))(*layers)
+    kv = (ctypes.c_int32 * max(n, 1))(*[int(k) for k in k_vec])
+    _check("moe_stack_forward",
+           load_library().moe_stack_forward(plan, h.data_ptr(), arr, n, kv, int(renorm),
+                                            h.shape[0], _stream(stream)))
+
+
+def moe_route_from_logits(plan: int, logits: torch.Tensor, k_l: int, renorm: bool, stream=None):
+    """Returns (topk_idx [T,k], topk_w [T,k], counts [E], offsets [E+1], perm [T*k]) on the device."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+    T, E = logits.shape
+    dev = logits.device
+    idx = torch.empty((T, k_l), dtype=torch.int32, device=dev)
+    wts = torch.empty((T, k_l), dtype=torch.float32, device=dev)
+    counts = torch.empty((E,), dtype=torch.int32, device=dev)
+    offsets = torch.empty((E + 1,), dtype=torch.int32, device=dev)
+    perm = torch.empty((T * k_l,), dtype=torch.int32, device=dev)
+    _check("moe_route_from_logits",
+           load_library().moe_route_from_logits(plan, logits.data_ptr(), T, k_l, int(renorm),
+                                                idx.data_ptr(), wts.data_ptr(), counts.data_ptr(),
+                                                offsets.data_ptr(), perm.data_ptr(), _stream(stream)))
+    return idx, wts, counts, offsets, perm
+
+
+def moe_last_routing(plan: int, T: int, k_l: int, E: int, device, stream=None):
+    """Routing artefacts of the plan's latest layer call, plus its logits [T,E]."""
+    idx = torch.empty((T, k_l), dtype=torch.int32, device=device)
+    wts = torch.empty((T, k_l), dtype=torch.float32, device=device)
+    counts = torch.empty((E,), dtype=torch.int32, device=device)
+    offsets = torch.empty((E + 1,), dtype=torch.int32, device=device)
+    perm = torch.empty((T * k_l,), dtype=torch.int32, device=device)
+    logits = torch.empty((T, E), dtype=torch.float32, device=device)
+    _check("moe_last_routing",
+           load_library().moe_last_routing(plan, idx.data_ptr(), wts.data_ptr(), counts.data_ptr(),
+                                           offsets.data_ptr(), perm.data_ptr(), logits.data_ptr(),
+                                           _stream(stream)))
+    return idx, wts, counts, offsets, perm, logits
+
+
+def moe_plan_set_stage_timing(plan: int, enable: bool) -> None:
+    _check("moe_plan_set_stage_timing", load_library().moe_plan_set_stage_timing(plan, int(enable)))
+
+
+def moe_plan_stage_times(plan: int):
+    """(dict stage -> total ms, number of layer calls summed) since the last read."""
+    ms = (ctypes.c_float * 5)()
+    n = ctypes.c_int32()
+    _check("moe_plan_stage_times", load_library().moe_plan_stage_times(plan, ms, ctypes.byref(n)))
+    return {name: float(ms[i]) for i, name in enumerate(STAGE_NAMES)}, int(n.value)
+
+
+def moe_device_status(plan: int, stream=None) -> int:
+    return int(load_library().moe_device_status(plan, _stream(stream)))
+
+
+class MoEPlan:
+    """Owns one plan handle; a convenience wrapper over the functions above."""
+
+    def __init__(self, d: int, E: int, I: int, max_T: int, max_k: int, dtype: torch.dtype, *,
+                 I_shared: int = 0, shared_gate: bool = False, routed_scale: float = 1.0):
+        self.d, self.E, self.I, self.dtype = d, E, I, dtype
+        self.handle = moe_plan_create(d, E, I, max_T, max_k, dtype, I_shared=I_shared,
+                                      shared_gate=shared_gate, routed_scale=routed_scale)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            moe_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def set_schedule(self, schedule: int):
+        moe_plan_set_schedule(self.handle, schedule)
+
+    def schedule_for(self, T: int, k_l: int) -> int:
+        return moe_plan_get_schedule(self.handle, T, k_l)
+
+    def layer_forward(self, x, w, k_l, renorm, y=None, stream=None):
+        if y is None:
+            y = torch.empty_like(x)
+        moe_layer_forward(self.handle, x, w, k_l, renorm, y, stream)
+        return y
+
+    def stack_forward(self, h, layers, k_vec, renorm, stream=None):
+        moe_stack_forward(self.handle, h, layers, k_vec, renorm, stream)
+        return h
+
+    def route_from_logits(self, logits, k_l, renorm, stream=None):
+        return moe_route_from_logits(self.handle, logits, k_l, renorm, stream)
+
+    def last_routing(self, T, k_l, device="cuda", stream=None):
+        return moe_last_routing(self.handle, T, k_l, self.E, device, stream)
+
+    def device_status(self, stream=None) -> int:
+        return moe_device_status(self.handle, stream)
+
+    @property
+    def workspace_bytes(self) -> int:
+        return moe_plan_workspace_bytes(self.handle)
+
+    @property
+    def launch_count(self) -> int:
+        return moe_plan_launch_count(self.handle)

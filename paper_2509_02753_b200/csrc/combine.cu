@@ -1,0 +1,106 @@
+// Combine: the weighted sum over the active experts of Section 2,
+//     y[t] = routed_scale * sum_{j < k_l} g[t,j] * o[inv_perm[t*k_l + j]]  +  gamma[t] * o_shared[t],
+// taken in slot order j = 0..k_l-1 in fp32 and rounded once.  Expert outputs may arrive as
+// several partial-sum slabs (split-K of the down projection); slabs are added in slab order,
+// so the result does not depend on the order in which tiles finished.
+#include "moe_internal.h"
+
+namespace lexi {
+
+__device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ float4 ld4(const __nv_bfloat16 *p) {
+    const uint2 raw = *reinterpret_cast<const uint2 *>(p);
+    const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162 *>(&raw.x);
+    const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162 *>(&raw.y);
+    return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+}
+__device__ __forceinline__ void st4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+__device__ __forceinline__ void st4(__nv_bfloat16 *p, float4 v) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 raw;
+    raw.x = *reinterpret_cast<uint32_t *>(&lo);
+    raw.y = *reinterpret_cast<uint32_t *>(&hi);
+    *reinterpret_cast<uint2 *>(p) = raw;
+}
+
+template <typename OT>
+__device__ __forceinline__ float4 sum_slabs(const OT *base, int slabs, size_t stride, size_t off) {
+    float4 acc = ld4(base + off);
+    for (int s = 1; s < slabs; ++s) {
+        const float4 v = ld4(base + (size_t)s * stride + off);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    return acc;
+}
+
+// One thread per 4 consecutive features of one token.
+template <typename YT, typename OT>
+__global__ void __launch_bounds__(256) combine_kernel(CombineArgs a) {
+    const int vec_per_row = a.d / 4;
+    const size_t n_vec = (size_t)a.T * vec_per_row;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec;
+         i += (size_t)gridDim.x * blockDim.x) {
+        const int t = (int)(i / vec_per_row);
+        const int c = (int)(i % vec_per_row) * 4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j = 0; j < a.k; ++j) {
+            const float g = a.topk_w[(size_t)t * a.k + j];
+            const int r = a.inv_perm[(size_t)t * a.k + j];
+            const float4 v = sum_slabs((const OT *)a.o, a.o_slabs, a.o_slab_stride, (size_t)r * a.d + c);
+            acc.x = fmaf(g, v.x, acc.x); acc.y = fmaf(g, v.y, acc.y);
+            acc.z = fmaf(g, v.z, acc.z); acc.w = fmaf(g, v.w, acc.w);
+        }
+        acc.x *= a.routed_scale; acc.y *= a.routed_scale; acc.z *= a.routed_scale; acc.w *= a.routed_scale;
+        if (a.o_s) {
+            const float gm = a.gamma ? a.gamma[t] : 1.0f;
+            const float4 v = sum_slabs((const OT *)a.o_s, a.os_slabs, a.os_slab_stride, (size_t)t * a.d + c);
+            acc.x = fmaf(gm, v.x, acc.x); acc.y = fmaf(gm, v.y, acc.y);
+            acc.z = fmaf(gm, v.z, acc.z); acc.w = fmaf(gm, v.w, acc.w);
+        }
+        const size_t off = (size_t)t * a.d + c;
+        YT *y = (YT *)a.y;
+        if (a.mode == 0) {
+            st4(y + off, acc);
+        } else if (a.mode == 1) {          // residual stream kept in fp32 beside the rounded copy
+            float4 hrun = ld4(a.h_run + off);
+            hrun.x += acc.x; hrun.y += acc.y; hrun.z += acc.z; hrun.w += acc.w;
+            st4(a.h_run + off, hrun);
+            st4(y + off, hrun);
+        } else {                           // y is the residual stream itself
+            float4 hv = ld4(y + off);
+            hv.x += acc.x; hv.y += acc.y; hv.z += acc.z; hv.w += acc.w;
+            st4(y + off, hv);
+        }
+    }
+}
+
+cudaError_t launch_combine(const CombineArgs &a, cudaStream_t s, uint64_t *launches) {
+    if (a.T <= 0) return cudaSuccess;
+    const size_t n_vec = (size_t)a.T * (a.d / 4);
+    const int grid = (int)min((n_vec + 255) / 256, (size_t)148 * 16);
+    const bool y_bf16 = a.dtype == MOE_BF16;
+    if (y_bf16 && a.o_is_f32) combine_kernel<__nv_bfloat16, float><<<grid, 256, 0, s>>>(a);
+    else if (y_bf16) combine_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, s>>>(a);
+    else combine_kernel<float, float><<<grid, 256, 0, s>>>(a);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) widen_kernel(const T *src, float *dst, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+         i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = (float)src[i];
+}
+
+cudaError_t launch_widen(const void *src, float *dst, size_t n, int dtype, cudaStream_t s,
+                         uint64_t *launches) {
+    if (n == 0) return cudaSuccess;
+    const int grid = (int)min((n + 255) / 256, (size_t)148 * 16);
+    if (dtype == MOE_BF16) widen_kernel<<<grid, 256, 0, s>>>((const __nv_bfloat16 *)src, dst, n);
+    else widen_kernel<<<grid, 256, 0, s>>>((const float *)src, dst, n);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace lexi

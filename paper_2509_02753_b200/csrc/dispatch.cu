@@ -1,0 +1,135 @@
+// Dispatch: group the (token, slot) pairs by expert.  The paper (Introduction; Section 3)
+// only says that tokens are routed to their top-k experts and that the per-expert token load
+// decides the time; the tables built here are the integer definition of that grouping:
+//   counts[e], offsets = exclusive scan, perm = pairs in expert-major order with ascending
+//   token inside an expert (a stable counting sort), inv_perm = its inverse,
+// followed by the gather of the token rows into that order.
+//
+// Everything is deterministic: ranks come from warp ballots over pairs taken in order, never
+// from the arrival order of atomics.
+#include "moe_internal.h"
+
+namespace lexi {
+
+// Each warp owns kPairsPerPart consecutive pairs.  Pass 1: histogram of the part.
+__global__ void __launch_bounds__(256) dispatch_count_kernel(DispatchArgs a, int n_pairs, int n_parts) {
+    __shared__ int32_t hist[8][kMaxExperts];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int part = blockIdx.x * 8 + warp;
+    for (int e = lane; e < a.E; e += 32) hist[warp][e] = 0;
+    __syncwarp();
+    if (part < n_parts) {
+        const int p0 = part * kPairsPerPart;
+        const int p1 = min(p0 + kPairsPerPart, n_pairs);
+        for (int p = p0 + lane; p < p1; p += 32) {
+            const int e = a.topk_idx[p];
+            if ((unsigned)e < (unsigned)a.E) atomicAdd(&hist[warp][e], 1);
+            else atomicOr(a.status, kStatusBadIndex);
+        }
+        __syncwarp();
+        for (int e = lane; e < a.E; e += 32) a.part_hist[(size_t)part * a.E + e] = hist[warp][e];
+    }
+}
+
+// Pass 2 (one block): counts, offsets, and for every (part, expert) the first output row.
+__global__ void __launch_bounds__(kMaxExperts) dispatch_scan_kernel(DispatchArgs a, int n_parts) {
+    __shared__ int32_t cnt[kMaxExperts];
+    __shared__ int32_t off[kMaxExperts + 1];
+    const int e = threadIdx.x;
+    int total = 0;
+    if (e < a.E)
+        for (int p = 0; p < n_parts; ++p) total += a.part_hist[(size_t)p * a.E + e];
+    cnt[e] = (e < a.E) ? total : 0;
+    __syncthreads();
+    if (e == 0) {
+        int run = 0;
+        for (int i = 0; i < a.E; ++i) { off[i] = run; run += cnt[i]; }
+        off[a.E] = run;
+    }
+    __syncthreads();
+    if (e < a.E) {
+        a.counts[e] = cnt[e];
+        a.offsets[e] = off[e];
+        int run = off[e];
+        for (int p = 0; p < n_parts; ++p) {
+            const int c = a.part_hist[(size_t)p * a.E + e];
+            a.part_hist[(size_t)p * a.E + e] = run;
+            run += c;
+        }
+    }
+    if (e == 0) a.offsets[a.E] = off[a.E];
+}
+
+// Pass 3: each warp walks its part in order, 32 pairs at a time; pairs of the same expert
+// inside a step are ranked by lane (ballot), across steps by a per-warp cursor.
+__global__ void __launch_bounds__(256) dispatch_scatter_kernel(DispatchArgs a, int n_pairs, int n_parts) {
+    __shared__ int32_t cursor[8][kMaxExperts];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int part = blockIdx.x * 8 + warp;
+    if (part >= n_parts) return;
+    for (int e = lane; e < a.E; e += 32) cursor[warp][e] = a.part_hist[(size_t)part * a.E + e];
+    __syncwarp();
+    const int p0 = part * kPairsPerPart;
+    const int p1 = min(p0 + kPairsPerPart, n_pairs);
+    for (int base = p0; base < p1; base += 32) {
+        const int p = base + lane;
+        const bool valid = p < p1;
+        int e = valid ? a.topk_idx[p] : -1;
+        if (valid && (unsigned)e >= (unsigned)a.E) e = -1;
+        const unsigned peers = __match_any_sync(0xffffffffu, e);
+        const int rank = __popc(peers & ((1u << lane) - 1u));
+        const int leader = __ffs(peers) - 1;
+        int first = 0;
+        if (e >= 0 && lane == leader) {
+            first = cursor[warp][e];
+            cursor[warp][e] = first + __popc(peers);
+        }
+        first = __shfl_sync(0xffffffffu, first, leader);
+        if (e >= 0) {
+            const int r = first + rank;
+            a.perm[r] = p;
+            a.inv_perm[p] = r;
+        }
+        __syncwarp();
+    }
+}
+
+cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches) {
+    const int n_pairs = a.T * a.k;
+    if (n_pairs <= 0) return cudaSuccess;
+    const int n_parts = (n_pairs + kPairsPerPart - 1) / kPairsPerPart;
+    const int grid = (n_parts + 7) / 8;
+    dispatch_count_kernel<<<grid, 256, 0, s>>>(a, n_pairs, n_parts);
+    dispatch_scan_kernel<<<1, kMaxExperts, 0, s>>>(a, n_parts);
+    dispatch_scatter_kernel<<<grid, 256, 0, s>>>(a, n_pairs, n_parts);
+    *launches += 3;
+    return cudaGetLastError();
+}
+
+// Gather: x_perm[r, :] = x[perm[r] / k, :], one warp per row, 16-byte loads and stores.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const uint4 *__restrict__ x,
+                                                          const int32_t *__restrict__ perm,
+                                                          int n_rows, int k, int vec_per_row,
+                                                          uint4 *__restrict__ x_perm) {
+    const int lane = threadIdx.x & 31;
+    const int warps = gridDim.x * 8;
+    for (int r = blockIdx.x * 8 + (threadIdx.x >> 5); r < n_rows; r += warps) {
+        const int t = perm[r] / k;
+        const uint4 *src = x + (size_t)t * vec_per_row;
+        uint4 *dst = x_perm + (size_t)r * vec_per_row;
+        for (int v = lane; v < vec_per_row; v += 32) dst[v] = src[v];
+    }
+}
+
+cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k, int d, int dtype,
+                          void *x_perm, cudaStream_t s, uint64_t *launches) {
+    if (n_rows <= 0) return cudaSuccess;
+    const int bytes_per_row = d * (dtype == MOE_BF16 ? 2 : 4);
+    const int grid = min((n_rows + 7) / 8, 148 * 8);
+    gather_rows_kernel<<<grid, 256, 0, s>>>((const uint4 *)x, perm, n_rows, k, bytes_per_row / 16,
+                                            (uint4 *)x_perm);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace lexi

@@ -1,0 +1,34 @@
+// Tensor-core (tcgen05 / TMEM / TMA) schedules of the expert FFNs: host-side interface.
+#pragma once
+
+#include "moe_internal.h"
+
+namespace lexi {
+
+struct TcState {
+    void *encode_fn = nullptr;   // cuTensorMapEncodeTiled, resolved through the runtime
+    int max_smem_optin = 0;
+    bool ready = false;
+};
+
+// How the combine step has to read the expert outputs a schedule produced.
+struct TcOutputLayout {
+    int o_is_f32 = 1;
+    int o_slabs = 1;
+    size_t o_slab_stride = 0;
+    int os_slabs = 1;
+    size_t os_slab_stride = 0;
+};
+
+bool   tc_shape_ok(const moe_config_t &c);
+int    tc_max_slabs(const moe_config_t &c);          // most split-K slabs of the routed output
+int    tc_max_shared_slabs(const moe_config_t &c);   // ... of the shared-expert output
+size_t tc_o_elems(const moe_config_t &c, int slabs);     // fp32-sized elements to hold `o`
+size_t tc_os_elems(const moe_config_t &c, int slabs);    // ... `o_s`
+size_t tc_max_tiles(const moe_config_t &c, int phase);   // capacity of a tile list
+int    tc_state_init(TcState *st, const moe_config_t &c);
+int    tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, const FfnArgs &a,
+                      int schedule, int sm_count, cudaStream_t s, uint64_t *launches,
+                      TcOutputLayout *layout);
+
+}  // namespace lexi

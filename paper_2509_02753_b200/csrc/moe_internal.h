@@ -1,0 +1,105 @@
+// Internal declarations shared by the translation units of the CUDA library.
+// Nothing here is part of the C ABI (that is include/moe.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "moe.h"
+
+namespace lexi {
+
+constexpr int kMaxExperts = 128;      // router holds a row of logits in one warp, 4 per lane
+constexpr int kExpertsPerLane = 4;
+constexpr int kPairsPerPart = 256;    // (token, slot) pairs ranked by one warp in dispatch
+constexpr int kTileRows = 128;        // token rows of one tensor-core tile (UMMA M)
+
+// bits of the device status word
+constexpr int kStatusTimeout = 1;
+constexpr int kStatusBadIndex = 2;
+
+// One unit of work of the tensor-core grouped GEMMs.  Built on the device from the
+// per-expert counts, consumed by the persistent GEMM kernels.
+struct __align__(16) Tile {
+    int32_t group;     // expert id, or E for the shared expert
+    int32_t row0;      // first row of the activation operand (expert-ordered, or token id)
+    int32_t rows;      // valid rows, 1..128
+    int32_t n0;        // first output feature (phase 1: first row of W_gate/W_up; phase 2: row of W_down)
+    int32_t k0;        // first element of the reduction range
+    int32_t klen;      // length of the reduction range
+    int32_t slot;      // which partial-sum slab of the output this tile writes (split-K)
+    int32_t pad;
+};
+
+struct Workspace {
+    float   *logits = nullptr;     // [max_T, E]
+    int32_t *topk_idx = nullptr;   // [max_T * max_k]
+    float   *topk_w = nullptr;     // [max_T * max_k]
+    int32_t *counts = nullptr;     // [E]
+    int32_t *offsets = nullptr;    // [E + 1]
+    int32_t *perm = nullptr;       // [max_T * max_k]
+    int32_t *inv_perm = nullptr;   // [max_T * max_k]
+    int32_t *part_hist = nullptr;  // [n_parts, E] per-partition histogram, then write cursors
+    float   *gamma = nullptr;      // [max_T] shared-expert gate
+    void    *x_perm = nullptr;     // [max_T * max_k, d]
+    void    *h = nullptr;          // [max_T * max_k, I]
+    void    *h_s = nullptr;        // [max_T, I_s]
+    void    *o = nullptr;          // routed expert outputs (layout depends on the schedule)
+    void    *o_s = nullptr;        // shared expert output
+    float   *h_run = nullptr;      // [max_T, d] fp32 residual stream of the stack (bf16 plans)
+    void    *x_stage = nullptr;    // [max_T, d] staging for the host-buffer entry point
+    void    *y_stage = nullptr;    // [max_T, d]
+    int32_t *status = nullptr;     // device status word
+    Tile    *tiles1 = nullptr;     // phase-1 tile list
+    Tile    *tiles2 = nullptr;     // phase-2 tile list
+    int32_t *n_tiles = nullptr;    // [2] tile counts
+    int32_t *ticket = nullptr;     // block-arrival counter of the fused small-T router
+};
+
+// ---- launchers (each returns the cudaError_t of its launches) -------------------------
+
+struct RouterArgs {
+    const void *x; const void *W; const float *bias; const void *w_s;
+    int T, d, E, k, renorm, dtype;
+    float *logits; int32_t *topk_idx; float *topk_w; float *gamma;
+};
+cudaError_t launch_router(const RouterArgs &a, cudaStream_t s, uint64_t *launches);
+cudaError_t launch_route_from_logits(const float *logits, int T, int E, int k, int renorm,
+                                     int32_t *topk_idx, float *topk_w, cudaStream_t s,
+                                     uint64_t *launches);
+
+struct DispatchArgs {
+    const int32_t *topk_idx; int T, k, E;
+    int32_t *counts, *offsets, *perm, *inv_perm, *part_hist; int32_t *status;
+};
+cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches);
+cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k, int d, int dtype,
+                          void *x_perm, cudaStream_t s, uint64_t *launches);
+
+struct FfnArgs {
+    int dtype, T, k, d, E, I, I_s;
+    const int32_t *counts, *offsets;
+    const void *x, *x_perm;
+    const void *W_gate, *W_up, *W_down, *Ws_gate, *Ws_up, *Ws_down;
+    void *h, *h_s, *o, *o_s;
+    cudaEvent_t mid_event;   // recorded between the two GEMM phases when not null
+};
+cudaError_t launch_ffn_simt(const FfnArgs &a, cudaStream_t s, uint64_t *launches);
+
+struct CombineArgs {
+    int dtype, T, k, d;
+    const float *topk_w; const int32_t *inv_perm; const float *gamma;  // gamma NULL: factor 1
+    const void *o; int o_is_f32; int o_slabs; size_t o_slab_stride;    // routed outputs
+    const void *o_s; int os_slabs; size_t os_slab_stride;              // shared outputs (NULL: none)
+    float routed_scale;
+    void *y;           // mode 0: y = result.  mode 1: h_run += result, y = round(h_run).  mode 2: y += result
+    float *h_run;
+    int mode;
+};
+cudaError_t launch_combine(const CombineArgs &a, cudaStream_t s, uint64_t *launches);
+
+cudaError_t launch_widen(const void *src, float *dst, size_t n, int dtype, cudaStream_t s,
+                         uint64_t *launches);
+
+}  // namespace lexi

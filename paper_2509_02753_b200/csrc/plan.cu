@@ -1,0 +1,393 @@
+// C ABI of the library (include/moe.h): plan, workspace, and the host-side sequencing of the
+// kernels of one MoE layer and of a stack of layers with a per-layer k vector.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "ffn_tc.h"
+#include "moe_internal.h"
+
+using namespace lexi;
+
+struct moe_plan {
+    moe_config_t cfg{};
+    Workspace ws{};
+    std::vector<void *> allocs;
+    uint64_t bytes = 0;
+    uint64_t launches = 0;
+    int32_t forced_schedule = MOE_SCHED_AUTO;
+    int32_t last_T = 0, last_k = 0;
+    int32_t *status_host = nullptr;   // pinned
+    int sm_count = 148;
+    TcState tc{};
+    // stage timing: kMaxTimedCalls sets of MOE_N_STAGES + 1 events
+    bool timing = false;
+    std::vector<cudaEvent_t> events;
+    int timed_calls = 0;
+};
+
+constexpr int kMaxTimedCalls = 256;
+
+namespace {
+
+size_t elem_size(int dtype) { return dtype == MOE_BF16 ? 2 : 4; }
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename T>
+bool ws_alloc(moe_plan *p, T **out, size_t count, size_t elem = sizeof(T)) {
+    size_t bytes = count * elem;
+    bytes = (bytes + 255) & ~size_t(255);
+    if (bytes == 0) bytes = 256;
+    void *ptr = nullptr;
+    if (cudaMalloc(&ptr, bytes) != cudaSuccess) { cudaGetLastError(); return false; }
+    p->allocs.push_back(ptr);
+    p->bytes += bytes;
+    *out = reinterpret_cast<T *>(ptr);
+    return true;
+}
+
+int check_weights(const moe_plan *p, const moe_layer_weights_t *w) {
+    if (!w || !w->router_W || !w->W_gate || !w->W_up || !w->W_down) return MOE_ERR_INVALID_ARG;
+    if (p->cfg.I_shared > 0) {
+        if (!w->Ws_gate || !w->Ws_up || !w->Ws_down) return MOE_ERR_INVALID_ARG;
+        if (p->cfg.shared_gate && !w->w_s) return MOE_ERR_INVALID_ARG;
+    }
+    const void *ptrs[] = {w->router_W, w->router_bias, w->W_gate, w->W_up, w->W_down,
+                          w->Ws_gate, w->Ws_up, w->Ws_down, w->w_s};
+    for (const void *q : ptrs)
+        if (q && !aligned16(q)) return MOE_ERR_ALIGN;
+    return MOE_OK;
+}
+
+int pick_schedule(const moe_plan *p, int T, int k) {
+    if (p->forced_schedule != MOE_SCHED_AUTO) return p->forced_schedule;
+    if (p->cfg.dtype != MOE_BF16 || !tc_shape_ok(p->cfg)) return MOE_SCHED_SIMT;
+    return ((int64_t)T * k < (int64_t)16 * p->cfg.E) ? MOE_SCHED_DECODE : MOE_SCHED_PREFILL;
+}
+
+// mode 0: y = MoE(x).  mode 1: h_run += MoE(x), y = round(h_run) (y may be x).  mode 2: y += MoE(x), y == x.
+int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, int k, int renorm,
+               void *y, int mode, cudaStream_t s) {
+    const moe_config_t &c = p->cfg;
+    Workspace &ws = p->ws;
+    cudaError_t err;
+    cudaEvent_t *ev = nullptr;      // this call's MOE_N_STAGES + 1 boundary events, if timed
+    if (p->timing && p->timed_calls < kMaxTimedCalls)
+        ev = &p->events[(size_t)p->timed_calls++ * (MOE_N_STAGES + 1)];
+    auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], s); };
+    mark(0);
+
+    RouterArgs ra{x, w->router_W, w->router_bias, (c.I_shared > 0 && c.shared_gate) ? w->w_s : nullptr,
+                  T, c.d, c.E, k, renorm, c.dtype, ws.logits, ws.topk_idx, ws.topk_w, ws.gamma};
+    if ((err = launch_router(ra, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
+    mark(1);
+
+    DispatchArgs da{ws.topk_idx, T, k, c.E, ws.counts, ws.offsets, ws.perm, ws.inv_perm,
+                    ws.part_hist, ws.status};
+    if ((err = launch_dispatch(da, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
+    if ((err = launch_gather(x, ws.perm, T * k, k, c.d, c.dtype, ws.x_perm, s, &p->launches)) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    mark(2);
+
+    FfnArgs fa{c.dtype, T, k, c.d, c.E, c.I, c.I_shared, ws.counts, ws.offsets, x, ws.x_perm,
+               w->W_gate, w->W_up, w->W_down, w->Ws_gate, w->Ws_up, w->Ws_down,
+               ws.h, ws.h_s, ws.o, ws.o_s, ev ? ev[3] : nullptr};
+    const int sched = pick_schedule(p, T, k);
+    CombineArgs ca{};
+    ca.dtype = c.dtype; ca.T = T; ca.k = k; ca.d = c.d;
+    ca.topk_w = ws.topk_w; ca.inv_perm = ws.inv_perm;
+    ca.gamma = (c.I_shared > 0 && c.shared_gate) ? ws.gamma : nullptr;
+    ca.o = ws.o; ca.o_s = c.I_shared > 0 ? ws.o_s : nullptr;
+    ca.routed_scale = c.routed_scale; ca.y = y; ca.h_run = ws.h_run; ca.mode = mode;
+    if (sched == MOE_SCHED_SIMT) {
+        if ((err = launch_ffn_simt(fa, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
+        ca.o_is_f32 = 1; ca.o_slabs = 1; ca.o_slab_stride = 0; ca.os_slabs = 1; ca.os_slab_stride = 0;
+    } else {
+        TcOutputLayout lay{};
+        const int rc = tc_ffn_forward(&p->tc, c, ws, fa, sched, p->sm_count, s, &p->launches, &lay);
+        if (rc != MOE_OK) return rc;
+        ca.o_is_f32 = lay.o_is_f32; ca.o_slabs = lay.o_slabs; ca.o_slab_stride = lay.o_slab_stride;
+        ca.os_slabs = lay.os_slabs; ca.os_slab_stride = lay.os_slab_stride;
+    }
+    mark(4);
+    if ((err = launch_combine(ca, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
+    mark(5);
+    p->last_T = T;
+    p->last_k = k;
+    return MOE_OK;
+}
+
+int check_call(const moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, int k, const void *y) {
+    if (!p || !x || !y) return MOE_ERR_INVALID_ARG;
+    if (T < 0 || T > p->cfg.max_T || k < 1 || k > p->cfg.max_k) return MOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y)) return MOE_ERR_ALIGN;
+    return check_weights(p, w);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *moe_status_string(int status) {
+    switch (status) {
+        case MOE_OK: return "ok";
+        case MOE_ERR_INVALID_ARG: return "invalid argument";
+        case MOE_ERR_SHAPE: return "unsupported shape";
+        case MOE_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case MOE_ERR_WORKSPACE: return "workspace allocation failed";
+        case MOE_ERR_CUDA: return "CUDA call failed";
+        case MOE_ERR_TIMEOUT: return "device-side wait timed out";
+        case MOE_ERR_NOT_IMPLEMENTED: return "not implemented";
+        case MOE_ERR_DEVICE_CHECK: return "device-side index check failed";
+        default: return "unknown status";
+    }
+}
+
+int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
+    if (out) *out = nullptr;
+    if (!cfg || !out) return MOE_ERR_INVALID_ARG;
+    if (cfg->dtype != MOE_F32 && cfg->dtype != MOE_BF16) return MOE_ERR_INVALID_ARG;
+    if (cfg->d < 8 || cfg->E < 1 || cfg->I < 8 || cfg->I_shared < 0 || cfg->max_T < 1 ||
+        cfg->max_k < 1 || cfg->max_k > cfg->E)
+        return MOE_ERR_INVALID_ARG;
+    if (cfg->shared_gate != 0 && cfg->shared_gate != 1) return MOE_ERR_INVALID_ARG;
+    if (cfg->d % 8 || cfg->I % 8 || cfg->I_shared % 8) return MOE_ERR_SHAPE;
+    if (cfg->E + (cfg->I_shared > 0 && cfg->shared_gate ? 1 : 0) > kMaxExperts) return MOE_ERR_SHAPE;
+    if (cfg->d > 8192) return MOE_ERR_SHAPE;
+    if ((int64_t)cfg->max_T * cfg->max_k > (int64_t)1 << 24) return MOE_ERR_SHAPE;
+
+    int dev = 0, major = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    if (major != 10) return MOE_ERR_CUDA;   // the kernels are sm_100a only
+
+    moe_plan *p = new (std::nothrow) moe_plan();
+    if (!p) return MOE_ERR_WORKSPACE;
+    p->cfg = *cfg;
+    p->sm_count = sms;
+    const moe_config_t &c = p->cfg;
+    Workspace &ws = p->ws;
+    const size_t es = elem_size(c.dtype);
+    const size_t pairs = (size_t)c.max_T * c.max_k;
+    const size_t n_parts = (pairs + kPairsPerPart - 1) / kPairsPerPart;
+    const int slabs = tc_max_slabs(c);
+    const int slabs_s = tc_max_shared_slabs(c);
+    bool ok = true;
+    ok = ok && ws_alloc(p, &ws.logits, (size_t)c.max_T * c.E);
+    ok = ok && ws_alloc(p, &ws.topk_idx, pairs);
+    ok = ok && ws_alloc(p, &ws.topk_w, pairs);
+    ok = ok && ws_alloc(p, &ws.counts, (size_t)c.E);
+    ok = ok && ws_alloc(p, &ws.offsets, (size_t)c.E + 1);
+    ok = ok && ws_alloc(p, &ws.perm, pairs);
+    ok = ok && ws_alloc(p, &ws.inv_perm, pairs);
+    ok = ok && ws_alloc(p, &ws.part_hist, n_parts * c.E);
+    ok = ok && ws_alloc(p, &ws.gamma, (size_t)c.max_T);
+    ok = ok && ws_alloc(p, &ws.x_perm, pairs * c.d + 128 * (size_t)c.d, es);
+    ok = ok && ws_alloc(p, &ws.h, pairs * c.I + 128 * (size_t)c.I, es);
+    ok = ok && ws_alloc(p, &ws.h_s, (size_t)c.max_T * c.I_shared + 128 * (size_t)c.I_shared, es);
+    // expert outputs: fp32 partial-sum slabs when the decode schedule splits K, else one slab
+    const size_t o_elems = tc_o_elems(c, slabs);
+    const size_t os_elems = tc_os_elems(c, slabs_s);
+    ok = ok && ws_alloc(p, &ws.o, o_elems, 4);
+    ok = ok && ws_alloc(p, &ws.o_s, c.I_shared > 0 ? os_elems : 0, 4);
+    ok = ok && ws_alloc(p, &ws.h_run, (size_t)c.max_T * c.d);
+    ok = ok && ws_alloc(p, &ws.x_stage, (size_t)c.max_T * c.d, es);
+    ok = ok && ws_alloc(p, &ws.y_stage, (size_t)c.max_T * c.d, es);
+    ok = ok && ws_alloc(p, &ws.status, (size_t)4);
+    ok = ok && ws_alloc(p, &ws.tiles1, tc_max_tiles(c, 1));
+    ok = ok && ws_alloc(p, &ws.tiles2, tc_max_tiles(c, 2));
+    ok = ok && ws_alloc(p, &ws.n_tiles, (size_t)4);
+    ok = ok && ws_alloc(p, &ws.ticket, (size_t)4);
+    if (ok && cudaMallocHost(&p->status_host, sizeof(int32_t)) != cudaSuccess) { cudaGetLastError(); ok = false; }
+    if (ok) {
+        ok = cudaMemset(ws.status, 0, 16) == cudaSuccess && cudaMemset(ws.ticket, 0, 16) == cudaSuccess &&
+             cudaMemset(ws.n_tiles, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        moe_plan_destroy(p);
+        return MOE_ERR_WORKSPACE;
+    }
+    const int rc = tc_state_init(&p->tc, c);
+    if (rc != MOE_OK) { moe_plan_destroy(p); return rc; }
+    *out = p;
+    return MOE_OK;
+}
+
+int moe_plan_destroy(moe_plan_t *p) {
+    if (!p) return MOE_OK;
+    cudaDeviceSynchronize();
+    for (void *q : p->allocs) cudaFree(q);
+    for (cudaEvent_t e : p->events) cudaEventDestroy(e);
+    if (p->status_host) cudaFreeHost(p->status_host);
+    cudaGetLastError();
+    delete p;
+    return MOE_OK;
+}
+
+uint64_t moe_plan_workspace_bytes(const moe_plan_t *p) { return p ? p->bytes : 0; }
+uint64_t moe_plan_launch_count(const moe_plan_t *p) { return p ? p->launches : 0; }
+
+int moe_plan_set_schedule(moe_plan_t *p, int32_t schedule) {
+    if (!p || schedule < MOE_SCHED_AUTO || schedule > MOE_SCHED_PREFILL) return MOE_ERR_INVALID_ARG;
+    if ((schedule == MOE_SCHED_DECODE || schedule == MOE_SCHED_PREFILL) &&
+        (p->cfg.dtype != MOE_BF16 || !tc_shape_ok(p->cfg)))
+        return MOE_ERR_SHAPE;
+    p->forced_schedule = schedule;
+    return MOE_OK;
+}
+
+int moe_plan_set_stage_timing(moe_plan_t *p, int32_t enable) {
+    if (!p) return MOE_ERR_INVALID_ARG;
+    if (enable && p->events.empty()) {
+        p->events.resize((size_t)kMaxTimedCalls * (MOE_N_STAGES + 1));
+        for (cudaEvent_t &e : p->events)
+            if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    } else if (!enable) {
+        for (cudaEvent_t e : p->events) cudaEventDestroy(e);
+        p->events.clear();
+    }
+    p->timing = enable != 0;
+    p->timed_calls = 0;
+    return MOE_OK;
+}
+
+int moe_plan_stage_times(moe_plan_t *p, float *ms, int32_t *n_calls) {
+    if (!p || !ms || !n_calls) return MOE_ERR_INVALID_ARG;
+    for (int i = 0; i < MOE_N_STAGES; ++i) ms[i] = 0.f;
+    *n_calls = p->timed_calls;
+    for (int c = 0; c < p->timed_calls; ++c) {
+        cudaEvent_t *ev = &p->events[(size_t)c * (MOE_N_STAGES + 1)];
+        if (cudaEventSynchronize(ev[MOE_N_STAGES]) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+        for (int i = 0; i < MOE_N_STAGES; ++i) {
+            float t = 0.f;
+            if (cudaEventElapsedTime(&t, ev[i], ev[i + 1]) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+            ms[i] += t;
+        }
+    }
+    p->timed_calls = 0;
+    return MOE_OK;
+}
+
+int moe_plan_get_schedule(const moe_plan_t *p, int32_t T, int32_t k_l) {
+    if (!p) return MOE_ERR_INVALID_ARG;
+    return pick_schedule(p, T, k_l);
+}
+
+int moe_layer_forward(moe_plan_t *p, const void *x, const moe_layer_weights_t *w, int32_t T,
+                      int32_t k_l, int32_t renorm, void *y, void *cuda_stream) {
+    const int rc = check_call(p, x, w, T, k_l, y);
+    if (rc != MOE_OK) return rc;
+    if (x == y) return MOE_ERR_INVALID_ARG;
+    if (T == 0) return MOE_OK;
+    return layer_impl(p, x, w, T, k_l, renorm ? 1 : 0, y, 0, (cudaStream_t)cuda_stream);
+}
+
+int moe_layer_forward_host(moe_plan_t *p, const void *x_host, const moe_layer_weights_t *w, int32_t T,
+                           int32_t k_l, int32_t renorm, void *y_host, void *cuda_stream) {
+    if (!p || !x_host || !y_host) return MOE_ERR_INVALID_ARG;
+    if (T < 0 || T > p->cfg.max_T || k_l < 1 || k_l > p->cfg.max_k) return MOE_ERR_INVALID_ARG;
+    int rc = check_weights(p, w);
+    if (rc != MOE_OK) return rc;
+    if (T == 0) return MOE_OK;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const size_t bytes = (size_t)T * p->cfg.d * elem_size(p->cfg.dtype);
+    if (cudaMemcpyAsync(p->ws.x_stage, x_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    rc = layer_impl(p, p->ws.x_stage, w, T, k_l, renorm ? 1 : 0, p->ws.y_stage, 0, s);
+    if (rc != MOE_OK) return rc;
+    if (cudaMemcpyAsync(y_host, p->ws.y_stage, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    return MOE_OK;
+}
+
+int moe_stack_forward(moe_plan_t *p, void *h, const moe_layer_weights_t *layers, int32_t n_layers,
+                      const int32_t *k_vec, int32_t renorm, int32_t T, void *cuda_stream) {
+    if (!p || !h || !layers || !k_vec || n_layers < 0) return MOE_ERR_INVALID_ARG;
+    if (T < 0 || T > p->cfg.max_T) return MOE_ERR_INVALID_ARG;
+    if (!aligned16(h)) return MOE_ERR_ALIGN;
+    for (int l = 0; l < n_layers; ++l) {
+        if (k_vec[l] < 1 || k_vec[l] > p->cfg.max_k) return MOE_ERR_INVALID_ARG;
+        const int rc = check_weights(p, &layers[l]);
+        if (rc != MOE_OK) return rc;
+    }
+    if (T == 0 || n_layers == 0) return MOE_OK;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const bool bf16 = p->cfg.dtype == MOE_BF16;
+    if (bf16 && launch_widen(h, p->ws.h_run, (size_t)T * p->cfg.d, MOE_BF16, s, &p->launches) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    for (int l = 0; l < n_layers; ++l) {
+        const int rc = layer_impl(p, h, &layers[l], T, k_vec[l], renorm ? 1 : 0, h, bf16 ? 1 : 2, s);
+        if (rc != MOE_OK) return rc;
+    }
+    return MOE_OK;
+}
+
+int moe_route_from_logits(moe_plan_t *p, const float *logits, int32_t T, int32_t k_l, int32_t renorm,
+                          int32_t *topk_idx, float *topk_w, int32_t *counts, int32_t *offsets,
+                          int32_t *perm, void *cuda_stream) {
+    if (!p || !logits) return MOE_ERR_INVALID_ARG;
+    if (T < 0 || T > p->cfg.max_T || k_l < 1 || k_l > p->cfg.max_k) return MOE_ERR_INVALID_ARG;
+    if (T == 0) return MOE_OK;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    Workspace &ws = p->ws;
+    const int E = p->cfg.E;
+    if (launch_route_from_logits(logits, T, E, k_l, renorm ? 1 : 0, ws.topk_idx, ws.topk_w, s,
+                                 &p->launches) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    DispatchArgs da{ws.topk_idx, T, k_l, E, ws.counts, ws.offsets, ws.perm, ws.inv_perm, ws.part_hist, ws.status};
+    if (launch_dispatch(da, s, &p->launches) != cudaSuccess) return MOE_ERR_CUDA;
+    cudaMemcpyAsync(ws.logits, logits, (size_t)T * E * sizeof(float), cudaMemcpyDeviceToDevice, s);
+    p->last_T = T;
+    p->last_k = k_l;
+    return moe_last_routing(p, topk_idx, topk_w, counts, offsets, perm, nullptr, cuda_stream);
+}
+
+int moe_last_routing(moe_plan_t *p, int32_t *topk_idx, float *topk_w, int32_t *counts, int32_t *offsets,
+                     int32_t *perm, float *logits, void *cuda_stream) {
+    if (!p) return MOE_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const Workspace &ws = p->ws;
+    const size_t pairs = (size_t)p->last_T * p->last_k;
+    const int E = p->cfg.E;
+    cudaError_t e = cudaSuccess;
+    auto cp = [&](void *dst, const void *src, size_t bytes) {
+        if (dst && bytes && e == cudaSuccess) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, s);
+    };
+    cp(topk_idx, ws.topk_idx, pairs * 4);
+    cp(topk_w, ws.topk_w, pairs * 4);
+    cp(counts, ws.counts, (size_t)E * 4);
+    cp(offsets, ws.offsets, (size_t)(E + 1) * 4);
+    cp(perm, ws.perm, pairs * 4);
+    cp(logits, ws.logits, (size_t)p->last_T * E * 4);
+    if (e != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    return MOE_OK;
+}
+
+int moe_device_status(moe_plan_t *p, void *cuda_stream) {
+    if (!p) return MOE_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(p->status_host, p->ws.status, sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemsetAsync(p->ws.status, 0, sizeof(int32_t), s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    const int32_t v = *p->status_host;
+    if (v & kStatusTimeout) return MOE_ERR_TIMEOUT;
+    if (v & kStatusBadIndex) return MOE_ERR_DEVICE_CHECK;
+    return MOE_OK;
+}
+
+}  // extern "C"

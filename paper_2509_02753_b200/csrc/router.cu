@@ -1,0 +1,265 @@
+// Router: logits z = x . W_g^T (+ bias), softmax, top-k_l selection, optional renormalisation.
+// Paper, Section 2: G(x) = Softmax(TopK[x . W_g]); k_l is the per-layer number of active
+// experts (Algorithm 1, UpdateTopk).  All router arithmetic is fp32.
+//
+// A warp owns a whole row of logits (expert e lives in lane e % 32, register e / 32), so the
+// softmax statistics and the k_l-step selection are warp shuffles only.
+#include <math_constants.h>
+
+#include "moe_internal.h"
+
+namespace lexi {
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        unsigned long long other = __shfl_xor_sync(0xffffffffu, v, o);
+        v = other > v ? other : v;
+    }
+    return v;
+}
+
+// Monotone map float -> uint32 (larger float <-> larger integer); -0 is folded onto +0 first.
+__device__ __forceinline__ uint32_t ordered_bits(float z) {
+    uint32_t u = __float_as_uint(z + 0.0f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(uint32_t o) {
+    uint32_t u = (o & 0x80000000u) ? (o & 0x7fffffffu) : ~o;
+    return __uint_as_float(u);
+}
+
+// TopK + Softmax on one row of logits held by a warp.  z[j] is the logit of expert
+// lane + 32 j (ignored where that is >= E).  Selection order: larger logit first, equal
+// logits -> lower expert index.  Gate of a selected expert: exp(z_i - max) / D with
+// D = sum over the selected experts (renorm) or over all experts (no renorm).
+__device__ void warp_route(const float (&z)[kExpertsPerLane], int E, int k, int renorm, int lane,
+                           int32_t *idx_out, float *w_out) {
+    float m = -CUDART_INF_F;
+    unsigned long long key[kExpertsPerLane];
+#pragma unroll
+    for (int j = 0; j < kExpertsPerLane; ++j) {
+        const int e = lane + 32 * j;
+        if (e < E) {
+            m = fmaxf(m, z[j]);
+            // value in the high word, inverted index in the low word: max-reduce picks the
+            // larger logit and, among equal logits, the lower index
+            key[j] = ((unsigned long long)ordered_bits(z[j]) << 32) | (uint32_t)(0x7fffffff - e);
+        } else {
+            key[j] = 0ull;
+        }
+    }
+    m = warp_max(m);
+    float s_all = 0.f;
+#pragma unroll
+    for (int j = 0; j < kExpertsPerLane; ++j)
+        if (lane + 32 * j < E) s_all += expf(z[j] - m);
+    s_all = warp_sum(s_all);
+
+    float p_keep[kExpertsPerLane];   // slot i is kept by lane i % 32 in register i / 32
+    int e_keep[kExpertsPerLane];
+    float s_sel = 0.f;
+    for (int i = 0; i < k; ++i) {
+        unsigned long long best = key[0];
+#pragma unroll
+        for (int j = 1; j < kExpertsPerLane; ++j) best = key[j] > best ? key[j] : best;
+        best = warp_max_u64(best);
+        const int e = 0x7fffffff - (int)(uint32_t)(best & 0xffffffffull);
+        const float zsel = from_ordered_bits((uint32_t)(best >> 32));
+        const float p = expf(zsel - m);
+        s_sel += p;
+#pragma unroll
+        for (int j = 0; j < kExpertsPerLane; ++j)
+            if (lane + 32 * j == e) key[j] = 0ull;
+#pragma unroll
+        for (int j = 0; j < kExpertsPerLane; ++j)
+            if (i == lane + 32 * j) { p_keep[j] = p; e_keep[j] = e; }
+    }
+    const float inv = 1.0f / (renorm ? s_sel : s_all);
+#pragma unroll
+    for (int j = 0; j < kExpertsPerLane; ++j) {
+        const int i = lane + 32 * j;
+        if (i < k) {
+            if (idx_out) idx_out[i] = e_keep[j];
+            if (w_out) w_out[i] = p_keep[j] * inv;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Small T: one block per token.  The token's row is widened into shared memory once; each
+// warp takes every 8th row of W_g (plus the shared-expert gate vector w_s as row E) with
+// 16-byte loads, reduces by shuffle, and warp 0 routes.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) router_token_kernel(RouterArgs a) {
+    extern __shared__ float smem[];
+    float *xs = smem;                 // [d]
+    float *zs = smem + a.d;           // [E + 1]
+    const int t = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const T *x = (const T *)a.x + (size_t)t * a.d;
+    for (int c = tid; c < a.d; c += 256) xs[c] = to_f32(x[c]);
+    __syncthreads();
+
+    const int rows = a.E + (a.w_s ? 1 : 0);
+    constexpr int V = 16 / sizeof(T);          // elements per 16-byte load
+    for (int r = warp; r < rows; r += 8) {
+        const T *w = (r < a.E) ? (const T *)a.W + (size_t)r * a.d : (const T *)a.w_s;
+        float acc = 0.f;
+        for (int c = lane * V; c < a.d; c += 32 * V) {
+            const uint4 raw = *reinterpret_cast<const uint4 *>(w + c);
+            const T *wv = reinterpret_cast<const T *>(&raw);
+#pragma unroll
+            for (int u = 0; u < V; ++u) acc = fmaf(to_f32(wv[u]), xs[c + u], acc);
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) zs[r] = acc;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        float z[kExpertsPerLane];
+#pragma unroll
+        for (int j = 0; j < kExpertsPerLane; ++j) {
+            const int e = lane + 32 * j;
+            z[j] = (e < a.E) ? zs[e] + (a.bias ? a.bias[e] : 0.f) : 0.f;
+            if (e < a.E && a.logits) a.logits[(size_t)t * a.E + e] = z[j];
+        }
+        if (a.w_s && lane == 0) a.gamma[t] = 1.0f / (1.0f + expf(-zs[a.E]));
+        warp_route(z, a.E, a.k, a.renorm, lane, a.topk_idx + (size_t)t * a.k,
+                   a.topk_w + (size_t)t * a.k);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Large T: a block takes 32 tokens; x and W_g go through shared memory in chunks of 64
+// along d; warp w accumulates tokens 4w..4w+3 against experts lane, lane+32, ... so that the
+// finished logits already sit in the layout warp_route wants.
+// ---------------------------------------------------------------------------------------
+constexpr int kRtTokens = 32;
+constexpr int kRtChunk = 64;
+
+template <typename T>
+__global__ void __launch_bounds__(256) router_tile_kernel(RouterArgs a) {
+    __shared__ float xs[kRtTokens][kRtChunk + 1];
+    __shared__ float ws[kMaxExperts][kRtChunk + 1];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int t0 = blockIdx.x * kRtTokens;
+    const int rows = a.E + (a.w_s ? 1 : 0);
+    const int nj = (rows + 31) / 32;
+    const T *x = (const T *)a.x;
+
+    float acc[4][kExpertsPerLane];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < kExpertsPerLane; ++j) acc[i][j] = 0.f;
+
+    for (int i = tid; i < kMaxExperts * (kRtChunk + 1); i += 256) (&ws[0][0])[i] = 0.f;
+
+    for (int c0 = 0; c0 < a.d; c0 += kRtChunk) {
+        __syncthreads();
+        for (int i = tid; i < kRtTokens * kRtChunk; i += 256) {
+            const int r = i / kRtChunk, c = i % kRtChunk;
+            const int t = t0 + r;
+            xs[r][c] = (t < a.T && c0 + c < a.d) ? to_f32(x[(size_t)t * a.d + c0 + c]) : 0.f;
+        }
+        for (int i = tid; i < rows * kRtChunk; i += 256) {
+            const int r = i / kRtChunk, c = i % kRtChunk;
+            const T *w = (r < a.E) ? (const T *)a.W + (size_t)r * a.d : (const T *)a.w_s;
+            ws[r][c] = (c0 + c < a.d) ? to_f32(w[c0 + c]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int kk = 0; kk < kRtChunk; ++kk) {
+            float xv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) xv[i] = xs[warp * 4 + i][kk];
+#pragma unroll
+            for (int j = 0; j < kExpertsPerLane; ++j) {
+                if (j < nj) {
+                    const float wv = ws[lane + 32 * j][kk];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[i][j] = fmaf(xv[i], wv, acc[i][j]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int t = t0 + warp * 4 + i;
+        if (t >= a.T) continue;      // whole warp takes the same branch
+        float z[kExpertsPerLane];
+#pragma unroll
+        for (int j = 0; j < kExpertsPerLane; ++j) {
+            const int e = lane + 32 * j;
+            z[j] = (e < a.E) ? acc[i][j] + (a.bias ? a.bias[e] : 0.f) : 0.f;
+            if (e < a.E && a.logits) a.logits[(size_t)t * a.E + e] = z[j];
+            if (a.w_s && e == a.E) a.gamma[t] = 1.0f / (1.0f + expf(-acc[i][j]));
+        }
+        warp_route(z, a.E, a.k, a.renorm, lane, a.topk_idx + (size_t)t * a.k,
+                   a.topk_w + (size_t)t * a.k);
+    }
+}
+
+// TopK + Softmax from logits handed in by the caller: one warp per token.
+__global__ void __launch_bounds__(256) route_logits_kernel(const float *logits, int T, int E, int k,
+                                                           int renorm, int32_t *topk_idx,
+                                                           float *topk_w) {
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (t >= T) return;
+    float z[kExpertsPerLane];
+#pragma unroll
+    for (int j = 0; j < kExpertsPerLane; ++j) {
+        const int e = lane + 32 * j;
+        z[j] = (e < E) ? logits[(size_t)t * E + e] : 0.f;
+    }
+    warp_route(z, E, k, renorm, lane, topk_idx ? topk_idx + (size_t)t * k : nullptr,
+               topk_w ? topk_w + (size_t)t * k : nullptr);
+}
+
+cudaError_t launch_router(const RouterArgs &a, cudaStream_t s, uint64_t *launches) {
+    if (a.T <= 0) return cudaSuccess;
+    const bool small = a.T <= 512;
+    if (small) {
+        const size_t smem = (size_t)(a.d + a.E + 1) * sizeof(float);
+        if (a.dtype == MOE_BF16)
+            router_token_kernel<__nv_bfloat16><<<a.T, 256, smem, s>>>(a);
+        else
+            router_token_kernel<float><<<a.T, 256, smem, s>>>(a);
+    } else {
+        const int grid = (a.T + kRtTokens - 1) / kRtTokens;
+        if (a.dtype == MOE_BF16)
+            router_tile_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(a);
+        else
+            router_tile_kernel<float><<<grid, 256, 0, s>>>(a);
+    }
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_route_from_logits(const float *logits, int T, int E, int k, int renorm,
+                                     int32_t *topk_idx, float *topk_w, cudaStream_t s,
+                                     uint64_t *launches) {
+    if (T <= 0) return cudaSuccess;
+    route_logits_kernel<<<(T + 7) / 8, 256, 0, s>>>(logits, T, E, k, renorm, topk_idx, topk_w);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace lexi

@@ -1,0 +1,82 @@
+"""Helpers of the GPU parity tests: run the CUDA path and the CPU oracle on the same bytes
+and compare element by element.  Tolerances are the ones the tests state:
+
+  * routing (indices, counts, offsets, permutation): bit-exact on every token whose
+    k-th and (k+1)-th logits differ by more than 1e-3 (margin taken by the oracle);
+  * outputs: max|y - y_ref| / rms(y_ref) <= 2e-2 for bf16 tensors, 1e-4 for fp32,
+    over the tokens whose routing agreed.
+"""
+from __future__ import annotations
+
+from typing import Dict, Optional, Sequence
+
+import numpy as np
+import torch
+
+from oracle import moe_oracle as orc
+from paper_2509_02753_b200 import binding as B
+
+MARGIN = 1e-3
+TOL = {torch.bfloat16: 2e-2, torch.float32: 1e-4}
+
+
+def oracle_weights(w_host: Dict[str, Optional[torch.Tensor]]) -> orc.LayerWeights:
+    return orc.LayerWeights(**{k: w_host.get(k) for k in
+                               ("router_W", "W_gate", "W_up", "W_down", "router_bias",
+                                "Ws_gate", "Ws_up", "Ws_down", "w_s")})
+
+
+def rel_err(y: np.ndarray, ref: np.ndarray) -> float:
+    rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
+    return float(np.max(np.abs(y.astype(np.float64) - ref))) / max(rms, 1e-30)
+
+
+def check_layer(plan: B.MoEPlan, x: torch.Tensor, w_dev: Dict[str, Optional[torch.Tensor]], k: int,
+                renorm: bool, *, shared_gate: bool = False, routed_scale: float = 1.0,
+                tokens: Optional[Sequence[int]] = None, tol: Optional[float] = None,
+                w_host: Optional[Dict[str, Optional[torch.Tensor]]] = None) -> dict:
+    """Runs one layer on the GPU and on the oracle; asserts parity; returns the figures."""
+    T, d = x.shape
+    E = w_dev["router_W"].shape[0]
+    ws = B.make_weights(w_dev)
+    y = torch.full_like(x, float("nan"))
+    plan.layer_forward(x, ws, k, renorm, y)
+    idx_g, wts_g, counts_g, offsets_g, perm_g, logits_g = plan.last_routing(T, k)
+    assert plan.device_status() == 0
+    torch.cuda.synchronize()
+
+    if w_host is None:
+        w_host = {n: (None if t is None else t.cpu()) for n, t in w_dev.items()}
+    ow = oracle_weights(w_host)
+    r = orc.moe_layer(x.cpu(), ow, k, renorm, shared_gate=shared_gate, routed_scale=routed_scale,
+                      tokens=tokens)
+
+    # logits: fp32 accumulation of exact products against the double sum
+    np.testing.assert_allclose(logits_g.cpu().numpy(), r.logits, rtol=0,
+                               atol=2e-4 * max(1.0, float(np.abs(r.logits).max())))
+    idx_gn = idx_g.cpu().numpy()
+    safe = r.margin > MARGIN
+    agree = np.all(idx_gn == r.idx, axis=1)
+    assert np.all(agree[safe]), f"routing differs on {int((~agree[safe]).sum())} tokens outside the margin"
+    excluded = float((~safe).mean())
+    # dispatch tables: the integer definition applied to the indices the GPU selected
+    counts_e, offsets_e, perm_e, _ = orc.dispatch(idx_gn, E)
+    assert np.array_equal(counts_g.cpu().numpy(), counts_e)
+    assert np.array_equal(offsets_g.cpu().numpy(), offsets_e)
+    assert np.array_equal(perm_g.cpu().numpy(), perm_e)
+    if np.all(agree):
+        assert np.array_equal(counts_e, r.counts) and np.array_equal(perm_e, r.perm)
+    # gates
+    np.testing.assert_allclose(wts_g.cpu().numpy()[agree], r.gate[agree], rtol=2e-4, atol=1e-7)
+
+    # outputs on the evaluated tokens whose routing agreed
+    toks = r.tokens
+    keep = agree[toks]
+    assert keep.any()
+    y_g = y.float().cpu().numpy()[toks][keep]
+    assert np.all(np.isfinite(y.float().cpu().numpy())), "output has non-finite entries"
+    err = rel_err(y_g, r.y[keep])
+    tol = TOL[x.dtype] if tol is None else tol
+    assert err <= tol, f"max|dy|/rms(y_ref) = {err:.3e} > {tol:g}"
+    return {"err": err, "excluded": excluded, "agree": float(agree.mean()),
+            "touched": int((counts_e > 0).sum())}

@@ -1,0 +1,249 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Tolerances: routing bit-exact (outside a 1e-3 logit margin when the logits come
+from the GPU's own fp32 GEMM), outputs max|dy|/rms(y_ref) <= 2e-2 (bf16) or 1e-4 (fp32)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as orc
+from paper_2509_02753_b200 import binding as B
+from paper_2509_02753_b200 import synth
+
+from parity import TOL, check_layer, oracle_weights, rel_err
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+def _custom(name, d, E, I, I_shared=0, shared_gate=False, bias=0.0, L=1, k_base=2):
+    return synth.Workload(name, d=d, E=E, I=I, k_base=k_base, L=L, I_shared=I_shared,
+                          shared_gate=shared_gate, router_bias_std=bias, w_std=0.05)
+
+
+def _plan(wl, max_T, max_k, dtype, routed_scale=1.0):
+    return B.MoEPlan(wl.d, wl.E, wl.I, max_T, max_k, dtype, I_shared=wl.I_shared,
+                     shared_gate=wl.shared_gate, routed_scale=routed_scale)
+
+
+def _schedules(plan):
+    out = [B.MOE_SCHED_SIMT]
+    for s in (B.MOE_SCHED_DECODE, B.MOE_SCHED_PREFILL):
+        try:
+            plan.set_schedule(s)
+            out.append(s)
+        except B.MoEError:
+            pass
+    plan.set_schedule(B.MOE_SCHED_AUTO)
+    return out
+
+
+# --------------------------------------------------------------------------- routing from logits
+
+@pytest.mark.parametrize("T,E,k,renorm", [
+    (1, 8, 1, True), (1, 8, 8, False), (64, 8, 2, True), (37, 60, 4, False), (300, 64, 8, False),
+    (2048, 60, 4, True), (5000, 64, 6, False), (129, 128, 7, True), (16384, 8, 2, True),
+    (33, 5, 5, True), (257, 64, 64, False)])
+def test_routing_from_given_logits_is_bit_exact(T, E, k, renorm):
+    g = torch.Generator().manual_seed(T * 131 + E * 7 + k)
+    logits = torch.randn((T, E), generator=g, dtype=torch.float32)
+    logits[:, 0] += 0.7                                   # skewed load
+    if T >= 8:                                            # planted exact ties
+        logits[3, :] = 0.25
+        logits[5, E // 2:] = logits[5, 0]
+        logits[7, -1] = logits[7].max()
+    with B.MoEPlan(64, E, 64, T, k, torch.float32) as plan:
+        idx, wts, counts, offsets, perm = plan.route_from_logits(logits.to(DEV), k, renorm)
+        assert plan.device_status() == 0
+    idx_o, gate_o, _ = orc.topk_gates(logits.numpy(), k, renorm, select_f32=True)
+    counts_o, offsets_o, perm_o, _ = orc.dispatch(idx_o, E)
+    assert np.array_equal(idx.cpu().numpy(), idx_o)
+    assert np.array_equal(counts.cpu().numpy(), counts_o)
+    assert np.array_equal(offsets.cpu().numpy(), offsets_o)
+    assert np.array_equal(perm.cpu().numpy(), perm_o)
+    assert int(counts.sum()) == T * k
+    np.testing.assert_allclose(wts.cpu().numpy(), gate_o, rtol=1e-5, atol=1e-8)
+    if renorm:
+        np.testing.assert_allclose(wts.sum(dim=1).cpu().numpy(), 1.0, atol=1e-5)
+
+
+# --------------------------------------------------------------------------- single layer
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_tiny_layer_all_schedules(dtype):
+    """T=64, d=256, E=8, I=512, top-2 renormalised, no shared expert; fp32 and bf16 variants."""
+    wl = synth.WORKLOADS["tiny"]
+    w = synth.make_layer(wl, 0, dtype, DEV)
+    x = synth.make_tokens(wl, 64, dtype, DEV)
+    with _plan(wl, 64, 8, dtype) as plan:
+        for sched in _schedules(plan):
+            plan.set_schedule(sched)
+            for k, renorm in [(2, True), (1, True), (8, False), (3, False)]:
+                check_layer(plan, x, w, k, renorm)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("T", [1, 5, 37, 130, 700])
+def test_ragged_shapes_with_gated_shared_expert(dtype, T):
+    wl = _custom("ragged", d=192, E=5, I=320, I_shared=448, shared_gate=True, bias=0.5)
+    w = synth.make_layer(wl, 0, dtype, DEV)
+    x = synth.make_tokens(wl, T, dtype, DEV)
+    with _plan(wl, 700, 5, dtype, routed_scale=1.25) as plan:
+        for sched in _schedules(plan):
+            plan.set_schedule(sched)
+            check_layer(plan, x, w, 2, False, shared_gate=True, routed_scale=1.25)
+            check_layer(plan, x, w, 5, True, shared_gate=True, routed_scale=1.25)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_simt_handles_sizes_that_are_only_multiples_of_8(dtype):
+    wl = _custom("odd", d=136, E=7, I=72, I_shared=40, shared_gate=False)
+    w = synth.make_layer(wl, 0, dtype, DEV)
+    x = synth.make_tokens(wl, 45, dtype, DEV)
+    with _plan(wl, 45, 7, dtype) as plan:
+        plan.set_schedule(B.MOE_SCHED_SIMT)
+        check_layer(plan, x, w, 3, True)
+        check_layer(plan, x, w, 7, False)
+
+
+def test_unused_experts_and_heavy_skew():
+    """All tokens prefer two experts: most experts receive no rows, one receives nearly all."""
+    wl = _custom("skew", d=256, E=16, I=256)
+    w = synth.make_layer(wl, 0, torch.bfloat16, DEV)
+    w["router_bias"] = torch.zeros(16, dtype=torch.float32, device=DEV)
+    w["router_bias"][3] = 20.0
+    w["router_bias"][11] = 10.0
+    x = synth.make_tokens(wl, 333, torch.bfloat16, DEV)
+    with _plan(wl, 333, 2, torch.bfloat16) as plan:
+        for sched in _schedules(plan):
+            plan.set_schedule(sched)
+            info = check_layer(plan, x, w, 2, True)
+            assert info["touched"] == 2
+            check_layer(plan, x, w, 1, False)
+
+
+def test_zero_tokens_is_a_no_op_and_bad_arguments_are_refused():
+    wl = synth.WORKLOADS["tiny"]
+    w = B.make_weights(synth.make_layer(wl, 0, torch.bfloat16, DEV))
+    x = synth.make_tokens(wl, 8, torch.bfloat16, DEV)
+    y = torch.zeros_like(x)
+    lib = B.load_library()
+    with _plan(wl, 8, 2, torch.bfloat16) as plan:
+        import ctypes
+        h = plan.handle
+        call = lambda xp, T, k, yp: lib.moe_layer_forward(h, xp, ctypes.byref(w), T, k, 1, yp, None)
+        assert call(x.data_ptr(), 0, 2, y.data_ptr()) == 0
+        assert float(y.abs().sum()) == 0.0
+        assert call(x.data_ptr(), 8, 0, y.data_ptr()) == -1          # k_l = 0
+        assert call(x.data_ptr(), 8, 3, y.data_ptr()) == -1          # k_l > max_k
+        assert call(x.data_ptr(), 9, 2, y.data_ptr()) == -1          # T > max_T
+        assert call(None, 8, 2, y.data_ptr()) == -1
+        assert call(x.data_ptr(), 8, 2, x.data_ptr()) == -1          # y aliases x
+        assert call(x.data_ptr() + 2, 8, 2, y.data_ptr()) == -3      # misaligned
+        bad = B.moe_layer_weights_t()
+        assert lib.moe_layer_forward(h, x.data_ptr(), ctypes.byref(bad), 8, 2, 1, y.data_ptr(), None) == -1
+        assert plan.device_status() == 0
+    with pytest.raises(B.MoEError):
+        B.MoEPlan(256, 8, 512, 8, 9, torch.bfloat16)                 # max_k > E
+    with pytest.raises(B.MoEError):
+        B.MoEPlan(250, 8, 512, 8, 2, torch.bfloat16)                 # d not a multiple of 8
+
+
+def test_two_calls_are_bit_identical():
+    """Algorithm 1 relies on Delta(k_base) = 0: the same call twice gives the same bits."""
+    wl = _custom("det", d=256, E=16, I=384, I_shared=256)
+    w = synth.make_layer(wl, 0, torch.bfloat16, DEV)
+    ws = B.make_weights(w)
+    x = synth.make_tokens(wl, 500, torch.bfloat16, DEV)
+    with _plan(wl, 500, 4, torch.bfloat16) as plan:
+        for sched in _schedules(plan):
+            plan.set_schedule(sched)
+            a = plan.layer_forward(x, ws, 4, False).clone()
+            plan.layer_forward(x, ws, 2, False)
+            b = plan.layer_forward(x, ws, 4, False)
+            assert torch.equal(a, b)
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    wl = synth.WORKLOADS["tiny"]
+    w = B.make_weights(synth.make_layer(wl, 0, torch.bfloat16, DEV))
+    x = synth.make_tokens(wl, 64, torch.bfloat16, "cpu").pin_memory()
+    y_host = torch.empty_like(x).pin_memory()
+    with _plan(wl, 64, 2, torch.bfloat16) as plan:
+        y_dev = plan.layer_forward(x.to(DEV), w, 2, True)
+        B.moe_layer_forward_host(plan.handle, x, w, 2, True, y_host)
+        torch.cuda.synchronize()
+        assert torch.equal(y_dev.cpu(), y_host)
+
+
+# --------------------------------------------------------------------------- model-shaped layers
+
+@pytest.mark.parametrize("T,k", [(1, 4), (8, 4), (64, 4), (64, 1), (2048, 4), (2048, 2), (8192, 4), (8192, 1)])
+def test_qwen15_shaped_layer(T, k):
+    """d=2048, E=60, I=1408, gated shared expert of 5632, biased router; sampled tokens at large T."""
+    wl = synth.WORKLOADS["qwen15"]
+    w = synth.make_layer(wl, 0, torch.bfloat16, DEV)
+    w_host = synth.to_host(w)
+    x = synth.make_tokens(wl, T, torch.bfloat16, DEV)
+    toks = None if T <= 64 else np.random.default_rng(T + k).choice(T, 48, replace=False)
+    with _plan(wl, T, 4, torch.bfloat16) as plan:
+        info = check_layer(plan, x, w, k, False, shared_gate=True, tokens=toks, w_host=w_host)
+        assert info["excluded"] < 0.05
+        if T == 64:
+            check_layer(plan, x, w, k, True, shared_gate=True, w_host=w_host)
+
+
+@pytest.mark.parametrize("T,k", [(1, 2), (16, 1), (256, 2)])
+def test_mixtral_shaped_layer(T, k):
+    """d=4096, E=8, I=14336, renormalised gates; 16 sampled tokens."""
+    wl = synth.WORKLOADS["mixtral"]
+    w = synth.make_layer(wl, 0, torch.bfloat16, DEV)
+    w_host = synth.to_host(w)
+    x = synth.make_tokens(wl, T, torch.bfloat16, DEV)
+    toks = None if T <= 16 else np.random.default_rng(T).choice(T, 16, replace=False)
+    with _plan(wl, T, 2, torch.bfloat16) as plan:
+        check_layer(plan, x, w, k, True, tokens=toks, w_host=w_host)
+
+
+# --------------------------------------------------------------------------- stack
+
+def _stack_case(wl, L, T, dtype):
+    layers = [synth.make_layer(wl, l, dtype, DEV) for l in range(L)]
+    x = synth.make_tokens(wl, T, dtype, DEV)
+    return layers, x
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_stack_with_per_layer_k(dtype):
+    wl = _custom("stack", d=256, E=16, I=256, I_shared=128, shared_gate=True, bias=0.3, L=5, k_base=6)
+    L, T = 5, 96
+    k_vec = [6, 2, 4, 1, 3]
+    layers, x = _stack_case(wl, L, T, dtype)
+    ows = [oracle_weights(synth.to_host(w)) for w in layers]
+    h_ref, inputs, margins = orc.moe_stack(x.cpu(), ows, k_vec, False, shared_gate=True)
+    structs = [B.make_weights(w) for w in layers]
+    with _plan(wl, T, 6, dtype) as plan:
+        for sched in _schedules(plan):
+            plan.set_schedule(sched)
+            # free running: final h on tokens whose margin exceeded 1e-3 in every layer
+            h = x.clone()
+            plan.stack_forward(h, structs, k_vec, False)
+            assert plan.device_status() == 0
+            safe = np.all(margins > 1e-3, axis=0)
+            assert safe.mean() > 0.8
+            err = rel_err(h.float().cpu().numpy()[safe], h_ref[safe])
+            assert err <= TOL[dtype], err
+            # teacher forcing: layer l fed the oracle's h_l (rounded to the plan's dtype)
+            for l in range(L):
+                h_in = torch.from_numpy(inputs[l]).to(dtype).to(DEV)
+                y = plan.layer_forward(h_in, structs[l], k_vec[l], False)
+                r = orc.moe_layer(h_in.cpu(), ows[l], k_vec[l], False, shared_gate=True)
+                ok = r.margin > 1e-3
+                assert rel_err(y.float().cpu().numpy()[ok], r.y[ok]) <= TOL[dtype]
+            # uniform k through the stack call equals chained layer calls plus residual
+            h2 = x.clone()
+            plan.stack_forward(h2, structs[:1], [3], False)
+            y1 = plan.layer_forward(x, structs[0], 3, False)
+            ref1 = (x.float() + y1.float())
+            assert rel_err(h2.float().cpu().numpy(), ref1.double().cpu().numpy()) <= \
+                (2e-2 if dtype == torch.bfloat16 else 1e-5)
