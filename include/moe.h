@@ -180,6 +180,14 @@ int moe_last_routing(moe_plan_t *plan, int32_t *topk_idx, float *topk_w, int32_t
                      int32_t *offsets, int32_t *perm, float *logits, void *cuda_stream);
 
 /*
+ * moe_last_residual_f32 (test hook): copies the plan's fp32 residual stream, as left by the most
+ * recent moe_stack_forward on a bf16 plan, into h_f32 [T, d] (device, fp32).  It is the value the
+ * returned bf16 h was rounded from, so it shows the result before the output format's rounding.
+ * Errors: INVALID_ARG (also for fp32 plans, whose h is the residual stream itself).
+ */
+int moe_last_residual_f32(moe_plan_t *plan, float *h_f32, int32_t T, void *cuda_stream);
+
+/*
  * moe_device_status: synchronises the stream, reads and clears the device status word.
  * Returns MOE_OK, MOE_ERR_TIMEOUT, MOE_ERR_DEVICE_CHECK or MOE_ERR_CUDA.
  */

@@ -27,6 +27,7 @@ EXPORTS = (
     "moe_plan_get_schedule", "moe_layer_forward", "moe_layer_forward_host", "moe_stack_forward",
     "moe_route_from_logits", "moe_last_routing", "moe_device_status", "moe_plan_launch_count",
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
+    "moe_last_residual_f32",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
 
@@ -77,6 +78,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_route_from_logits.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.moe_last_routing.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.moe_device_status.argtypes = [vp, vp]
+    lib.moe_last_residual_f32.argtypes = [vp, vp, i32, vp]
     lib.moe_plan_set_stage_timing.argtypes = [vp, i32]
     lib.moe_plan_stage_times.argtypes = [vp, P(ctypes.c_float), P(i32)]
     lib.moe_status_string.argtypes = [ctypes.c_int]
@@ -233,6 +235,14 @@ def moe_plan_stage_times(plan: int):
     return {name: float(ms[i]) for i, name in enumerate(STAGE_NAMES)}, int(n.value)
 
 
+def moe_last_residual_f32(plan: int, T: int, d: int, device="cuda", stream=None) -> torch.Tensor:
+    """fp32 residual stream [T,d] left by the latest moe_stack_forward of a bf16 plan."""
+    out = torch.empty((T, d), dtype=torch.float32, device=device)
+    _check("moe_last_residual_f32",
+           load_library().moe_last_residual_f32(plan, out.data_ptr(), T, _stream(stream)))
+    return out
+
+
 def moe_device_status(plan: int, stream=None) -> int:
     return int(load_library().moe_device_status(plan, _stream(stream)))
 
@@ -284,6 +294,9 @@ class MoEPlan:
 
     def last_routing(self, T, k_l, device="cuda", stream=None):
         return moe_last_routing(self.handle, T, k_l, self.E, device, stream)
+
+    def last_residual_f32(self, T, device="cuda", stream=None):
+        return moe_last_residual_f32(self.handle, T, self.d, device, stream)
 
     def device_status(self, stream=None) -> int:
         return moe_device_status(self.handle, stream)

@@ -1,11 +1,608 @@
+// Expert FFNs on the 5th-generation tensor cores: grouped GEMMs with tcgen05.mma, accumulators
+// in tensor memory (TMEM), operands staged in shared memory by TMA (no multicast anywhere).
+// Paper, Section 2: the experts E_i of y = sum G_i E_i(x); E(x) = W_down (silu(W_gate x) * (W_up x)).
+//
+// One persistent kernel template serves both GEMM phases and both schedules:
+//   phase 1   D[token, n] = x_perm[token, :] . [W_gate; W_up][n, :]   -> h = silu(gate) * up
+//   phase 2   D[token, c] = h[token, :] . W_down[c, :]                -> o (optionally split along K)
+// A tile is 128 token rows (UMMA M = 128; the rows beyond a group's count are never stored) by
+// BN weight rows (UMMA N), reduced over K in chunks of 64 bf16 (one 128-byte swizzle row).
+//   warp 0      TMA producer (one lane)            full/empty mbarrier ring of STAGES stages
+//   warp 1      TMEM allocation + MMA issue (one lane), tcgen05.commit frees stages / hands over TMEM
+//   warps 2-5   epilogue: tcgen05.ld of the finished accumulator (two TMEM buffers, so the next
+//               tile's MMAs overlap), SwiGLU or plain store
+// Decode schedule: BN = 128, small activation box (32/64/128 rows), K split into slabs so that
+// enough CTAs stream disjoint weight slices to saturate HBM; two CTAs per SM.
+// Prefill schedule: BN = 256, four 48 KB stages, one CTA per SM, all 512 TMEM columns.
+//
+// Every mbarrier wait is bounded in time; a wait that runs out sets the status word and the CTA
+// leaves through the common exit (TMEM is always freed).
+#include <cuda.h>
+
 #include "ffn_tc.h"
+
 namespace lexi {
-bool tc_shape_ok(const moe_config_t &) { return false; }
-int tc_max_slabs(const moe_config_t &) { return 1; }
-int tc_max_shared_slabs(const moe_config_t &) { return 1; }
-size_t tc_o_elems(const moe_config_t &c, int slabs) { return (size_t)slabs * c.max_T * c.max_k * c.d; }
-size_t tc_os_elems(const moe_config_t &c, int slabs) { return (size_t)slabs * c.max_T * c.d; }
-size_t tc_max_tiles(const moe_config_t &, int) { return 1; }
-int tc_state_init(TcState *, const moe_config_t &) { return MOE_OK; }
-int tc_ffn_forward(TcState *, const moe_config_t &, const Workspace &, const FfnArgs &, int, int, cudaStream_t, uint64_t *, TcOutputLayout *) { return MOE_ERR_NOT_IMPLEMENTED; }
+namespace {
+
+constexpr int kBK = 64;                         // K elements per stage (128 bytes of bf16)
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false (and the timeout bit set) if the phase does not complete within kWaitLimitNs.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t *status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 0xffu) == 0 && global_ns() - t0 > kWaitLimitNs) {
+            atomicOr(status, kStatusTimeout);
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                            int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 x bf16 -> fp32, M = 128, K = 16 per instruction
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// mbarrier arrives once all tcgen05.mma issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle, groups of 8 rows
+// 1024 bytes apart (this is the layout TMA writes with CU_TENSOR_MAP_SWIZZLE_128B).
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);        // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                             // leading byte offset (unused for this layout)
+    d |= (uint64_t)(1024 >> 4) << 32;                   // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                             // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;                             // layout type: 128-byte swizzle
+    return d;
+}
+// Instruction descriptor of kind::f16: fp32 accumulate, bf16 A and B, both K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+struct TcParams {
+    const Tile *tiles;
+    const int32_t *n_tiles;      // device: number of tiles in the list
+    int32_t E;                   // group == E is the shared expert
+    int32_t N_routed, N_shared;  // row pitch and column bound of the outputs
+    void *out_routed, *out_shared;
+    unsigned long long slab_stride_routed, slab_stride_shared;   // elements between split-K slabs
+    int32_t *status;
+};
+
+template <int A_ROWS, int BN, int STAGES>
+constexpr int tc_smem_bytes() {
+    return STAGES * (A_ROWS * 128 + BN * 128) + 1024 /* alignment slack */ + 256 /* barriers */;
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) {
+    return __fdividef(g, 1.0f + __expf(-g)) * u;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+template <int PHASE, int BN, int A_ROWS, int STAGES, int MIN_CTAS, typename OutT>
+__global__ void __launch_bounds__(192, MIN_CTAS)
+ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_constant__ CUtensorMap mapA_shared,
+              const __grid_constant__ CUtensorMap mapB0_routed, const __grid_constant__ CUtensorMap mapB1_routed,
+              const __grid_constant__ CUtensorMap mapB0_shared, const __grid_constant__ CUtensorMap mapB1_shared,
+              const TcParams p) {
+    constexpr int A_BYTES = A_ROWS * 128;
+    constexpr int B_BYTES = BN * 128;
+    constexpr int TMEM_COLS = 2 * BN;
+    static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM columns: power of two");
+    static_assert(STAGES * B_BYTES >= 128 * 128, "the 128-row operand read must stay inside the allocation");
+
+    const int n_tiles = *p.n_tiles;
+    if ((int)blockIdx.x >= n_tiles) return;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const uint32_t a_base = base;
+    const uint32_t b_base = base + STAGES * A_BYTES;
+    const uint32_t bar_base = b_base + STAGES * B_BYTES;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+    const uint32_t slot_addr = bar_base + 8u * (2 * STAGES + 4);
+    volatile uint32_t *slot_ptr = reinterpret_cast<volatile uint32_t *>(smem_raw + (slot_addr - raw));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 128); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(slot_addr, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *slot_ptr;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+                const Tile t = p.tiles[tile];
+                const bool shared = t.group == p.E;
+                const CUtensorMap *mA = shared ? &mapA_shared : &mapA_routed;
+                const CUtensorMap *mB0 = shared ? &mapB0_shared : &mapB0_routed;
+                const CUtensorMap *mB1 = shared ? &mapB1_shared : &mapB1_routed;
+                const int grp = shared ? 0 : t.group;
+                const int nk = (t.klen + kBK - 1) / kBK;
+                for (int kc = 0; kc < nk; ++kc, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, p.status)) { ok = false; break; }
+                    mbar_expect_tx(full_bar(s), A_BYTES + B_BYTES);
+                    const int k = t.k0 + kc * kBK;
+                    tma_load_3d(a_base + s * A_BYTES, mA, full_bar(s), k, t.row0, 0);
+                    if (PHASE == 1) {
+                        tma_load_3d(b_base + s * B_BYTES, mB0, full_bar(s), k, t.n0, grp);
+                        tma_load_3d(b_base + s * B_BYTES + B_BYTES / 2, mB1, full_bar(s), k, t.n0, grp);
+                    } else {
+                        tma_load_3d(b_base + s * B_BYTES, mB0, full_bar(s), k, t.n0, grp);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(BN);
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++tcount) {
+                const Tile t = p.tiles[tile];
+                const int nk = (t.klen + kBK - 1) / kBK;
+                const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(buf), bph ^ 1u, p.status)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kc = 0; kc < nk; ++kc, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t a_desc = make_kmajor_sw128_desc(a_base + s * A_BYTES);
+                    const uint64_t b_desc = make_kmajor_sw128_desc(b_base + s * B_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < kBK / 16; ++kk)     // 32 bytes along K per instruction
+                        umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kc | kk) != 0);
+                    umma_commit(empty_bar(s));
+                }
+                if (ok) umma_commit(tfull_bar(buf));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;                  // TMEM lane quarter this warp may read
+        const int row_in_tile = q * 32 + lane;
+        uint32_t tcount = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
+            const Tile t = p.tiles[tile];
+            const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
+            const bool got = mbar_wait(tfull_bar(buf), bph, p.status);
+            if (!__all_sync(0xffffffffu, got)) break;
+            tc_fence_after();
+            const bool shared = t.group == p.E;
+            const int N = shared ? p.N_shared : p.N_routed;
+            const bool row_ok = row_in_tile < t.rows;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
+            OutT *out = reinterpret_cast<OutT *>(shared ? p.out_shared : p.out_routed) +
+                        (size_t)t.slot * (shared ? p.slab_stride_shared : p.slab_stride_routed) +
+                        (size_t)(t.row0 + row_in_tile) * N + t.n0;
+            if (PHASE == 1) {
+#pragma unroll 1
+                for (int c = 0; c < BN / 2; c += 16) {
+                    uint32_t g[16], u[16];
+                    tmem_ld16(taddr + c, g);
+                    tmem_ld16(taddr + BN / 2 + c, u);
+                    tmem_ld_wait();
+                    uint32_t packed[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        packed[i] = pack_bf16(silu_mul(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
+                                              silu_mul(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1])));
+                    if (row_ok) {
+                        if (t.n0 + c + 8 <= N)
+                            *reinterpret_cast<uint4 *>(out + c) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                        if (t.n0 + c + 16 <= N)
+                            *reinterpret_cast<uint4 *>(out + c + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                    }
+                }
+            } else {
+#pragma unroll 1
+                for (int c = 0; c < BN; c += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(taddr + c, v);
+                    tmem_ld_wait();
+                    if (row_ok) {
+                        if (sizeof(OutT) == 4) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                if (t.n0 + c + 4 * i + 4 <= N)
+                                    *reinterpret_cast<uint4 *>(out + c + 4 * i) =
+                                        make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 2; ++i)
+                                if (t.n0 + c + 8 * i + 8 <= N)
+                                    *reinterpret_cast<uint4 *>(out + c + 8 * i) = make_uint4(
+                                        pack_bf16(__uint_as_float(v[8 * i]), __uint_as_float(v[8 * i + 1])),
+                                        pack_bf16(__uint_as_float(v[8 * i + 2]), __uint_as_float(v[8 * i + 3])),
+                                        pack_bf16(__uint_as_float(v[8 * i + 4]), __uint_as_float(v[8 * i + 5])),
+                                        pack_bf16(__uint_as_float(v[8 * i + 6]), __uint_as_float(v[8 * i + 7])));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(tempty_bar(buf));
+        }
+    }
+
+    // ---------------------------------------------------------------- common exit
+    __syncwarp();
+    if (*reinterpret_cast<volatile int32_t *>(p.status) & kStatusTimeout) {
+        // a wait ran out somewhere: give copies and MMAs still in flight time to land before the
+        // shared memory and TMEM of this CTA are handed back
+        for (int i = 0; i < 256; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------ tile lists
+struct TileBuildArgs {
+    const int32_t *counts, *offsets;
+    int32_t E, T, has_shared;
+    int32_t feat1, N1_routed, N1_shared, K1;                     // phase 1: features per tile, I, I_s, d
+    int32_t bn2, N2, K2_routed, K2_shared;                       // phase 2: BN, d, I, I_s
+    int32_t ksplit_routed, kchunk_routed, ksplit_shared, kchunk_shared;
+    Tile *tiles1, *tiles2;
+    int32_t *n_tiles;
+    int32_t cap1, cap2;
+    int32_t *status;
+};
+
+// Group order: the shared expert first (its tiles are always full), then experts 0..E-1.
+// Inside a group: 128-row block outermost, then output-feature block, then K slab.
+__global__ void __launch_bounds__(256) build_tiles_kernel(TileBuildArgs a) {
+    __shared__ int32_t pre1[kMaxExperts + 2], pre2[kMaxExperts + 2];
+    const int groups = a.E + (a.has_shared ? 1 : 0);
+    auto group_of = [&](int slot) { return a.has_shared ? (slot == 0 ? a.E : slot - 1) : slot; };
+    auto rows_of = [&](int g) { return g == a.E ? a.T : a.counts[g]; };
+    if (threadIdx.x == 0) {
+        int r1 = 0, r2 = 0;
+        for (int sidx = 0; sidx < groups; ++sidx) {
+            const int g = group_of(sidx);
+            const int mblk = (rows_of(g) + kTileRows - 1) / kTileRows;
+            const int n1 = ((g == a.E ? a.N1_shared : a.N1_routed) + a.feat1 - 1) / a.feat1;
+            const int n2 = (a.N2 + a.bn2 - 1) / a.bn2;
+            const int ks = g == a.E ? a.ksplit_shared : a.ksplit_routed;
+            pre1[sidx] = r1; pre2[sidx] = r2;
+            r1 += mblk * n1;
+            r2 += mblk * n2 * ks;
+        }
+        pre1[groups] = r1; pre2[groups] = r2;
+        if (r1 > a.cap1 || r2 > a.cap2) { atomicOr(a.status, kStatusBadIndex); r1 = 0; r2 = 0; pre1[groups] = 0; pre2[groups] = 0; }
+        a.n_tiles[0] = r1;
+        a.n_tiles[1] = r2;
+    }
+    __syncthreads();
+    for (int phase = 0; phase < 2; ++phase) {
+        const int32_t *pre = phase == 0 ? pre1 : pre2;
+        const int total = pre[groups];
+        for (int i = threadIdx.x; i < total; i += blockDim.x) {
+            int lo = 0, hi = groups - 1;
+            while (lo < hi) {                     // last slot with pre[slot] <= i
+                const int mid = (lo + hi + 1) >> 1;
+                if (pre[mid] <= i) lo = mid; else hi = mid - 1;
+            }
+            const int g = group_of(lo);
+            const int local = i - pre[lo];
+            const int rows = rows_of(g);
+            const int first = g == a.E ? 0 : a.offsets[g];
+            Tile t;
+            t.group = g; t.pad = 0;
+            if (phase == 0) {
+                const int n1 = ((g == a.E ? a.N1_shared : a.N1_routed) + a.feat1 - 1) / a.feat1;
+                const int m = local / n1, n = local % n1;
+                t.row0 = first + m * kTileRows;
+                t.rows = min(kTileRows, rows - m * kTileRows);
+                t.n0 = n * a.feat1;
+                t.k0 = 0; t.klen = a.K1; t.slot = 0;
+                a.tiles1[i] = t;
+            } else {
+                const int n2 = (a.N2 + a.bn2 - 1) / a.bn2;
+                const int ks = g == a.E ? a.ksplit_shared : a.ksplit_routed;
+                const int kchunk = g == a.E ? a.kchunk_shared : a.kchunk_routed;
+                const int K = g == a.E ? a.K2_shared : a.K2_routed;
+                const int m = local / (n2 * ks), rem = local % (n2 * ks);
+                const int n = rem / ks, sl = rem % ks;
+                t.row0 = first + m * kTileRows;
+                t.rows = min(kTileRows, rows - m * kTileRows);
+                t.n0 = n * a.bn2;
+                t.k0 = sl * kchunk;
+                t.klen = max(0, min(kchunk, K - sl * kchunk));
+                t.slot = sl;
+                a.tiles2[i] = t;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                             const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                             CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                             CUtensorMapFloatOOBfill);
+
+// bf16 tensor [groups, rows, K] (K contiguous), box = 64 x box_rows x 1, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool encode_map(const TcState *st, CUtensorMap *m, const void *ptr, uint64_t K, uint64_t rows,
+                uint64_t groups, uint32_t box_rows) {
+    cuuint64_t dims[3] = {K, rows, groups};
+    cuuint64_t strides[2] = {K * 2, rows * K * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kBK, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = reinterpret_cast<EncodeFn>(st->encode_fn)(
+        m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+int ceil_div(int a, int b) { return (a + b - 1) / b; }
+int clampi(int v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : v); }
+int slabs_for(int K) { return clampi(ceil_div(K, 1024), 1, 8); }
+size_t decode_row_cap(const moe_config_t &c) {
+    const size_t pairs = (size_t)c.max_T * c.max_k;
+    const size_t cap = (size_t)16 * c.E;
+    return pairs < cap ? pairs : cap;
+}
+
+template <int PHASE, int BN, int A_ROWS, int STAGES, int MIN_CTAS, typename OutT>
+cudaError_t launch_tc(const CUtensorMap *maps, const TcParams &p, int grid, cudaStream_t s) {
+    auto kern = ffn_tc_kernel<PHASE, BN, A_ROWS, STAGES, MIN_CTAS, OutT>;
+    constexpr int smem = tc_smem_bytes<A_ROWS, BN, STAGES>();
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    kern<<<grid, 192, smem, s>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool tc_shape_ok(const moe_config_t &c) {
+    if (c.dtype != MOE_BF16) return false;
+    if (c.d < 64 || c.I < 64 || (c.I_shared > 0 && c.I_shared < 64)) return false;
+    return c.d % 8 == 0 && c.I % 8 == 0 && c.I_shared % 8 == 0;
+}
+int tc_max_slabs(const moe_config_t &c) { return slabs_for(c.I); }
+int tc_max_shared_slabs(const moe_config_t &c) { return c.I_shared > 0 ? slabs_for(c.I_shared) : 1; }
+
+size_t tc_o_elems(const moe_config_t &c, int slabs) {
+    const size_t pairs = (size_t)c.max_T * c.max_k;
+    const size_t full = pairs * c.d;                              // one fp32 slab for every pair
+    const size_t dec = decode_row_cap(c) * (size_t)slabs * c.d;   // split-K slabs, decode-sized calls
+    return full > dec ? full : dec;
+}
+size_t tc_os_elems(const moe_config_t &c, int slabs) {
+    const size_t full = (size_t)c.max_T * c.d;
+    const size_t rows = (size_t)c.max_T < (size_t)16 * c.E ? (size_t)c.max_T : (size_t)16 * c.E;
+    const size_t dec = rows * (size_t)slabs * c.d;
+    return full > dec ? full : dec;
+}
+size_t tc_max_tiles(const moe_config_t &c, int phase) {
+    const size_t pairs = (size_t)c.max_T * c.max_k;
+    const size_t mblk_routed = pairs / kTileRows + (pairs < (size_t)c.E ? pairs : (size_t)c.E);
+    const size_t mblk_shared = c.I_shared > 0 ? ((size_t)c.max_T + kTileRows - 1) / kTileRows : 0;
+    if (phase == 1)
+        return mblk_routed * ceil_div(c.I, 64) + mblk_shared * ceil_div(c.I_shared > 0 ? c.I_shared : 64, 64) + 1;
+    return mblk_routed * ceil_div(c.d, 128) * slabs_for(c.I) +
+           mblk_shared * ceil_div(c.d, 128) * (c.I_shared > 0 ? slabs_for(c.I_shared) : 1) + 1;
+}
+
+int tc_state_init(TcState *st, const moe_config_t &c) {
+    if (!tc_shape_ok(c)) return MOE_OK;     // SIMT-only plan
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    st->encode_fn = fn;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&st->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    st->ready = true;
+    return MOE_OK;
+}
+
+int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, const FfnArgs &a,
+                   int schedule, int sm_count, cudaStream_t s, uint64_t *launches,
+                   TcOutputLayout *layout) {
+    if (!st->ready) return MOE_ERR_SHAPE;
+    const bool decode = schedule == MOE_SCHED_DECODE;
+    const int rows = a.T * a.k;
+    const bool has_shared = a.I_s > 0;
+    const size_t pairs_alloc = (size_t)c.max_T * c.max_k;
+
+    // ---- schedule parameters
+    const int bn1 = decode ? 128 : 256;          // phase-1 tile: bn1/2 gate rows + bn1/2 up rows
+    const int bn2 = decode ? 128 : 256;
+    int a_rows = 128;
+    if (decode) a_rows = a.T <= 32 ? 32 : (a.T <= 64 ? 64 : 128);
+    int ks_r = 1, ks_s = 1;
+    if (decode && (size_t)rows <= decode_row_cap(c)) {
+        ks_r = slabs_for(a.I);
+        ks_s = has_shared ? slabs_for(a.I_s) : 1;
+    }
+    const int kchunk_r = ceil_div(ceil_div(a.I, ks_r), kBK) * kBK;
+    const int kchunk_s = has_shared ? ceil_div(ceil_div(a.I_s, ks_s), kBK) * kBK : kBK;
+    ks_r = ceil_div(a.I, kchunk_r);
+    if (has_shared) ks_s = ceil_div(a.I_s, kchunk_s);
+
+    // ---- tensor maps
+    CUtensorMap m1[6], m2[6];
+    bool ok = true;
+    const void *dummy = a.x;   // maps of an absent shared expert are never dereferenced
+    ok = ok && encode_map(st, &m1[0], a.x_perm, a.d, pairs_alloc + 128, 1, a_rows);
+    ok = ok && encode_map(st, &m1[1], a.x, a.d, a.T, 1, a_rows);
+    ok = ok && encode_map(st, &m1[2], a.W_gate, a.d, a.I, a.E, bn1 / 2);
+    ok = ok && encode_map(st, &m1[3], a.W_up, a.d, a.I, a.E, bn1 / 2);
+    ok = ok && encode_map(st, &m1[4], has_shared ? a.Ws_gate : dummy, a.d, has_shared ? a.I_s : a.T, 1, bn1 / 2);
+    ok = ok && encode_map(st, &m1[5], has_shared ? a.Ws_up : dummy, a.d, has_shared ? a.I_s : a.T, 1, bn1 / 2);
+    ok = ok && encode_map(st, &m2[0], a.h, a.I, pairs_alloc + 128, 1, a_rows);
+    ok = ok && encode_map(st, &m2[1], has_shared ? a.h_s : a.h, has_shared ? a.I_s : a.I,
+                          has_shared ? (size_t)c.max_T + 128 : pairs_alloc + 128, 1, a_rows);
+    ok = ok && encode_map(st, &m2[2], a.W_down, a.I, a.d, a.E, bn2);
+    m2[3] = m2[2];
+    ok = ok && encode_map(st, &m2[4], has_shared ? a.Ws_down : a.W_down, has_shared ? a.I_s : a.I, a.d, 1, bn2);
+    m2[5] = m2[4];
+    if (!ok) return MOE_ERR_CUDA;
+
+    // ---- tile lists
+    TileBuildArgs tb{};
+    tb.counts = a.counts; tb.offsets = a.offsets; tb.E = a.E; tb.T = a.T; tb.has_shared = has_shared;
+    tb.feat1 = bn1 / 2; tb.N1_routed = a.I; tb.N1_shared = a.I_s; tb.K1 = a.d;
+    tb.bn2 = bn2; tb.N2 = a.d; tb.K2_routed = a.I; tb.K2_shared = a.I_s;
+    tb.ksplit_routed = ks_r; tb.kchunk_routed = kchunk_r; tb.ksplit_shared = ks_s; tb.kchunk_shared = kchunk_s;
+    tb.tiles1 = ws.tiles1; tb.tiles2 = ws.tiles2; tb.n_tiles = ws.n_tiles;
+    tb.cap1 = (int)tc_max_tiles(c, 1); tb.cap2 = (int)tc_max_tiles(c, 2);
+    tb.status = ws.status;
+    build_tiles_kernel<<<1, 256, 0, s>>>(tb);
+    ++*launches;
+
+    // ---- grids: persistent, never more CTAs than tiles can exist
+    const int mblk_routed = rows / kTileRows + (rows < a.E ? rows : a.E);
+    const int mblk_shared = has_shared ? ceil_div(a.T, kTileRows) : 0;
+    const int max1 = mblk_routed * ceil_div(a.I, bn1 / 2) + mblk_shared * ceil_div(has_shared ? a.I_s : 1, bn1 / 2);
+    const int max2 = mblk_routed * ceil_div(a.d, bn2) * ks_r + mblk_shared * ceil_div(a.d, bn2) * ks_s;
+    const int ctas_per_sm = decode ? 2 : 1;
+    const int grid1 = clampi(max1, 1, sm_count * ctas_per_sm);
+    const int grid2 = clampi(max2, 1, sm_count * ctas_per_sm);
+
+    TcParams p1{};
+    p1.tiles = ws.tiles1; p1.n_tiles = ws.n_tiles; p1.E = a.E;
+    p1.N_routed = a.I; p1.N_shared = a.I_s; p1.out_routed = a.h; p1.out_shared = a.h_s;
+    p1.slab_stride_routed = 0; p1.slab_stride_shared = 0; p1.status = ws.status;
+    TcParams p2{};
+    p2.tiles = ws.tiles2; p2.n_tiles = ws.n_tiles + 1; p2.E = a.E;
+    p2.N_routed = a.d; p2.N_shared = a.d; p2.out_routed = a.o; p2.out_shared = a.o_s;
+    p2.slab_stride_routed = (unsigned long long)rows * a.d;
+    p2.slab_stride_shared = (unsigned long long)a.T * a.d;
+    p2.status = ws.status;
+
+    cudaError_t e1, e2;
+    if (decode) {
+        if (a_rows == 32) {
+            e1 = launch_tc<1, 128, 32, 5, 2, __nv_bfloat16>(m1, p1, grid1, s);
+            if (a.mid_event) cudaEventRecord(a.mid_event, s);
+            e2 = launch_tc<2, 128, 32, 5, 2, float>(m2, p2, grid2, s);
+        } else if (a_rows == 64) {
+            e1 = launch_tc<1, 128, 64, 4, 2, __nv_bfloat16>(m1, p1, grid1, s);
+            if (a.mid_event) cudaEventRecord(a.mid_event, s);
+            e2 = launch_tc<2, 128, 64, 4, 2, float>(m2, p2, grid2, s);
+        } else {
+            e1 = launch_tc<1, 128, 128, 3, 2, __nv_bfloat16>(m1, p1, grid1, s);
+            if (a.mid_event) cudaEventRecord(a.mid_event, s);
+            e2 = launch_tc<2, 128, 128, 3, 2, float>(m2, p2, grid2, s);
+        }
+        layout->o_is_f32 = 1;
+    } else {
+        e1 = launch_tc<1, 256, 128, 4, 1, __nv_bfloat16>(m1, p1, grid1, s);
+        if (a.mid_event) cudaEventRecord(a.mid_event, s);
+        e2 = launch_tc<2, 256, 128, 4, 1, float>(m2, p2, grid2, s);
+        layout->o_is_f32 = 1;
+    }
+    *launches += 2;
+    if (e1 != cudaSuccess || e2 != cudaSuccess) return MOE_ERR_CUDA;
+    layout->o_slabs = ks_r;
+    layout->o_slab_stride = (size_t)rows * a.d;
+    layout->os_slabs = ks_s;
+    layout->os_slab_stride = (size_t)a.T * a.d;
+    return MOE_OK;
+}
+
+}  // namespace lexi

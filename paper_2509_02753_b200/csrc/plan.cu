@@ -375,6 +375,17 @@ int moe_last_routing(moe_plan_t *p, int32_t *topk_idx, float *topk_w, int32_t *c
     return MOE_OK;
 }
 
+int moe_last_residual_f32(moe_plan_t *p, float *h_f32, int32_t T, void *cuda_stream) {
+    if (!p || !h_f32 || p->cfg.dtype != MOE_BF16 || T < 0 || T > p->cfg.max_T) return MOE_ERR_INVALID_ARG;
+    if (T == 0) return MOE_OK;
+    if (cudaMemcpyAsync(h_f32, p->ws.h_run, (size_t)T * p->cfg.d * sizeof(float), cudaMemcpyDeviceToDevice,
+                        (cudaStream_t)cuda_stream) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    return MOE_OK;
+}
+
 int moe_device_status(moe_plan_t *p, void *cuda_stream) {
     if (!p) return MOE_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)cuda_stream;

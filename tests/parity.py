@@ -4,7 +4,12 @@ and compare element by element.  Tolerances are the ones the tests state:
   * routing (indices, counts, offsets, permutation): bit-exact on every token whose
     k-th and (k+1)-th logits differ by more than 1e-3 (margin taken by the oracle);
   * outputs: max|y - y_ref| / rms(y_ref) <= 2e-2 for bf16 tensors, 1e-4 for fp32,
-    over the tokens whose routing agreed.
+    over the tokens whose routing agreed.  For bf16 plans that bound is asserted on the
+    value the library holds before it rounds y to bf16 (the fp32 residual stream of a
+    one-layer stack call, minus x).  The returned bf16 y itself cannot be closer than its
+    own spacing: one bf16 ulp is 2^-7 |y|, which at the largest outputs (5-6 rms) already
+    exceeds 2e-2 rms, so for it each element must meet
+    |dy| <= max(2e-2 rms, 1 bf16 ulp of y_ref).
 """
 from __future__ import annotations
 
@@ -29,6 +34,21 @@ def oracle_weights(w_host: Dict[str, Optional[torch.Tensor]]) -> orc.LayerWeight
 def rel_err(y: np.ndarray, ref: np.ndarray) -> float:
     rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
     return float(np.max(np.abs(y.astype(np.float64) - ref))) / max(rms, 1e-30)
+
+
+def assert_out_close(y_g: np.ndarray, y_ref: np.ndarray, dtype: torch.dtype, what: str = "") -> float:
+    """Output-format-aware bound: fp32 -> max|dy| <= 1e-4 rms; bf16 -> every element within
+    max(2e-2 rms, one bf16 ulp of the reference value)."""
+    tol = TOL[dtype]
+    err = rel_err(y_g, y_ref)
+    if dtype == torch.float32:
+        assert err <= tol, f"max|dy|/rms = {err:.3e} > {tol:g} {what}"
+        return err
+    rms = float(np.sqrt(np.mean(y_ref.astype(np.float64) ** 2)))
+    ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(y_ref), 1e-30))) - 7)
+    bad = np.abs(y_g - y_ref) > np.maximum(tol * rms, ulp)
+    assert not bad.any(), f"{int(bad.sum())} bf16 outputs off by more than max({tol:g} rms, 1 ulp) {what}"
+    return err
 
 
 def check_layer(plan: B.MoEPlan, x: torch.Tensor, w_dev: Dict[str, Optional[torch.Tensor]], k: int,
@@ -73,10 +93,25 @@ def check_layer(plan: B.MoEPlan, x: torch.Tensor, w_dev: Dict[str, Optional[torc
     toks = r.tokens
     keep = agree[toks]
     assert keep.any()
-    y_g = y.float().cpu().numpy()[toks][keep]
-    assert np.all(np.isfinite(y.float().cpu().numpy())), "output has non-finite entries"
-    err = rel_err(y_g, r.y[keep])
+    y_all = y.float().cpu().numpy()
+    assert np.all(np.isfinite(y_all)), "output has non-finite entries"
+    y_g = y_all[toks][keep]
+    y_ref = r.y[keep]
     tol = TOL[x.dtype] if tol is None else tol
-    assert err <= tol, f"max|dy|/rms(y_ref) = {err:.3e} > {tol:g}"
-    return {"err": err, "excluded": excluded, "agree": float(agree.mean()),
+    sched = B.SCHEDULE_NAMES.get(plan.schedule_for(T, k), "?")
+    where = f"(schedule {sched}, T={T}, k={k})"
+    if x.dtype == torch.float32:
+        err = rel_err(y_g, y_ref)
+        assert err <= tol, f"max|dy|/rms(y_ref) = {err:.3e} > {tol:g} {where}"
+        err_out = err
+    else:
+        # (a) the stated bound, on the value before the output rounding
+        h = x.clone()
+        plan.stack_forward(h, [ws], [k], renorm)
+        y32 = (plan.last_residual_f32(T) - x.float()).cpu().numpy()[toks][keep]
+        err = rel_err(y32, y_ref)
+        assert err <= tol, f"max|dy|/rms(y_ref) = {err:.3e} > {tol:g} before output rounding {where}"
+        # (b) the bf16 output: the same bound, or one unit of the output format where that is coarser
+        err_out = assert_out_close(y_g, y_ref, x.dtype, where)
+    return {"err": err, "err_out": err_out, "excluded": excluded, "agree": float(agree.mean()),
             "touched": int((counts_e > 0).sum())}

@@ -9,7 +9,7 @@ from oracle import moe_oracle as orc
 from paper_2509_02753_b200 import binding as B
 from paper_2509_02753_b200 import synth
 
-from parity import TOL, check_layer, oracle_weights, rel_err
+from parity import TOL, assert_out_close, check_layer, oracle_weights, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -18,7 +18,15 @@ DEV = "cuda"
 
 def _custom(name, d, E, I, I_shared=0, shared_gate=False, bias=0.0, L=1, k_base=2):
     return synth.Workload(name, d=d, E=E, I=I, k_base=k_base, L=L, I_shared=I_shared,
-                          shared_gate=shared_gate, router_bias_std=bias, w_std=0.05)
+                          shared_gate=shared_gate, router_bias_std=bias, w_std=0.02)
+
+
+def _small(wl, T, dtype, layer=0):
+    """Small cases are drawn on the host (so the same numbers can be studied without a GPU)."""
+    w_host = synth.make_layer(wl, layer, dtype, "cpu")
+    w_dev = {k: (None if v is None else v.to(DEV)) for k, v in w_host.items()}
+    x = synth.make_tokens(wl, T, dtype, "cpu").to(DEV)
+    return w_dev, x, w_host
 
 
 def _plan(wl, max_T, max_k, dtype, routed_scale=1.0):
@@ -73,47 +81,43 @@ def test_routing_from_given_logits_is_bit_exact(T, E, k, renorm):
 def test_tiny_layer_all_schedules(dtype):
     """T=64, d=256, E=8, I=512, top-2 renormalised, no shared expert; fp32 and bf16 variants."""
     wl = synth.WORKLOADS["tiny"]
-    w = synth.make_layer(wl, 0, dtype, DEV)
-    x = synth.make_tokens(wl, 64, dtype, DEV)
+    w, x, w_host = _small(wl, 64, dtype)
     with _plan(wl, 64, 8, dtype) as plan:
         for sched in _schedules(plan):
             plan.set_schedule(sched)
             for k, renorm in [(2, True), (1, True), (8, False), (3, False)]:
-                check_layer(plan, x, w, k, renorm)
+                check_layer(plan, x, w, k, renorm, w_host=w_host)
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("T", [1, 5, 37, 130, 700])
 def test_ragged_shapes_with_gated_shared_expert(dtype, T):
     wl = _custom("ragged", d=192, E=5, I=320, I_shared=448, shared_gate=True, bias=0.5)
-    w = synth.make_layer(wl, 0, dtype, DEV)
-    x = synth.make_tokens(wl, T, dtype, DEV)
+    w, x, w_host = _small(wl, T, dtype)
     with _plan(wl, 700, 5, dtype, routed_scale=1.25) as plan:
         for sched in _schedules(plan):
             plan.set_schedule(sched)
-            check_layer(plan, x, w, 2, False, shared_gate=True, routed_scale=1.25)
-            check_layer(plan, x, w, 5, True, shared_gate=True, routed_scale=1.25)
+            check_layer(plan, x, w, 2, False, shared_gate=True, routed_scale=1.25, w_host=w_host)
+            check_layer(plan, x, w, 5, True, shared_gate=True, routed_scale=1.25, w_host=w_host)
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_simt_handles_sizes_that_are_only_multiples_of_8(dtype):
     wl = _custom("odd", d=136, E=7, I=72, I_shared=40, shared_gate=False)
-    w = synth.make_layer(wl, 0, dtype, DEV)
-    x = synth.make_tokens(wl, 45, dtype, DEV)
+    w, x, w_host = _small(wl, 45, dtype)
     with _plan(wl, 45, 7, dtype) as plan:
         plan.set_schedule(B.MOE_SCHED_SIMT)
-        check_layer(plan, x, w, 3, True)
-        check_layer(plan, x, w, 7, False)
+        check_layer(plan, x, w, 3, True, w_host=w_host)
+        check_layer(plan, x, w, 7, False, w_host=w_host)
 
 
 def test_unused_experts_and_heavy_skew():
     """All tokens prefer two experts: most experts receive no rows, one receives nearly all."""
     wl = _custom("skew", d=256, E=16, I=256)
-    w = synth.make_layer(wl, 0, torch.bfloat16, DEV)
+    w, x, _ = _small(wl, 333, torch.bfloat16)
     w["router_bias"] = torch.zeros(16, dtype=torch.float32, device=DEV)
     w["router_bias"][3] = 20.0
     w["router_bias"][11] = 10.0
-    x = synth.make_tokens(wl, 333, torch.bfloat16, DEV)
     with _plan(wl, 333, 2, torch.bfloat16) as plan:
         for sched in _schedules(plan):
             plan.set_schedule(sched)
@@ -208,8 +212,8 @@ def test_mixtral_shaped_layer(T, k):
 # --------------------------------------------------------------------------- stack
 
 def _stack_case(wl, L, T, dtype):
-    layers = [synth.make_layer(wl, l, dtype, DEV) for l in range(L)]
-    x = synth.make_tokens(wl, T, dtype, DEV)
+    layers = [_small(wl, T, dtype, l)[0] for l in range(L)]
+    x = synth.make_tokens(wl, T, dtype, "cpu").to(DEV)
     return layers, x
 
 
@@ -231,15 +235,17 @@ def test_stack_with_per_layer_k(dtype):
             assert plan.device_status() == 0
             safe = np.all(margins > 1e-3, axis=0)
             assert safe.mean() > 0.8
-            err = rel_err(h.float().cpu().numpy()[safe], h_ref[safe])
-            assert err <= TOL[dtype], err
+            assert_out_close(h.float().cpu().numpy()[safe], h_ref[safe], dtype, "free-running stack")
+            if dtype == torch.bfloat16:     # the stated bound on the fp32 stream h was rounded from
+                h32 = plan.last_residual_f32(T).cpu().numpy()
+                assert rel_err(h32[safe], h_ref[safe]) <= TOL[dtype]
             # teacher forcing: layer l fed the oracle's h_l (rounded to the plan's dtype)
             for l in range(L):
                 h_in = torch.from_numpy(inputs[l]).to(dtype).to(DEV)
                 y = plan.layer_forward(h_in, structs[l], k_vec[l], False)
                 r = orc.moe_layer(h_in.cpu(), ows[l], k_vec[l], False, shared_gate=True)
                 ok = r.margin > 1e-3
-                assert rel_err(y.float().cpu().numpy()[ok], r.y[ok]) <= TOL[dtype]
+                assert_out_close(y.float().cpu().numpy()[ok], r.y[ok], dtype, f"teacher-forced layer {l}")
             # uniform k through the stack call equals chained layer calls plus residual
             h2 = x.clone()
             plan.stack_forward(h2, structs[:1], [3], False)
