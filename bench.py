@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the per-layer top-k MoE forward pass.
+
+    python bench.py --gpus N --steps K --warmup W [--workload qwen15 --T 8192 --k 4]
+    python bench.py --impl reference ...        (the CPU oracle, timed on the host cores)
+
+A step is one pass of the whole hot path (router, dispatch, gate/up GEMM + SwiGLU, down GEMM,
+combine + shared expert) over one batch of T synthetic tokens of the Qwen1.5-MoE-shaped layer.
+Rank 0 prints ONE JSON line.  With N > 1 (torchrun) every rank runs the same work on its own
+tokens (the layer is token-parallel: replicas, no collective on the data path); value is the
+tokens all ranks processed divided by the slowest rank's device time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2509_02753_b200 import synth  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0      # "about 8 TB/s" of the target statement
+NOMINAL_BF16_TFLOPS = 2250.0  # dense bf16 peak of a B200
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+# ------------------------------------------------------------------------------ work model
+
+def layer_flops(wl, T, k):
+    """Algorithmic flops of one layer call: T (k 6 d I + 6 d I_s + 2 d E)."""
+    return T * (k * 6 * wl.d * wl.I + 6 * wl.d * wl.I_shared + 2 * wl.d * wl.E)
+
+
+def layer_bytes(wl, T, touched, elem=2):
+    """Algorithmic bytes: weights of the experts actually touched + shared expert + router +
+    x read + y written."""
+    gate_vec = wl.d if wl.shared_gate else 0
+    w = touched * 3 * wl.d * wl.I + 3 * wl.d * wl.I_shared + wl.d * wl.E + gate_vec
+    return w * elem + 2 * T * wl.d * elem
+
+
+def ffn1_flops(wl, T, k):
+    return T * (k * 4 * wl.d * wl.I + 4 * wl.d * wl.I_shared)
+
+
+def ffn1_bytes(wl, T, k, touched, elem=2):
+    """Phase-1 GEMM: gate/up weights of touched experts + shared, activations read, h written."""
+    w = touched * 2 * wl.d * wl.I + 2 * wl.d * wl.I_shared
+    act = T * k * wl.d + T * wl.d + T * k * wl.I + T * wl.I_shared
+    return (w + act) * elem
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples during the timed region (read-only query)."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = f"/tmp/lexi_clocks_{os.getpid()}.csv"
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                c = [v.strip() for v in line.split(",")]
+                if len(c) < 9:
+                    continue
+                try:
+                    sm.append(float(c[1])); mx.append(float(c[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                    "sw_power_cap"), c[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------ reference arm
+
+def oracle_weights(w_host):
+    from oracle import moe_oracle as orc
+    return orc.LayerWeights(**{k: w_host.get(k) for k in
+                               ("router_W", "W_gate", "W_up", "W_down", "router_bias",
+                                "Ws_gate", "Ws_up", "Ws_down", "w_s")})
+
+
+def time_oracle(wl, w_host, x_host, k, n_tok, repeats=1):
+    """Wall-clock tokens/s of the oracle on the first n_tok tokens (its own batch)."""
+    from oracle import moe_oracle as orc
+    ow = oracle_weights(w_host)
+    xs = x_host[:n_tok].contiguous()
+    best = float("inf")
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        orc.moe_layer(xs, ow, k, wl.renorm, shared_gate=wl.shared_gate)
+        best = min(best, time.perf_counter() - t0)
+    return n_tok / best, best, orc.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    wl = synth.WORKLOADS[args.workload]
+    w_host = synth.make_layer(wl, 0, torch.bfloat16, "cpu")
+    n_tok = min(args.T, args.ref_tokens)
+    x_host = synth.make_tokens(wl, n_tok, torch.bfloat16, "cpu")
+    for _ in range(args.warmup):
+        time_oracle(wl, w_host, x_host, args.k, min(n_tok, 8))
+    t0 = time.perf_counter()
+    cores = 1
+    for _ in range(args.steps):
+        _, _, cores = time_oracle(wl, w_host, x_host, args.k, n_tok)
+    dt = time.perf_counter() - t0
+    value = n_tok * args.steps / dt
+    line = {
+        "impl": "reference", "metric": "MoE layer tokens/s at per-layer top-k", "value": value,
+        "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{wl.name} layer, T={args.T}, k={args.k}",
+                   "sample": f"first {n_tok} tokens per step"},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                         "sample": f"{n_tok} tokens per step x {args.steps} steps"},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------ our arm
+
+def run_case(B, plan, wl, wsets, x, y, k, steps, warmup, stage_timing, dist_barrier=None):
+    """Times `steps` layer calls (cycling the weight sets).  Returns total ms (device), stage ms."""
+    T = x.shape[0]
+    nw = len(wsets)
+    for i in range(warmup):
+        B.moe_layer_forward(plan.handle, x, wsets[i % nw], k, wl.renorm, y)
+    torch.cuda.synchronize()
+    if stage_timing:
+        B.moe_plan_set_stage_timing(plan.handle, True)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if dist_barrier:
+        dist_barrier()
+    torch.cuda.synchronize()
+    launches0 = plan.launch_count
+    start.record()
+    for i in range(steps):
+        B.moe_layer_forward(plan.handle, x, wsets[(warmup + i) % nw], k, wl.renorm, y)
+    stop.record()
+    run_case.launches = plan.launch_count - launches0
+    torch.cuda.synchronize()
+    if dist_barrier:
+        dist_barrier()
+    ms = start.elapsed_time(stop)
+    stages, n_calls = ({}, 0)
+    if stage_timing:
+        stages, n_calls = B.moe_plan_stage_times(plan.handle)
+        B.moe_plan_set_stage_timing(plan.handle, False)
+        stages = {s: v / max(n_calls, 1) for s, v in stages.items()}
+    return ms, stages
+
+
+def case_report(B, plan, wl, T, k, ms_per_step, stages, peaks, device):
+    _, _, counts, _, _, _ = plan.last_routing(T, k, device)
+    touched = int((counts > 0).sum())
+    flops = layer_flops(wl, T, k)
+    byts = layer_bytes(wl, T, touched)
+    t_hbm_nom = byts / (NOMINAL_HBM_GBS * 1e9)
+    t_tc_nom = flops / (NOMINAL_BF16_TFLOPS * 1e12)
+    t_hbm_meas = byts / (peaks["hbm_gbs"] * 1e9)
+    t_tc_meas = flops / (peaks["bf16_tflops_sustained"] * 1e12)
+    t = ms_per_step * 1e-3
+    sched = B.SCHEDULE_NAMES[plan.schedule_for(T, k)]
+    return {
+        "T": T, "k": k, "schedule": sched, "touched_experts": touched,
+        "ms": ms_per_step, "tokens_per_s": T / t,
+        "bound": "hbm" if t_hbm_meas >= t_tc_meas else "tensor",
+        "alg_bytes": byts, "alg_flops": flops,
+        "achieved_GBs": byts / t / 1e9, "achieved_TFLOPs": flops / t / 1e12,
+        "frac_roof_nominal": max(t_hbm_nom, t_tc_nom) / t,
+        "frac_roof_measured": max(t_hbm_meas, t_tc_meas) / t,
+        "stage_ms": stages,
+    }
+
+
+def run_ours(args):
+    from paper_2509_02753_b200 import binding as B
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=device)
+        dist = dist_mod
+    barrier = (lambda: dist.barrier()) if dist else None
+    B.load_library()
+    peaks = load_peaks()
+
+    wl = synth.WORKLOADS[args.workload]
+    T, k = args.T, args.k
+    dtype = torch.bfloat16
+    n_sets = args.weight_sets
+    layers = [synth.make_layer(wl, l, dtype, device, seed=rank) for l in range(n_sets)]
+    wsets = [B.make_weights(w) for w in layers]
+    max_T = max([T] + ([c[0] for c in SWEEP[wl.name]] if (args.sweep and wl.name in SWEEP) else []))
+    plan = B.MoEPlan(wl.d, wl.E, wl.I, max_T, wl.k_base, dtype, I_shared=wl.I_shared,
+                     shared_gate=wl.shared_gate)
+    x = synth.make_tokens(wl, T, dtype, device, seed=rank)
+    y = torch.empty_like(x)
+
+    # ---- main timed region (device-resident inputs), clocks sampled meanwhile
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms, stages = run_case(B, plan, wl, wsets, x, y, k, args.steps, args.warmup, True, barrier)
+    clocks = sampler.stop() if rank == 0 else {}
+    gpu_launches = run_case.launches
+    assert plan.device_status() == 0, "device status word set during the timed region"
+    if dist:
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * T * args.steps / (ms * 1e-3)
+    main = case_report(B, plan, wl, T, k, ms_per_step, stages, peaks, device)
+
+    # ---- dominant kernel: the gate/up grouped GEMM (phase 1), timed by CUDA events on the stream
+    touched = main["touched_experts"]
+    dur = stages.get("ffn1", 0.0) * 1e-3
+    if main["bound"] == "tensor":
+        ach = ffn1_flops(wl, T, k) / dur / 1e12 if dur > 0 else 0.0
+        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
+                "unit": "TFLOP/s"}
+    else:
+        ach = ffn1_bytes(wl, T, k, touched) / dur / 1e9 if dur > 0 else 0.0
+        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof["kernel"] = "ffn_tc_kernel<phase 1> (gate/up GEMM + SwiGLU)"
+    roof["launch_ms"] = stages.get("ffn1")
+    roof["peak_source"] = peaks["source"] + (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy)")
+
+    # ---- end to end through the host-buffer entry point: H2D of x and D2H of y inside the region
+    x_host = x.cpu().pin_memory()
+    y_host = torch.empty_like(x_host).pin_memory()
+    for i in range(max(3, args.warmup)):
+        B.moe_layer_forward_host(plan.handle, x_host, wsets[i % n_sets], k, wl.renorm, y_host)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if barrier:
+        barrier()
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(args.steps):
+        B.moe_layer_forward_host(plan.handle, x_host, wsets[i % n_sets], k, wl.renorm, y_host)
+    e1.record()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist:
+        t = torch.tensor([e2e_ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    bytes_io = T * wl.d * 2
+    e2e = {"value": world * T * args.steps / (e2e_ms * 1e-3), "unit": "tokens/s",
+           "h2d_bytes_per_step": bytes_io, "d2h_bytes_per_step": bytes_io,
+           "ms_per_step": e2e_ms / args.steps}
+
+    # ---- other shapes of the same workload (decode / ridge / prefill, k sweep), rank 0 at N = 1
+    sweep = []
+    if args.sweep and world == 1 and wl.name in SWEEP:
+        for (Ts, ks) in SWEEP[wl.name]:
+            xs = synth.make_tokens(wl, Ts, dtype, device, seed=1)
+            ys = torch.empty_like(xs)
+            st = max(10, min(50, args.steps))
+            ms_s, _ = run_case(B, plan, wl, wsets, xs, ys, ks, st, 5, False)
+            _, stg = run_case(B, plan, wl, wsets, xs, ys, ks, st, 2, True)
+            sweep.append(case_report(B, plan, wl, Ts, ks, ms_s / st, stg, peaks, device))
+        assert plan.device_status() == 0
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, N = 1)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        w_host = synth.to_host(layers[0])
+        n0 = min(T, 16)
+        tps0, _, cores = time_oracle(wl, w_host, x_host, k, n0)
+        n_tok = int(max(n0, min(T, tps0 * args.cpu_seconds)))
+        tps, secs, cores = time_oracle(wl, w_host, x_host, k, n_tok)
+        cpu_baseline = {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                        "sample": f"first {n_tok} of the {T} tokens, one pass, {secs:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": "MoE layer tokens/s at per-layer top-k", "value": value, "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"{wl.name} layer (d={wl.d}, E={wl.E}, I={wl.I}, shared {wl.I_shared}), "
+                                   f"T={T} tokens per GPU, k_l={k}, schedule {main['schedule']}",
+                       "cold_cache": f"inputs larger than L2: {n_sets} distinct weight sets of "
+                                     f"{layer_bytes(wl, 0, wl.E) / 1e9:.2f} GB cycled between steps",
+                       "parallelism": "replicas" if world > 1 else "single GPU"},
+            "clocks": {"sm_mhz": clocks.get("sm_mhz"), "sm_max_mhz": clocks.get("sm_max_mhz"),
+                       "reasons": clocks.get("reasons", []), "samples": clocks.get("samples", 0)},
+            "e2e": e2e, "gpu_launches": gpu_launches,
+            "roofline": roof, "cpu_baseline": cpu_baseline,
+            "layer": main, "sweep": sweep,
+            "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
+                      "bf16_tflops_burst": peaks["bf16_tflops"], "source": peaks["source"],
+                      "nominal_hbm_gbs": NOMINAL_HBM_GBS, "nominal_bf16_tflops": NOMINAL_BF16_TFLOPS},
+        }
+        print(json.dumps(line))
+    plan.close()
+    if dist:
+        dist.destroy_process_group()
+    return 0
+
+
+# (T, k) cases reported beside the headline, per workload
+SWEEP = {
+    "qwen15": [(1, 4), (1, 1), (8, 4), (64, 4), (64, 1), (2048, 4), (2048, 2), (8192, 4), (8192, 2), (8192, 1)],
+    "tiny": [(64, 2)],
+}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen15", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--T", type=int, default=8192)
+    ap.add_argument("--k", type=int, default=4)
+    ap.add_argument("--weight-sets", type=int, default=4)
+    ap.add_argument("--no-sweep", dest="sweep", action="store_false")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--ref-tokens", type=int, default=32)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

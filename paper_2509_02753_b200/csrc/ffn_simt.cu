@@ -113,6 +113,7 @@ static cudaError_t run_simt(const FfnArgs &a, cudaStream_t s, uint64_t *launches
     const int groups = a.E + (a.I_s > 0 ? 1 : 0);
     const int n1 = (max(a.I, a.I_s) + kBN - 1) / kBN;
     dim3 g1(n1, groups);
+    if (a.begin_event) cudaEventRecord(a.begin_event, s);
     // phase 1: K = d, outputs h [rows, I] / h_s [T, I_s] in the plan's dtype
     ffn_simt_kernel<T, T, true><<<g1, 256, 0, s>>>(
         (const T *)a.x_perm, (const T *)a.x, a.T, a.offsets, a.E,

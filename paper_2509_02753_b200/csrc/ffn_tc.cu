@@ -553,6 +553,7 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
     tb.status = ws.status;
     build_tiles_kernel<<<1, 256, 0, s>>>(tb);
     ++*launches;
+    if (a.begin_event) cudaEventRecord(a.begin_event, s);
 
     // ---- grids: persistent, never more CTAs than tiles can exist
     const int mblk_routed = rows / kTileRows + (rows < a.E ? rows : a.E);

@@ -83,6 +83,7 @@ struct FfnArgs {
     const void *x, *x_perm;
     const void *W_gate, *W_up, *W_down, *Ws_gate, *Ws_up, *Ws_down;
     void *h, *h_s, *o, *o_s;
+    cudaEvent_t begin_event; // recorded right before the first GEMM phase when not null
     cudaEvent_t mid_event;   // recorded between the two GEMM phases when not null
 };
 cudaError_t launch_ffn_simt(const FfnArgs &a, cudaStream_t s, uint64_t *launches);

@@ -90,11 +90,10 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
     if ((err = launch_dispatch(da, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
     if ((err = launch_gather(x, ws.perm, T * k, k, c.d, c.dtype, ws.x_perm, s, &p->launches)) != cudaSuccess)
         return MOE_ERR_CUDA;
-    mark(2);
 
     FfnArgs fa{c.dtype, T, k, c.d, c.E, c.I, c.I_shared, ws.counts, ws.offsets, x, ws.x_perm,
                w->W_gate, w->W_up, w->W_down, w->Ws_gate, w->Ws_up, w->Ws_down,
-               ws.h, ws.h_s, ws.o, ws.o_s, ev ? ev[3] : nullptr};
+               ws.h, ws.h_s, ws.o, ws.o_s, ev ? ev[2] : nullptr, ev ? ev[3] : nullptr};
     const int sched = pick_schedule(p, T, k);
     CombineArgs ca{};
     ca.dtype = c.dtype; ca.T = T; ca.k = k; ca.d = c.d;
