@@ -45,6 +45,23 @@ def load_peaks():
     return p
 
 
+def recorded_traffic(key):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel,
+    from the ncu summary under profiles/ ("traffic_key <key> <bytes> <source>:<sha256[:16]>").
+    None when no capture exists or the kernel source changed since the counters were taken."""
+    import glob
+    import hashlib
+    for path in glob.glob(os.path.join(ROOT, "profiles", "*.md")):
+        for line in open(path):
+            f = line.split()
+            if len(f) == 4 and f[0] == "traffic_key" and f[1] == key:
+                src, sha = f[3].split(":")
+                cur = hashlib.sha256(open(os.path.join(ROOT, "paper_2509_02753_b200", "csrc", src),
+                                          "rb").read()).hexdigest()[:16]
+                return int(f[2]) if cur == sha else None
+    return None
+
+
 # ------------------------------------------------------------------------------ work model
 
 def layer_flops(wl, T, k):
@@ -291,7 +308,7 @@ def run_ours(args):
         ach = ffn1_bytes(wl, T, k, touched) / dur / 1e9 if dur > 0 else 0.0
         roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = None
+    roof["traffic"] = recorded_traffic(f"{wl.name}_T{T}_k{k}_ffn1")
     roof["kernel"] = "ffn_tc_kernel<phase 1> (gate/up GEMM + SwiGLU)"
     roof["launch_ms"] = stages.get("ffn1")
     roof["peak_source"] = peaks["source"] + (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy)")
