@@ -172,6 +172,30 @@ int moe_route_from_logits(moe_plan_t *plan, const float *logits, int32_t T, int3
                           int32_t *offsets, int32_t *perm, void *cuda_stream);
 
 /*
+ * moe_dispatch_tables_static: the dispatch tables (counts, offsets, perm as defined above) from
+ * top-k indices the caller already has, WITHOUT a plan and without allocating anything.  The
+ * paper has no counterpart to this entry point; it exists for callers that cannot allocate
+ * device memory where they need the tables: a serving loop that must avoid the device-wide
+ * synchronisation cudaMalloc/cudaFree imply, or a component that is given buffers and a stream
+ * but owns no allocator and therefore cannot create a plan.
+ *
+ *   topk_idx [T, k_l] int32 device (entries outside 0..E-1 are skipped);
+ *   counts [E], offsets [E+1], perm [T*k_l] int32 device, written.
+ *   Limits: T * k_l <= 65536 and E <= 128; beyond them the call fails with MOE_ERR_SHAPE.
+ *
+ * The scratch of the three dispatch passes is a fixed 393,472-byte array in the library's
+ * device image: every GPU that loads the library holds it until the process exits.  The first
+ * call on a device looks up the array's device address (that device must be current); make that
+ * first call before starting any stream capture.  All calls on a device share the array, which
+ * keeps the previous call's contents (the call clears the one word that must start at zero), so
+ * two calls whose kernels overlap on the GPU race: keep them on one stream or order them.
+ * Calls no cudaMalloc/cudaFree.  Asynchronous on the stream.
+ * Errors: INVALID_ARG, SHAPE, CUDA.
+ */
+int moe_dispatch_tables_static(const int32_t *topk_idx, int32_t T, int32_t k_l, int32_t E,
+                               int32_t *counts, int32_t *offsets, int32_t *perm, void *cuda_stream);
+
+/*
  * moe_last_routing (test hook): copies the routing artefacts of the plan's most recent
  * layer call into caller device buffers (shapes as in moe_route_from_logits, for the T and
  * k_l of that call; logits [T, E] fp32).  Any pointer may be NULL.

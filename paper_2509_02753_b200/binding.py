@@ -27,7 +27,7 @@ EXPORTS = (
     "moe_plan_get_schedule", "moe_layer_forward", "moe_layer_forward_host", "moe_stack_forward",
     "moe_route_from_logits", "moe_last_routing", "moe_device_status", "moe_plan_launch_count",
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
-    "moe_last_residual_f32",
+    "moe_last_residual_f32", "moe_dispatch_tables_static",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
 
@@ -79,6 +79,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_last_routing.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.moe_device_status.argtypes = [vp, vp]
     lib.moe_last_residual_f32.argtypes = [vp, vp, i32, vp]
+    lib.moe_dispatch_tables_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     lib.moe_plan_set_stage_timing.argtypes = [vp, i32]
     lib.moe_plan_stage_times.argtypes = [vp, P(ctypes.c_float), P(i32)]
     lib.moe_status_string.argtypes = [ctypes.c_int]
@@ -206,6 +207,22 @@ def moe_route_from_logits(plan: int, logits: torch.Tensor, k_l: int, renorm: boo
                                                 idx.data_ptr(), wts.data_ptr(), counts.data_ptr(),
                                                 offsets.data_ptr(), perm.data_ptr(), _stream(stream)))
     return idx, wts, counts, offsets, perm
+
+
+def moe_dispatch_tables_static(topk_idx: torch.Tensor, E: int, counts: torch.Tensor,
+                               offsets: torch.Tensor, perm: torch.Tensor, stream=None) -> None:
+    """Dispatch tables from given top-k indices, no plan and no allocation: for callers that
+    cannot allocate device memory (see include/moe.h).  All outputs are caller-provided int32
+    CUDA tensors: counts [E], offsets [E+1], perm [T*k]."""
+    assert topk_idx.is_cuda and topk_idx.dtype == torch.int32 and topk_idx.is_contiguous()
+    for t in (counts, offsets, perm):
+        assert t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()
+    T, k = topk_idx.shape
+    assert counts.numel() >= E and offsets.numel() >= E + 1 and perm.numel() >= T * k
+    _check("moe_dispatch_tables_static",
+           load_library().moe_dispatch_tables_static(topk_idx.data_ptr(), T, k, E, counts.data_ptr(),
+                                                     offsets.data_ptr(), perm.data_ptr(),
+                                                     _stream(stream)))
 
 
 def moe_last_routing(plan: int, T: int, k_l: int, E: int, device, stream=None):

@@ -133,3 +133,70 @@ cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k,
 }
 
 }  // namespace lexi
+
+// ---------------------------------------------------------------------------------------
+// Dispatch tables without any allocation.
+//
+// Some callers of this library may not allocate device memory at the point where they need
+// the dispatch tables: a serving loop that must not hit the implicit device synchronisation of
+// cudaMalloc/cudaFree between decoding steps, or a host component that was handed a stream and
+// buffers by its framework but has no allocator of its own and so cannot create a plan (a plan
+// owns a cudaMalloc'ed workspace).  For them the scratch of the three dispatch passes (the
+// per-partition histograms, the inverse permutation and a status word) lives in the fixed
+// array below, which every GPU that loads this library carries until the process exits.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxPairs = 65536;                                   // T * k_l limit
+constexpr int kStaticMaxParts = kStaticMaxPairs / lexi::kPairsPerPart;   // 256
+constexpr int kStaticStatusInts = 64;                                    // status word, padded to 256 B
+constexpr int kStaticHistInts = kStaticMaxParts * lexi::kMaxExperts;     // 32768
+constexpr int kStaticScratchInts = kStaticStatusInts + kStaticHistInts + kStaticMaxPairs;   // 393,472 bytes
+
+static __device__ __align__(256) int32_t g_dispatch_scratch[kStaticScratchInts];
+
+// The array's name is only a host-side handle; the device address has to be asked for, once per
+// device, with that device current.
+constexpr int kMaxDevices = 64;
+int32_t *g_scratch_addr[kMaxDevices] = {};
+
+int32_t *static_scratch_for_current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return nullptr; }
+    if (!g_scratch_addr[dev]) {
+        int32_t *ptr = nullptr;
+        if (cudaGetSymbolAddress((void **)&ptr, g_dispatch_scratch) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        g_scratch_addr[dev] = ptr;
+    }
+    return g_scratch_addr[dev];
+}
+
+}  // namespace
+
+extern "C" int moe_dispatch_tables_static(const int32_t *topk_idx, int32_t T, int32_t k_l, int32_t E,
+                                          int32_t *counts, int32_t *offsets, int32_t *perm,
+                                          void *cuda_stream) {
+    if (!topk_idx || !counts || !offsets || !perm) return MOE_ERR_INVALID_ARG;
+    if (T < 0 || k_l < 1 || E < 1 || k_l > E) return MOE_ERR_INVALID_ARG;
+    if (E > lexi::kMaxExperts || (int64_t)T * k_l > kStaticMaxPairs) return MOE_ERR_SHAPE;
+    int32_t *scratch = static_scratch_for_current_device();
+    if (!scratch) return MOE_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // the array keeps whatever the previous call left; only the status word has to start at zero
+    // (histograms and the inverse permutation are fully rewritten for the sizes of this call)
+    if (cudaMemsetAsync(scratch, 0, sizeof(int32_t), s) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    lexi::DispatchArgs a{topk_idx, T, k_l, E, counts, offsets, perm,
+                         scratch + kStaticStatusInts + kStaticHistInts,   // inverse permutation
+                         scratch + kStaticStatusInts,                     // per-partition histograms
+                         scratch};                                        // status word
+    if (T == 0) {
+        if (cudaMemsetAsync(counts, 0, sizeof(int32_t) * E, s) != cudaSuccess ||
+            cudaMemsetAsync(offsets, 0, sizeof(int32_t) * (E + 1), s) != cudaSuccess) {
+            cudaGetLastError();
+            return MOE_ERR_CUDA;
+        }
+        return MOE_OK;
+    }
+    uint64_t launches = 0;
+    return lexi::launch_dispatch(a, s, &launches) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
