@@ -32,32 +32,43 @@ __global__ void __launch_bounds__(256) dispatch_count_kernel(DispatchArgs a, int
 }
 
 // Pass 2 (one block): counts, offsets, and for every (part, expert) the first output row.
-__global__ void __launch_bounds__(kMaxExperts) dispatch_scan_kernel(DispatchArgs a, int n_parts) {
-    __shared__ int32_t cnt[kMaxExperts];
+// Thread (e, seg): expert e = tid % 128, seg = tid / 128 owns one of 8 contiguous ranges of parts,
+// so the serial walk over the parts is 8 times shorter and loads are coalesced over e.
+constexpr int kScanSegs = 8;
+__global__ void __launch_bounds__(kMaxExperts * kScanSegs) dispatch_scan_kernel(DispatchArgs a, int n_parts) {
+    __shared__ int32_t seg_sum[kScanSegs][kMaxExperts];
     __shared__ int32_t off[kMaxExperts + 1];
-    const int e = threadIdx.x;
+    const int e = threadIdx.x % kMaxExperts, seg = threadIdx.x / kMaxExperts;
+    const int per = (n_parts + kScanSegs - 1) / kScanSegs;
+    const int p_begin = min(seg * per, n_parts), p_end = min(p_begin + per, n_parts);
     int total = 0;
     if (e < a.E)
-        for (int p = 0; p < n_parts; ++p) total += a.part_hist[(size_t)p * a.E + e];
-    cnt[e] = (e < a.E) ? total : 0;
+        for (int p = p_begin; p < p_end; ++p) total += a.part_hist[(size_t)p * a.E + e];
+    seg_sum[seg][e] = total;
     __syncthreads();
-    if (e == 0) {
+    if (threadIdx.x == 0) {
         int run = 0;
-        for (int i = 0; i < a.E; ++i) { off[i] = run; run += cnt[i]; }
+        for (int i = 0; i < a.E; ++i) {
+            off[i] = run;
+            for (int sg = 0; sg < kScanSegs; ++sg) run += seg_sum[sg][i];
+        }
         off[a.E] = run;
     }
     __syncthreads();
     if (e < a.E) {
-        a.counts[e] = cnt[e];
-        a.offsets[e] = off[e];
         int run = off[e];
-        for (int p = 0; p < n_parts; ++p) {
+        for (int sg = 0; sg < seg; ++sg) run += seg_sum[sg][e];
+        if (seg == 0) {
+            a.counts[e] = off[e + 1] - off[e];
+            a.offsets[e] = off[e];
+        }
+        for (int p = p_begin; p < p_end; ++p) {
             const int c = a.part_hist[(size_t)p * a.E + e];
             a.part_hist[(size_t)p * a.E + e] = run;
             run += c;
         }
     }
-    if (e == 0) a.offsets[a.E] = off[a.E];
+    if (threadIdx.x == 0) a.offsets[a.E] = off[a.E];
 }
 
 // Pass 3: each warp walks its part in order, 32 pairs at a time; pairs of the same expert
@@ -100,7 +111,7 @@ cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *lau
     const int n_parts = (n_pairs + kPairsPerPart - 1) / kPairsPerPart;
     const int grid = (n_parts + 7) / 8;
     dispatch_count_kernel<<<grid, 256, 0, s>>>(a, n_pairs, n_parts);
-    dispatch_scan_kernel<<<1, kMaxExperts, 0, s>>>(a, n_parts);
+    dispatch_scan_kernel<<<1, kMaxExperts * kScanSegs, 0, s>>>(a, n_parts);
     dispatch_scatter_kernel<<<grid, 256, 0, s>>>(a, n_pairs, n_parts);
     *launches += 3;
     return cudaGetLastError();

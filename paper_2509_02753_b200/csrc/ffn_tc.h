@@ -27,6 +27,14 @@ size_t tc_o_elems(const moe_config_t &c, int slabs);     // fp32-sized elements 
 size_t tc_os_elems(const moe_config_t &c, int slabs);    // ... `o_s`
 size_t tc_max_tiles(const moe_config_t &c, int phase);   // capacity of a tile list
 int    tc_state_init(TcState *st, const moe_config_t &c);
+// Encodes a TMA tensor map (into the 128-byte CUtensorMap at `map`) of a bf16 tensor
+// [groups, rows, K] with K contiguous: box 64 x box_rows x 1, 128-byte swizzle, zero fill outside.
+bool   tc_encode_bf16_map(const TcState *st, void *map, const void *ptr, uint64_t K, uint64_t rows,
+                          uint64_t groups, uint32_t box_rows);
+// Tensor-core router for large T (router_tc.cu); returns false if the shape is not covered.
+bool   tc_router_supported(const TcState *st, const RouterArgs &a);
+cudaError_t launch_router_tc(const TcState *st, const RouterArgs &a, int sm_count, cudaStream_t s,
+                             uint64_t *launches);
 int    tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, const FfnArgs &a,
                       int schedule, int sm_count, cudaStream_t s, uint64_t *launches,
                       TcOutputLayout *layout);

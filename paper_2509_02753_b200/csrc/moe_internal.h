@@ -63,6 +63,7 @@ struct RouterArgs {
     const void *x; const void *W; const float *bias; const void *w_s;
     int T, d, E, k, renorm, dtype;
     float *logits; int32_t *topk_idx; float *topk_w; float *gamma;
+    int32_t *status;
 };
 cudaError_t launch_router(const RouterArgs &a, cudaStream_t s, uint64_t *launches);
 cudaError_t launch_route_from_logits(const float *logits, int T, int E, int k, int renorm,

@@ -21,6 +21,7 @@ struct moe_plan {
     int32_t last_T = 0, last_k = 0;
     int32_t *status_host = nullptr;   // pinned
     int sm_count = 148;
+    bool use_tc_router = true;   // cleared by MOE_SCHED_SIMT so that schedule stays tensor-core free
     TcState tc{};
     // stage timing: kMaxTimedCalls sets of MOE_N_STAGES + 1 events
     bool timing = false;
@@ -81,8 +82,13 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
     mark(0);
 
     RouterArgs ra{x, w->router_W, w->router_bias, (c.I_shared > 0 && c.shared_gate) ? w->w_s : nullptr,
-                  T, c.d, c.E, k, renorm, c.dtype, ws.logits, ws.topk_idx, ws.topk_w, ws.gamma};
-    if ((err = launch_router(ra, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
+                  T, c.d, c.E, k, renorm, c.dtype, ws.logits, ws.topk_idx, ws.topk_w, ws.gamma,
+                  ws.status};
+    if (T > 512 && p->use_tc_router && tc_router_supported(&p->tc, ra))
+        err = launch_router_tc(&p->tc, ra, p->sm_count, s, &p->launches);
+    else
+        err = launch_router(ra, s, &p->launches);
+    if (err != cudaSuccess) return MOE_ERR_CUDA;
     mark(1);
 
     DispatchArgs da{ws.topk_idx, T, k, c.E, ws.counts, ws.offsets, ws.perm, ws.inv_perm,
@@ -240,6 +246,7 @@ int moe_plan_set_schedule(moe_plan_t *p, int32_t schedule) {
         (p->cfg.dtype != MOE_BF16 || !tc_shape_ok(p->cfg)))
         return MOE_ERR_SHAPE;
     p->forced_schedule = schedule;
+    p->use_tc_router = schedule != MOE_SCHED_SIMT;
     return MOE_OK;
 }
 

@@ -197,6 +197,20 @@ def test_qwen15_shaped_layer(T, k):
             check_layer(plan, x, w, k, True, shared_gate=True, w_host=w_host)
 
 
+@pytest.mark.parametrize("name,T,k", [("olmoe", 32, 8), ("olmoe", 4096, 8), ("olmoe", 4096, 3),
+                                      ("dsv2lite", 64, 6), ("dsv2lite", 1500, 4)])
+def test_olmoe_and_deepseek_shaped_layers(name, T, k):
+    """E=64 (a full 64-column router tile), no renormalisation; ungated double-width shared expert."""
+    wl = synth.WORKLOADS[name]
+    w = synth.make_layer(wl, 1, torch.bfloat16, DEV)
+    w_host = synth.to_host(w)
+    x = synth.make_tokens(wl, T, torch.bfloat16, DEV)
+    toks = None if T <= 64 else np.random.default_rng(T + k).choice(T, 40, replace=False)
+    with _plan(wl, T, wl.k_base, torch.bfloat16) as plan:
+        info = check_layer(plan, x, w, k, wl.renorm, shared_gate=wl.shared_gate, tokens=toks, w_host=w_host)
+        assert info["excluded"] < 0.05
+
+
 @pytest.mark.parametrize("T,k", [(1, 2), (16, 1), (256, 2)])
 def test_mixtral_shaped_layer(T, k):
     """d=4096, E=8, I=14336, renormalised gates; 16 sampled tokens."""
