@@ -23,19 +23,11 @@ __device__ __forceinline__ void st4(__nv_bfloat16 *p, float4 v) {
     *reinterpret_cast<uint2 *>(p) = raw;
 }
 
-template <typename OT>
-__device__ __forceinline__ float4 sum_slabs(const OT *base, int slabs, size_t stride, size_t off) {
-    float4 acc = ld4(base + off);
-    for (int s = 1; s < slabs; ++s) {
-        const float4 v = ld4(base + (size_t)s * stride + off);
-        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-    }
-    return acc;
-}
-
 // One thread per 4 consecutive features of one token.
-template <typename YT, typename OT>
+template <typename YT, typename OT, bool SLABS>
 __global__ void __launch_bounds__(256) combine_kernel(CombineArgs a) {
+    pdl_trigger();
+    pdl_wait();
     const int vec_per_row = a.d / 4;
     const size_t n_vec = (size_t)a.T * vec_per_row;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec;
@@ -43,19 +35,72 @@ __global__ void __launch_bounds__(256) combine_kernel(CombineArgs a) {
         const int t = (int)(i / vec_per_row);
         const int c = (int)(i % vec_per_row) * 4;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int j = 0; j < a.k; ++j) {
-            const float g = a.topk_w[(size_t)t * a.k + j];
-            const int r = a.inv_perm[(size_t)t * a.k + j];
-            const float4 v = sum_slabs((const OT *)a.o, a.o_slabs, a.o_slab_stride, (size_t)r * a.d + c);
-            acc.x = fmaf(g, v.x, acc.x); acc.y = fmaf(g, v.y, acc.y);
-            acc.z = fmaf(g, v.z, acc.z); acc.w = fmaf(g, v.w, acc.w);
-        }
-        acc.x *= a.routed_scale; acc.y *= a.routed_scale; acc.z *= a.routed_scale; acc.w *= a.routed_scale;
-        if (a.o_s) {
-            const float gm = a.gamma ? a.gamma[t] : 1.0f;
-            const float4 v = sum_slabs((const OT *)a.o_s, a.os_slabs, a.os_slab_stride, (size_t)t * a.d + c);
-            acc.x = fmaf(gm, v.x, acc.x); acc.y = fmaf(gm, v.y, acc.y);
-            acc.z = fmaf(gm, v.z, acc.z); acc.w = fmaf(gm, v.w, acc.w);
+        if (!SLABS) {
+            // one slab each (large calls): plain slot loop
+            for (int j = 0; j < a.k; ++j) {
+                const float g = a.topk_w[(size_t)t * a.k + j];
+                const int r = a.inv_perm[(size_t)t * a.k + j];
+                const float4 v = ld4((const OT *)a.o + (size_t)r * a.d + c);
+                acc.x = fmaf(g, v.x, acc.x); acc.y = fmaf(g, v.y, acc.y);
+                acc.z = fmaf(g, v.z, acc.z); acc.w = fmaf(g, v.w, acc.w);
+            }
+            acc.x *= a.routed_scale; acc.y *= a.routed_scale; acc.z *= a.routed_scale; acc.w *= a.routed_scale;
+            if (a.o_s) {
+                const float gm = a.gamma ? a.gamma[t] : 1.0f;
+                const float4 v = ld4((const OT *)a.o_s + (size_t)t * a.d + c);
+                acc.x = fmaf(gm, v.x, acc.x); acc.y = fmaf(gm, v.y, acc.y);
+                acc.z = fmaf(gm, v.z, acc.z); acc.w = fmaf(gm, v.w, acc.w);
+            }
+        } else {
+            const OT *o = (const OT *)a.o;
+            // four slots at a time: their gates, rows and slab loads are independent, so they are in
+            // flight together; the sums are still taken slab by slab per slot, then slot by slot
+            for (int j0 = 0; j0 < a.k; j0 += 4) {
+                float g[4];
+                int r[4];
+    #pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const bool on = j0 + u < a.k;
+                    g[u] = on ? a.topk_w[(size_t)t * a.k + j0 + u] : 0.f;
+                    r[u] = on ? a.inv_perm[(size_t)t * a.k + j0 + u] : -1;
+                }
+                float4 vs[4];
+    #pragma unroll
+                for (int u = 0; u < 4; ++u) vs[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int sl = 0; sl < a.o_slabs; ++sl) {
+                    float4 v[4];
+    #pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        v[u] = r[u] >= 0 ? ld4(o + (size_t)sl * a.o_slab_stride + (size_t)r[u] * a.d + c)
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+    #pragma unroll
+                    for (int u = 0; u < 4; ++u) { vs[u].x += v[u].x; vs[u].y += v[u].y; vs[u].z += v[u].z; vs[u].w += v[u].w; }
+                }
+    #pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (r[u] >= 0) {
+                        acc.x = fmaf(g[u], vs[u].x, acc.x); acc.y = fmaf(g[u], vs[u].y, acc.y);
+                        acc.z = fmaf(g[u], vs[u].z, acc.z); acc.w = fmaf(g[u], vs[u].w, acc.w);
+                    }
+                }
+            }
+            acc.x *= a.routed_scale; acc.y *= a.routed_scale; acc.z *= a.routed_scale; acc.w *= a.routed_scale;
+            if (a.o_s) {
+                const float gm = a.gamma ? a.gamma[t] : 1.0f;
+                const OT *os = (const OT *)a.o_s + (size_t)t * a.d + c;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int s0 = 0; s0 < a.os_slabs; s0 += 4) {
+                    float4 w4[4];
+    #pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        w4[u] = s0 + u < a.os_slabs ? ld4(os + (size_t)(s0 + u) * a.os_slab_stride)
+                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+    #pragma unroll
+                    for (int u = 0; u < 4; ++u) { v.x += w4[u].x; v.y += w4[u].y; v.z += w4[u].z; v.w += w4[u].w; }
+                }
+                acc.x = fmaf(gm, v.x, acc.x); acc.y = fmaf(gm, v.y, acc.y);
+                acc.z = fmaf(gm, v.z, acc.z); acc.w = fmaf(gm, v.w, acc.w);
+            }
         }
         const size_t off = (size_t)t * a.d + c;
         YT *y = (YT *)a.y;
@@ -79,11 +124,18 @@ cudaError_t launch_combine(const CombineArgs &a, cudaStream_t s, uint64_t *launc
     const size_t n_vec = (size_t)a.T * (a.d / 4);
     const int grid = (int)min((n_vec + 255) / 256, (size_t)148 * 16);
     const bool y_bf16 = a.dtype == MOE_BF16;
-    if (y_bf16 && a.o_is_f32) combine_kernel<__nv_bfloat16, float><<<grid, 256, 0, s>>>(a);
-    else if (y_bf16) combine_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, s>>>(a);
-    else combine_kernel<float, float><<<grid, 256, 0, s>>>(a);
+    cudaError_t e;
+    const bool slabs = a.o_slabs != 1 || (a.o_s && a.os_slabs != 1);
+    if (y_bf16 && a.o_is_f32)
+        e = slabs ? launch_chained(combine_kernel<__nv_bfloat16, float, true>, dim3(grid), dim3(256), 0, s, a.chained, a)
+                  : launch_chained(combine_kernel<__nv_bfloat16, float, false>, dim3(grid), dim3(256), 0, s, a.chained, a);
+    else if (y_bf16)
+        e = launch_chained(combine_kernel<__nv_bfloat16, __nv_bfloat16, true>, dim3(grid), dim3(256), 0, s, a.chained, a);
+    else
+        e = slabs ? launch_chained(combine_kernel<float, float, true>, dim3(grid), dim3(256), 0, s, a.chained, a)
+                  : launch_chained(combine_kernel<float, float, false>, dim3(grid), dim3(256), 0, s, a.chained, a);
     ++*launches;
-    return cudaGetLastError();
+    return e;
 }
 
 template <typename T>

@@ -1,0 +1,174 @@
+// Fused front end of small decode calls (T <= 128 tokens, T * k_l <= 2048 pairs): one launch does
+// what router + dispatch + gather + tile-list builder do for large calls.
+//
+//   every block (token t, slice s): logits of the experts r = s (mod S) for token t, fp32
+//       (Section 2: x . W_g), plus the shared expert's gate sigmoid(x . w_s);
+//   the last slice block of a token (per-token ticket, no spinning): Softmax(TopK[.]) of that token
+//       with the warp-shuffle router;
+//   the last token block to finish (global ticket): the dispatch tables counts / offsets / perm / inv_perm, the position
+//       table pos[e][t] (row of token t in expert e's segment, or -1) that lets the gate/up GEMM read
+//       x directly instead of a gathered copy, and the tile lists of both GEMM phases.
+// Order inside an expert is ascending token, as in the large-T dispatch (ballot ranks over pairs
+// taken in order), so the tables are the same stable counting sort.
+#include "ffn_tc.h"
+#include "router_common.cuh"
+
+namespace lexi {
+namespace {
+
+template <typename T>
+__global__ void __launch_bounds__(256) decode_front_kernel(FrontArgs a) {
+    extern __shared__ float xs[];                 // [d] the token's row, widened
+    __shared__ int32_t s_last;
+    __shared__ int32_t s_idx[kFrontMaxPairs];
+    __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1], cursor_s[kMaxExperts + 1];
+    __shared__ TileBuildSmem tb_sm;
+
+    pdl_trigger();
+    pdl_wait();          // x may be the previous layer's output
+    const RouterArgs &r = a.r;
+    const int t = blockIdx.x, S = gridDim.y, sl = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const T *x = (const T *)r.x + (size_t)t * r.d;
+    constexpr int V = 16 / sizeof(T);
+    for (int c = tid * V; c < r.d; c += 256 * V) {
+        const uint4 raw = *reinterpret_cast<const uint4 *>(x + c);
+        const T *xv = reinterpret_cast<const T *>(&raw);
+#pragma unroll
+        for (int v = 0; v < V; ++v) xs[c + v] = to_f32(xv[v]);
+    }
+    __syncthreads();
+
+    const int rows = r.E + (r.w_s ? 1 : 0);
+    for (int row = sl + S * warp; row < rows; row += S * 8) {
+        const T *w = (row < r.E) ? (const T *)r.W + (size_t)row * r.d : (const T *)r.w_s;
+        float acc = 0.f;
+        // eight 16-byte loads in flight per lane before any of them is consumed
+        for (int c0 = lane * V; c0 < r.d; c0 += 8 * 32 * V) {
+            uint4 raw[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int c = c0 + u * 32 * V;
+                raw[u] = c < r.d ? *reinterpret_cast<const uint4 *>(w + c) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int c = c0 + u * 32 * V;
+                if (c < r.d) {
+                    const T *wv = reinterpret_cast<const T *>(&raw[u]);
+#pragma unroll
+                    for (int v = 0; v < V; ++v) acc = fmaf(to_f32(wv[v]), xs[c + v], acc);
+                }
+            }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) {
+            if (row < r.E) r.logits[(size_t)t * r.E + row] = acc + (r.bias ? r.bias[row] : 0.f);
+            else r.gamma[t] = 1.0f / (1.0f + expf(-acc));
+        }
+    }
+
+    // ---- last slice of this token: TopK + Softmax for the token (one warp)
+    const int Tn = r.T, k = r.k, E = r.E;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(a.ticket + 1 + t, 1) == S - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (warp == 0) {
+        float z[kExpertsPerLane];
+#pragma unroll
+        for (int j = 0; j < kExpertsPerLane; ++j) {
+            const int e = lane + 32 * j;
+            z[j] = (e < E) ? __ldcg(r.logits + (size_t)t * E + e) : 0.f;
+        }
+        warp_route(z, E, k, r.renorm, lane, r.topk_idx + (size_t)t * k, r.topk_w + (size_t)t * k);
+        if (lane == 0) a.ticket[1 + t] = 0;
+    }
+    // ---- last token to be routed: dispatch tables and tile lists
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(a.ticket, 1) == Tn - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int i = tid; i < Tn * k; i += 256) s_idx[i] = __ldcg(r.topk_idx + i);
+    for (int i = tid; i < E * Tn; i += 256) a.pos[i] = -1;
+    __syncthreads();
+
+    // ---- dispatch tables.  Counts: shared-memory atomics (order does not matter for a count).
+    const int n_pairs = Tn * k;
+    for (int e = tid; e <= E; e += 256) cnt_s[e] = 0;
+    __syncthreads();
+    for (int p = tid; p < n_pairs; p += 256) atomicAdd(&cnt_s[s_idx[p]], 1);
+    __syncthreads();
+    if (warp == 0) {
+        // exclusive scan of the counts (<= 128 experts, 4 per lane), then the ranked placement:
+        // the warp takes the pairs in order, 32 at a time; pairs of one expert inside a step are
+        // ranked by lane, across steps by a cursor - a stable counting sort
+        int c[kExpertsPerLane], sum = 0;
+#pragma unroll
+        for (int j = 0; j < kExpertsPerLane; ++j) {
+            const int e = lane * kExpertsPerLane + j;
+            c[j] = e < E ? cnt_s[e] : 0;
+            sum += c[j];
+        }
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        int run = incl - sum;
+#pragma unroll
+        for (int j = 0; j < kExpertsPerLane; ++j) {
+            const int e = lane * kExpertsPerLane + j;
+            if (e < E) { off_s[e] = run; a.counts[e] = c[j]; a.offsets[e] = run; cursor_s[e] = run; }
+            run += c[j];
+        }
+        if (lane == 31) { off_s[E] = incl; a.offsets[E] = incl; }
+        __syncwarp();
+        for (int base = 0; base < n_pairs; base += 32) {
+            const int p = base + lane;
+            const int e = p < n_pairs ? s_idx[p] : -1;
+            const unsigned peers = __match_any_sync(0xffffffffu, e);
+            const int rank = __popc(peers & ((1u << lane) - 1u));
+            const int leader = __ffs(peers) - 1;
+            int first = 0;
+            if (e >= 0 && lane == leader) {
+                first = cursor_s[e];
+                cursor_s[e] = first + __popc(peers);
+            }
+            first = __shfl_sync(0xffffffffu, first, leader);
+            if (e >= 0) {
+                const int row = first + rank;
+                a.perm[row] = p;
+                a.inv_perm[p] = row;
+                a.pos[e * Tn + p / k] = row;
+            }
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    build_tiles_block(a.tb, cnt_s, off_s, tb_sm);
+    if (tid == 0) *a.ticket = 0;          // ready for the next call on this plan
+}
+
+}  // namespace
+
+cudaError_t launch_decode_front(const FrontArgs &a, cudaStream_t s, uint64_t *launches) {
+    const int T = a.r.T;
+    const int rows = a.r.E + (a.r.w_s ? 1 : 0);
+    int S = (rows + 7) / 8;                              // slices of W_g rows: one row per warp
+    S = S < 1 ? 1 : (S > 8 ? 8 : S);
+    const size_t smem = (size_t)a.r.d * sizeof(float);
+    dim3 grid(T, S);
+    cudaError_t e;
+    if (a.r.dtype == MOE_BF16) e = launch_chained(decode_front_kernel<__nv_bfloat16>, grid, dim3(256), smem, s, a.r.chained, a);
+    else e = launch_chained(decode_front_kernel<float>, grid, dim3(256), smem, s, a.r.chained, a);
+    ++*launches;
+    return e;
+}
+
+}  // namespace lexi

@@ -19,8 +19,11 @@
 // leaves through the common exit (TMEM is always freed).
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "ffn_tc.h"
 #include "tc_ptx.cuh"
+#include "tile_build.cuh"
 
 namespace lexi {
 namespace {
@@ -35,6 +38,8 @@ struct TcParams {
     void *out_routed, *out_shared;
     unsigned long long slab_stride_routed, slab_stride_shared;   // elements between split-K slabs
     int32_t *status;
+    const int32_t *pos;          // direct mode: pos[group * pos_stride + token] = output row or -1
+    int32_t pos_stride;
 };
 
 template <int A_ROWS, int BN, int STAGES>
@@ -62,9 +67,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
     static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM columns: power of two");
     static_assert(STAGES * B_BYTES >= 128 * 128, "the 128-row operand read must stay inside the allocation");
 
-    const int n_tiles = *p.n_tiles;
-    if ((int)blockIdx.x >= n_tiles) return;
-
+    pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -90,6 +93,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *slot_ptr;
+    // everything above overlaps the tail of the previous kernel; its results are needed from here on
+    pdl_wait();
+    const int n_tiles = *p.n_tiles;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -161,11 +167,16 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
             tc_fence_after();
             const bool shared = t.group == p.E;
             const int N = shared ? p.N_shared : p.N_routed;
-            const bool row_ok = row_in_tile < t.rows;
+            bool row_ok = row_in_tile < t.rows;
+            int out_row = t.row0 + row_in_tile;
+            if (p.pos != nullptr && !shared) {   // direct mode: the tile holds all tokens, keep the routed ones
+                out_row = row_ok ? p.pos[t.group * p.pos_stride + row_in_tile] : -1;
+                row_ok = out_row >= 0;
+            }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
             OutT *out = reinterpret_cast<OutT *>(shared ? p.out_shared : p.out_routed) +
                         (size_t)t.slot * (shared ? p.slab_stride_shared : p.slab_stride_routed) +
-                        (size_t)(t.row0 + row_in_tile) * N + t.n0;
+                        (size_t)(row_ok ? out_row : 0) * N + t.n0;
             if (PHASE == 1) {
 #pragma unroll 1
                 for (int c = 0; c < BN / 2; c += 16) {
@@ -232,86 +243,12 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
 }
 
 // ------------------------------------------------------------------ tile lists
-struct TileBuildArgs {
-    const int32_t *counts, *offsets;
-    int32_t E, T, has_shared;
-    int32_t feat1, N1_routed, N1_shared, K1;                     // phase 1: features per tile, I, I_s, d
-    int32_t bn2, N2, K2_routed, K2_shared;                       // phase 2: BN, d, I, I_s
-    int32_t ksplit_routed, kchunk_routed, ksplit_shared, kchunk_shared;
-    Tile *tiles1, *tiles2;
-    int32_t *n_tiles;
-    int32_t cap1, cap2;
-    int32_t *status;
-};
-
-// Group order: the shared expert first (its tiles are always full), then experts 0..E-1.
-// Inside a group: 128-row block outermost, then output-feature block, then K slab.
 __global__ void __launch_bounds__(1024) build_tiles_kernel(TileBuildArgs a) {
-    __shared__ int32_t pre1[kMaxExperts + 2], pre2[kMaxExperts + 2];
+    __shared__ TileBuildSmem sm;
     __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1];
-    const int groups = a.E + (a.has_shared ? 1 : 0);
     for (int e = threadIdx.x; e < a.E; e += blockDim.x) { cnt_s[e] = a.counts[e]; off_s[e] = a.offsets[e]; }
     __syncthreads();
-    auto group_of = [&](int slot) { return a.has_shared ? (slot == 0 ? a.E : slot - 1) : slot; };
-    auto rows_of = [&](int g) { return g == a.E ? a.T : cnt_s[g]; };
-    if (threadIdx.x == 0) {
-        int r1 = 0, r2 = 0;
-        for (int sidx = 0; sidx < groups; ++sidx) {
-            const int g = group_of(sidx);
-            const int mblk = (rows_of(g) + kTileRows - 1) / kTileRows;
-            const int n1 = ((g == a.E ? a.N1_shared : a.N1_routed) + a.feat1 - 1) / a.feat1;
-            const int n2 = (a.N2 + a.bn2 - 1) / a.bn2;
-            const int ks = g == a.E ? a.ksplit_shared : a.ksplit_routed;
-            pre1[sidx] = r1; pre2[sidx] = r2;
-            r1 += mblk * n1;
-            r2 += mblk * n2 * ks;
-        }
-        pre1[groups] = r1; pre2[groups] = r2;
-        if (r1 > a.cap1 || r2 > a.cap2) { atomicOr(a.status, kStatusBadIndex); r1 = 0; r2 = 0; pre1[groups] = 0; pre2[groups] = 0; }
-        a.n_tiles[0] = r1;
-        a.n_tiles[1] = r2;
-    }
-    __syncthreads();
-    for (int phase = 0; phase < 2; ++phase) {
-        const int32_t *pre = phase == 0 ? pre1 : pre2;
-        const int total = pre[groups];
-        for (int i = threadIdx.x; i < total; i += blockDim.x) {
-            int lo = 0, hi = groups - 1;
-            while (lo < hi) {                     // last slot with pre[slot] <= i
-                const int mid = (lo + hi + 1) >> 1;
-                if (pre[mid] <= i) lo = mid; else hi = mid - 1;
-            }
-            const int g = group_of(lo);
-            const int local = i - pre[lo];
-            const int rows = rows_of(g);
-            const int first = g == a.E ? 0 : off_s[g];
-            Tile t;
-            t.group = g; t.pad = 0;
-            if (phase == 0) {
-                const int n1 = ((g == a.E ? a.N1_shared : a.N1_routed) + a.feat1 - 1) / a.feat1;
-                const int m = local / n1, n = local % n1;
-                t.row0 = first + m * kTileRows;
-                t.rows = min(kTileRows, rows - m * kTileRows);
-                t.n0 = n * a.feat1;
-                t.k0 = 0; t.klen = a.K1; t.slot = 0;
-                a.tiles1[i] = t;
-            } else {
-                const int n2 = (a.N2 + a.bn2 - 1) / a.bn2;
-                const int ks = g == a.E ? a.ksplit_shared : a.ksplit_routed;
-                const int kchunk = g == a.E ? a.kchunk_shared : a.kchunk_routed;
-                const int K = g == a.E ? a.K2_shared : a.K2_routed;
-                const int m = local / (n2 * ks), rem = local % (n2 * ks);
-                const int n = rem / ks, sl = rem % ks;
-                t.row0 = first + m * kTileRows;
-                t.rows = min(kTileRows, rows - m * kTileRows);
-                t.n0 = n * a.bn2;
-                t.k0 = sl * kchunk;
-                t.klen = max(0, min(kchunk, K - sl * kchunk));
-                t.slot = sl;
-                a.tiles2[i] = t;
-            }
-        }
-    }
+    build_tiles_block(a, cnt_s, off_s, sm);
 }
 
 // ------------------------------------------------------------------ host side
@@ -336,6 +273,16 @@ bool encode_map(const TcState *st, CUtensorMap *m, const void *ptr, uint64_t K, 
 }
 
 int ceil_div(int a, int b) { return (a + b - 1) / b; }
+// LEXI_DECODE_BN=64|128 overrides the weight-tile height of the decode schedule (tuning aid).
+int decode_bn_override() {
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("LEXI_DECODE_BN");
+        const int n = e ? atoi(e) : 0;
+        v = (n == 64 || n == 128) ? n : 0;
+    }
+    return v;
+}
 int clampi(int v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : v); }
 int slabs_for(int K) { return clampi(ceil_div(K, 1024), 1, 8); }
 size_t decode_row_cap(const moe_config_t &c) {
@@ -345,7 +292,7 @@ size_t decode_row_cap(const moe_config_t &c) {
 }
 
 template <int PHASE, int BN, int A_ROWS, int STAGES, int MIN_CTAS, typename OutT>
-cudaError_t launch_tc(const CUtensorMap *maps, const TcParams &p, int grid, cudaStream_t s) {
+cudaError_t launch_tc(const CUtensorMap *maps, const TcParams &p, int grid, cudaStream_t s, bool chained) {
     auto kern = ffn_tc_kernel<PHASE, BN, A_ROWS, STAGES, MIN_CTAS, OutT>;
     constexpr int smem = tc_smem_bytes<A_ROWS, BN, STAGES>();
     static bool configured = false;
@@ -354,8 +301,8 @@ cudaError_t launch_tc(const CUtensorMap *maps, const TcParams &p, int grid, cuda
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<grid, 192, smem, s>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], p);
-    return cudaGetLastError();
+    return launch_chained(kern, dim3(grid), dim3(192), smem, s, chained,
+                          maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], p);
 }
 
 }  // namespace
@@ -390,9 +337,9 @@ size_t tc_max_tiles(const moe_config_t &c, int phase) {
     const size_t mblk_routed = pairs / kTileRows + (pairs < (size_t)c.E ? pairs : (size_t)c.E);
     const size_t mblk_shared = c.I_shared > 0 ? ((size_t)c.max_T + kTileRows - 1) / kTileRows : 0;
     if (phase == 1)
-        return mblk_routed * ceil_div(c.I, 64) + mblk_shared * ceil_div(c.I_shared > 0 ? c.I_shared : 64, 64) + 1;
-    return mblk_routed * ceil_div(c.d, 128) * slabs_for(c.I) +
-           mblk_shared * ceil_div(c.d, 128) * (c.I_shared > 0 ? slabs_for(c.I_shared) : 1) + 1;
+        return mblk_routed * ceil_div(c.I, 32) + mblk_shared * ceil_div(c.I_shared > 0 ? c.I_shared : 32, 32) + 1;
+    return mblk_routed * ceil_div(c.d, 64) * slabs_for(c.I) +
+           mblk_shared * ceil_div(c.d, 64) * (c.I_shared > 0 ? slabs_for(c.I_shared) : 1) + 1;
 }
 
 int tc_state_init(TcState *st, const moe_config_t &c) {
@@ -412,35 +359,58 @@ int tc_state_init(TcState *st, const moe_config_t &c) {
     return MOE_OK;
 }
 
-int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, const FfnArgs &a,
-                   int schedule, int sm_count, cudaStream_t s, uint64_t *launches,
-                   TcOutputLayout *layout) {
-    if (!st->ready) return MOE_ERR_SHAPE;
+void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs &a, int schedule,
+                      bool direct, TcSchedule *out) {
     const bool decode = schedule == MOE_SCHED_DECODE;
     const int rows = a.T * a.k;
     const bool has_shared = a.I_s > 0;
-    const size_t pairs_alloc = (size_t)c.max_T * c.max_k;
-
-    // ---- schedule parameters
-    const int bn1 = decode ? 128 : 256;          // phase-1 tile: bn1/2 gate rows + bn1/2 up rows
-    const int bn2 = decode ? 128 : 256;
-    int a_rows = 128;
-    if (decode) a_rows = a.T <= 32 ? 32 : (a.T <= 64 ? 64 : 128);
+    TcSchedule &sc = *out;
+    sc.decode = decode;
+    sc.direct = direct;
+    const int dec_bn = decode_bn_override() ? decode_bn_override() : 128;
+    sc.bn1 = decode ? dec_bn : 256;       // phase-1 tile: bn1/2 gate rows + bn1/2 up rows
+    sc.bn2 = decode ? dec_bn : 256;
+    sc.a_rows = 128;
+    if (decode) sc.a_rows = a.T <= 32 ? 32 : (a.T <= 64 ? 64 : 128);
     int ks_r = 1, ks_s = 1;
     if (decode && (size_t)rows <= decode_row_cap(c)) {
         ks_r = slabs_for(a.I);
         ks_s = has_shared ? slabs_for(a.I_s) : 1;
     }
-    const int kchunk_r = ceil_div(ceil_div(a.I, ks_r), kBK) * kBK;
-    const int kchunk_s = has_shared ? ceil_div(ceil_div(a.I_s, ks_s), kBK) * kBK : kBK;
-    ks_r = ceil_div(a.I, kchunk_r);
-    if (has_shared) ks_s = ceil_div(a.I_s, kchunk_s);
+    sc.kchunk_r = ceil_div(ceil_div(a.I, ks_r), kBK) * kBK;
+    sc.kchunk_s = has_shared ? ceil_div(ceil_div(a.I_s, ks_s), kBK) * kBK : kBK;
+    sc.ks_r = ceil_div(a.I, sc.kchunk_r);
+    sc.ks_s = has_shared ? ceil_div(a.I_s, sc.kchunk_s) : 1;
+
+    TileBuildArgs &tb = sc.tb;
+    tb = TileBuildArgs{};
+    tb.counts = a.counts; tb.offsets = a.offsets; tb.E = a.E; tb.T = a.T; tb.has_shared = has_shared;
+    tb.feat1 = sc.bn1 / 2; tb.N1_routed = a.I; tb.N1_shared = a.I_s; tb.K1 = a.d;
+    tb.bn2 = sc.bn2; tb.N2 = a.d; tb.K2_routed = a.I; tb.K2_shared = a.I_s;
+    tb.ksplit_routed = sc.ks_r; tb.kchunk_routed = sc.kchunk_r;
+    tb.ksplit_shared = sc.ks_s; tb.kchunk_shared = sc.kchunk_s;
+    tb.tiles1 = ws.tiles1; tb.tiles2 = ws.tiles2; tb.n_tiles = ws.n_tiles;
+    tb.cap1 = (int)tc_max_tiles(c, 1); tb.cap2 = (int)tc_max_tiles(c, 2);
+    tb.status = ws.status;
+    tb.direct = direct ? 1 : 0;
+}
+
+int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, const FfnArgs &a,
+                   const TcSchedule &sc, int sm_count, cudaStream_t s, uint64_t *launches,
+                   TcOutputLayout *layout) {
+    if (!st->ready) return MOE_ERR_SHAPE;
+    const bool decode = sc.decode;
+    const int rows = a.T * a.k;
+    const bool has_shared = a.I_s > 0;
+    const size_t pairs_alloc = (size_t)c.max_T * c.max_k;
+    const int bn1 = sc.bn1, bn2 = sc.bn2, a_rows = sc.a_rows, ks_r = sc.ks_r, ks_s = sc.ks_s;
 
     // ---- tensor maps
     CUtensorMap m1[6], m2[6];
     bool ok = true;
     const void *dummy = a.x;   // maps of an absent shared expert are never dereferenced
-    ok = ok && encode_map(st, &m1[0], a.x_perm, a.d, pairs_alloc + 128, 1, a_rows);
+    if (sc.direct) ok = ok && encode_map(st, &m1[0], a.x, a.d, a.T, 1, a_rows);   // every group reads x itself
+    else ok = ok && encode_map(st, &m1[0], a.x_perm, a.d, pairs_alloc + 128, 1, a_rows);
     ok = ok && encode_map(st, &m1[1], a.x, a.d, a.T, 1, a_rows);
     ok = ok && encode_map(st, &m1[2], a.W_gate, a.d, a.I, a.E, bn1 / 2);
     ok = ok && encode_map(st, &m1[3], a.W_up, a.d, a.I, a.E, bn1 / 2);
@@ -455,17 +425,11 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
     m2[5] = m2[4];
     if (!ok) return MOE_ERR_CUDA;
 
-    // ---- tile lists
-    TileBuildArgs tb{};
-    tb.counts = a.counts; tb.offsets = a.offsets; tb.E = a.E; tb.T = a.T; tb.has_shared = has_shared;
-    tb.feat1 = bn1 / 2; tb.N1_routed = a.I; tb.N1_shared = a.I_s; tb.K1 = a.d;
-    tb.bn2 = bn2; tb.N2 = a.d; tb.K2_routed = a.I; tb.K2_shared = a.I_s;
-    tb.ksplit_routed = ks_r; tb.kchunk_routed = kchunk_r; tb.ksplit_shared = ks_s; tb.kchunk_shared = kchunk_s;
-    tb.tiles1 = ws.tiles1; tb.tiles2 = ws.tiles2; tb.n_tiles = ws.n_tiles;
-    tb.cap1 = (int)tc_max_tiles(c, 1); tb.cap2 = (int)tc_max_tiles(c, 2);
-    tb.status = ws.status;
-    build_tiles_kernel<<<1, 1024, 0, s>>>(tb);
-    ++*launches;
+    // ---- tile lists (already built by the fused front end in direct mode)
+    if (!sc.direct) {
+        build_tiles_kernel<<<1, 1024, 0, s>>>(sc.tb);
+        ++*launches;
+    }
     if (a.begin_event) cudaEventRecord(a.begin_event, s);
 
     // ---- grids: persistent, never more CTAs than tiles can exist
@@ -473,7 +437,7 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
     const int mblk_shared = has_shared ? ceil_div(a.T, kTileRows) : 0;
     const int max1 = mblk_routed * ceil_div(a.I, bn1 / 2) + mblk_shared * ceil_div(has_shared ? a.I_s : 1, bn1 / 2);
     const int max2 = mblk_routed * ceil_div(a.d, bn2) * ks_r + mblk_shared * ceil_div(a.d, bn2) * ks_s;
-    const int ctas_per_sm = decode ? 2 : 1;
+    const int ctas_per_sm = decode ? (bn1 == 64 ? 3 : 2) : 1;
     const int grid1 = clampi(max1, 1, sm_count * ctas_per_sm);
     const int grid2 = clampi(max2, 1, sm_count * ctas_per_sm);
 
@@ -481,33 +445,39 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
     p1.tiles = ws.tiles1; p1.n_tiles = ws.n_tiles; p1.E = a.E;
     p1.N_routed = a.I; p1.N_shared = a.I_s; p1.out_routed = a.h; p1.out_shared = a.h_s;
     p1.slab_stride_routed = 0; p1.slab_stride_shared = 0; p1.status = ws.status;
+    p1.pos = sc.direct ? ws.pos : nullptr; p1.pos_stride = a.T;
     TcParams p2{};
     p2.tiles = ws.tiles2; p2.n_tiles = ws.n_tiles + 1; p2.E = a.E;
     p2.N_routed = a.d; p2.N_shared = a.d; p2.out_routed = a.o; p2.out_shared = a.o_s;
     p2.slab_stride_routed = (unsigned long long)rows * a.d;
     p2.slab_stride_shared = (unsigned long long)a.T * a.d;
     p2.status = ws.status;
+    p2.pos = nullptr; p2.pos_stride = 0;
 
     cudaError_t e1, e2;
+    const bool ch = a.chained && !a.mid_event;
+#define LEXI_DECODE_PAIR(BN_, AR_, ST_, CTAS_)                                                     \
+    do {                                                                                           \
+        e1 = launch_tc<1, BN_, AR_, ST_, CTAS_, __nv_bfloat16>(m1, p1, grid1, s, ch);              \
+        if (a.mid_event) cudaEventRecord(a.mid_event, s);                                          \
+        e2 = launch_tc<2, BN_, AR_, ST_, CTAS_, float>(m2, p2, grid2, s, ch);                      \
+    } while (0)
     if (decode) {
-        if (a_rows == 32) {
-            e1 = launch_tc<1, 128, 32, 5, 2, __nv_bfloat16>(m1, p1, grid1, s);
-            if (a.mid_event) cudaEventRecord(a.mid_event, s);
-            e2 = launch_tc<2, 128, 32, 5, 2, float>(m2, p2, grid2, s);
-        } else if (a_rows == 64) {
-            e1 = launch_tc<1, 128, 64, 4, 2, __nv_bfloat16>(m1, p1, grid1, s);
-            if (a.mid_event) cudaEventRecord(a.mid_event, s);
-            e2 = launch_tc<2, 128, 64, 4, 2, float>(m2, p2, grid2, s);
+        if (bn1 == 64) {
+            if (a_rows == 32) LEXI_DECODE_PAIR(64, 32, 6, 3);
+            else if (a_rows == 64) LEXI_DECODE_PAIR(64, 64, 4, 3);
+            else LEXI_DECODE_PAIR(64, 128, 3, 3);
         } else {
-            e1 = launch_tc<1, 128, 128, 3, 2, __nv_bfloat16>(m1, p1, grid1, s);
-            if (a.mid_event) cudaEventRecord(a.mid_event, s);
-            e2 = launch_tc<2, 128, 128, 3, 2, float>(m2, p2, grid2, s);
+            if (a_rows == 32) LEXI_DECODE_PAIR(128, 32, 5, 2);
+            else if (a_rows == 64) LEXI_DECODE_PAIR(128, 64, 4, 2);
+            else LEXI_DECODE_PAIR(128, 128, 3, 2);
         }
+#undef LEXI_DECODE_PAIR
         layout->o_is_f32 = 1;
     } else {
-        e1 = launch_tc<1, 256, 128, 4, 1, __nv_bfloat16>(m1, p1, grid1, s);
+        e1 = launch_tc<1, 256, 128, 4, 1, __nv_bfloat16>(m1, p1, grid1, s, ch);
         if (a.mid_event) cudaEventRecord(a.mid_event, s);
-        e2 = launch_tc<2, 256, 128, 4, 1, float>(m2, p2, grid2, s);
+        e2 = launch_tc<2, 256, 128, 4, 1, float>(m2, p2, grid2, s, ch);
         layout->o_is_f32 = 1;
     }
     *launches += 2;

@@ -2,6 +2,7 @@
 #pragma once
 
 #include "moe_internal.h"
+#include "tile_build.cuh"
 
 namespace lexi {
 
@@ -35,8 +36,27 @@ bool   tc_encode_bf16_map(const TcState *st, void *map, const void *ptr, uint64_
 bool   tc_router_supported(const TcState *st, const RouterArgs &a);
 cudaError_t launch_router_tc(const TcState *st, const RouterArgs &a, int sm_count, cudaStream_t s,
                              uint64_t *launches);
+// Tile shapes, split-K factors and the tile-list recipe of one call.
+struct TcSchedule {
+    bool decode = false, direct = false;
+    int bn1 = 256, bn2 = 256, a_rows = 128, ks_r = 1, ks_s = 1, kchunk_r = 64, kchunk_s = 64;
+    TileBuildArgs tb{};
+};
+void   tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs &a, int schedule,
+                        bool direct, TcSchedule *out);
 int    tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, const FfnArgs &a,
-                      int schedule, int sm_count, cudaStream_t s, uint64_t *launches,
+                      const TcSchedule &sc, int sm_count, cudaStream_t s, uint64_t *launches,
                       TcOutputLayout *layout);
+
+// Fused front end of small decode calls (decode_front.cu): router, top-k, dispatch tables, position
+// table and both tile lists in one launch; the last block to finish the logits does the rest.
+struct FrontArgs {
+    RouterArgs r;
+    int32_t *counts, *offsets, *perm, *inv_perm, *pos, *ticket;
+    TileBuildArgs tb;
+};
+constexpr int kFrontMaxTokens = 128;
+constexpr int kFrontMaxPairs = 2048;
+cudaError_t launch_decode_front(const FrontArgs &a, cudaStream_t s, uint64_t *launches);
 
 }  // namespace lexi

@@ -54,8 +54,33 @@ struct Workspace {
     Tile    *tiles1 = nullptr;     // phase-1 tile list
     Tile    *tiles2 = nullptr;     // phase-2 tile list
     int32_t *n_tiles = nullptr;    // [2] tile counts
-    int32_t *ticket = nullptr;     // block-arrival counter of the fused small-T router
+    int32_t *ticket = nullptr;     // block-arrival counter of the fused small-T front end
+    int32_t *pos = nullptr;        // [E, 128] direct mode: output row of (expert, token) or -1
 };
+
+#ifdef __CUDACC__
+// Programmatic dependent launch.  A kernel launched with launch_chained() may start while the
+// kernel before it on the stream is still running; it must call pdl_wait() before it reads or
+// writes anything that kernel (or any earlier one) touches, and every block must reach pdl_wait()
+// before it exits so that completion stays transitive along the chain.  pdl_trigger() lets the
+// next kernel's blocks be scheduled as soon as all blocks of this one have started.  Both are
+// no-ops in a kernel that was launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                  cudaStream_t s, bool chained, Args &&...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = chained ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
 
 // ---- launchers (each returns the cudaError_t of its launches) -------------------------
 
@@ -64,6 +89,7 @@ struct RouterArgs {
     int T, d, E, k, renorm, dtype;
     float *logits; int32_t *topk_idx; float *topk_w; float *gamma;
     int32_t *status;
+    bool chained;
 };
 cudaError_t launch_router(const RouterArgs &a, cudaStream_t s, uint64_t *launches);
 cudaError_t launch_route_from_logits(const float *logits, int T, int E, int k, int renorm,
@@ -84,6 +110,7 @@ struct FfnArgs {
     const void *x, *x_perm;
     const void *W_gate, *W_up, *W_down, *Ws_gate, *Ws_up, *Ws_down;
     void *h, *h_s, *o, *o_s;
+    bool chained;            // launch the GEMM kernels as programmatic dependents of their predecessors
     cudaEvent_t begin_event; // recorded right before the first GEMM phase when not null
     cudaEvent_t mid_event;   // recorded between the two GEMM phases when not null
 };
@@ -98,6 +125,7 @@ struct CombineArgs {
     void *y;           // mode 0: y = result.  mode 1: h_run += result, y = round(h_run).  mode 2: y += result
     float *h_run;
     int mode;
+    bool chained;
 };
 cudaError_t launch_combine(const CombineArgs &a, cudaStream_t s, uint64_t *launches);
 

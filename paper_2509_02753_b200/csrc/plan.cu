@@ -22,6 +22,8 @@ struct moe_plan {
     int32_t *status_host = nullptr;   // pinned
     int sm_count = 148;
     bool use_tc_router = true;   // cleared by MOE_SCHED_SIMT so that schedule stays tensor-core free
+    bool use_direct = true;      // fused front end + direct-x gate/up GEMM for small decode calls
+    bool use_pdl = true;         // programmatic dependent launch along the decode chain
     TcState tc{};
     // stage timing: kMaxTimedCalls sets of MOE_N_STAGES + 1 events
     bool timing = false;
@@ -83,36 +85,53 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
 
     RouterArgs ra{x, w->router_W, w->router_bias, (c.I_shared > 0 && c.shared_gate) ? w->w_s : nullptr,
                   T, c.d, c.E, k, renorm, c.dtype, ws.logits, ws.topk_idx, ws.topk_w, ws.gamma,
-                  ws.status};
-    if (T > 512 && p->use_tc_router && tc_router_supported(&p->tc, ra))
-        err = launch_router_tc(&p->tc, ra, p->sm_count, s, &p->launches);
-    else
-        err = launch_router(ra, s, &p->launches);
-    if (err != cudaSuccess) return MOE_ERR_CUDA;
-    mark(1);
-
-    DispatchArgs da{ws.topk_idx, T, k, c.E, ws.counts, ws.offsets, ws.perm, ws.inv_perm,
-                    ws.part_hist, ws.status};
-    if ((err = launch_dispatch(da, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
-    if ((err = launch_gather(x, ws.perm, T * k, k, c.d, c.dtype, ws.x_perm, s, &p->launches)) != cudaSuccess)
-        return MOE_ERR_CUDA;
-
+                  ws.status, false};
+    // kernels of a small decode call are chained as programmatic dependents (not while stage
+    // events are being recorded between them)
+    const bool chained = p->use_pdl && !ev;
     FfnArgs fa{c.dtype, T, k, c.d, c.E, c.I, c.I_shared, ws.counts, ws.offsets, x, ws.x_perm,
                w->W_gate, w->W_up, w->W_down, w->Ws_gate, w->Ws_up, w->Ws_down,
-               ws.h, ws.h_s, ws.o, ws.o_s, ev ? ev[2] : nullptr, ev ? ev[3] : nullptr};
+               ws.h, ws.h_s, ws.o, ws.o_s, false, ev ? ev[2] : nullptr, ev ? ev[3] : nullptr};
     const int sched = pick_schedule(p, T, k);
+    // small decode calls: one fused front-end launch, and the gate/up GEMM reads x directly
+    const bool direct = sched == MOE_SCHED_DECODE && p->use_direct && T <= kFrontMaxTokens &&
+                        T * k <= kFrontMaxPairs;
+    TcSchedule sc{};
+    if (sched != MOE_SCHED_SIMT) tc_make_schedule(c, ws, fa, sched, direct, &sc);
+
+    if (direct) {
+        ra.chained = chained;
+        fa.chained = chained;
+        FrontArgs fr{ra, ws.counts, ws.offsets, ws.perm, ws.inv_perm, ws.pos, ws.ticket, sc.tb};
+        if ((err = launch_decode_front(fr, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
+        mark(1);
+    } else {
+        if (T > 512 && p->use_tc_router && tc_router_supported(&p->tc, ra))
+            err = launch_router_tc(&p->tc, ra, p->sm_count, s, &p->launches);
+        else
+            err = launch_router(ra, s, &p->launches);
+        if (err != cudaSuccess) return MOE_ERR_CUDA;
+        mark(1);
+        DispatchArgs da{ws.topk_idx, T, k, c.E, ws.counts, ws.offsets, ws.perm, ws.inv_perm,
+                        ws.part_hist, ws.status};
+        if ((err = launch_dispatch(da, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
+        if ((err = launch_gather(x, ws.perm, T * k, k, c.d, c.dtype, ws.x_perm, s, &p->launches)) != cudaSuccess)
+            return MOE_ERR_CUDA;
+    }
+
     CombineArgs ca{};
     ca.dtype = c.dtype; ca.T = T; ca.k = k; ca.d = c.d;
     ca.topk_w = ws.topk_w; ca.inv_perm = ws.inv_perm;
     ca.gamma = (c.I_shared > 0 && c.shared_gate) ? ws.gamma : nullptr;
     ca.o = ws.o; ca.o_s = c.I_shared > 0 ? ws.o_s : nullptr;
     ca.routed_scale = c.routed_scale; ca.y = y; ca.h_run = ws.h_run; ca.mode = mode;
+    ca.chained = direct && chained;
     if (sched == MOE_SCHED_SIMT) {
         if ((err = launch_ffn_simt(fa, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
         ca.o_is_f32 = 1; ca.o_slabs = 1; ca.o_slab_stride = 0; ca.os_slabs = 1; ca.os_slab_stride = 0;
     } else {
         TcOutputLayout lay{};
-        const int rc = tc_ffn_forward(&p->tc, c, ws, fa, sched, p->sm_count, s, &p->launches, &lay);
+        const int rc = tc_ffn_forward(&p->tc, c, ws, fa, sc, p->sm_count, s, &p->launches, &lay);
         if (rc != MOE_OK) return rc;
         ca.o_is_f32 = lay.o_is_f32; ca.o_slabs = lay.o_slabs; ca.o_slab_stride = lay.o_slab_stride;
         ca.os_slabs = lay.os_slabs; ca.os_slab_stride = lay.os_slab_stride;
@@ -209,10 +228,11 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
     ok = ok && ws_alloc(p, &ws.tiles1, tc_max_tiles(c, 1));
     ok = ok && ws_alloc(p, &ws.tiles2, tc_max_tiles(c, 2));
     ok = ok && ws_alloc(p, &ws.n_tiles, (size_t)4);
-    ok = ok && ws_alloc(p, &ws.ticket, (size_t)4);
+    ok = ok && ws_alloc(p, &ws.ticket, (size_t)4 + kFrontMaxTokens);
+    ok = ok && ws_alloc(p, &ws.pos, (size_t)c.E * kFrontMaxTokens);
     if (ok && cudaMallocHost(&p->status_host, sizeof(int32_t)) != cudaSuccess) { cudaGetLastError(); ok = false; }
     if (ok) {
-        ok = cudaMemset(ws.status, 0, 16) == cudaSuccess && cudaMemset(ws.ticket, 0, 16) == cudaSuccess &&
+        ok = cudaMemset(ws.status, 0, 16) == cudaSuccess && cudaMemset(ws.ticket, 0, sizeof(int32_t) * (4 + kFrontMaxTokens)) == cudaSuccess &&
              cudaMemset(ws.n_tiles, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
     if (!ok) {

@@ -1,0 +1,126 @@
+// Work lists of the tensor-core grouped GEMMs, built on the device from the per-expert counts.
+#pragma once
+
+#include "moe_internal.h"
+
+namespace lexi {
+
+struct TileBuildArgs {
+    const int32_t *counts, *offsets;
+    int32_t E, T, has_shared;
+    int32_t feat1, N1_routed, N1_shared, K1;                     // phase 1: features per tile, I, I_s, d
+    int32_t bn2, N2, K2_routed, K2_shared;                       // phase 2: BN, d, I, I_s
+    int32_t ksplit_routed, kchunk_routed, ksplit_shared, kchunk_shared;
+    Tile *tiles1, *tiles2;
+    int32_t *n_tiles;
+    int32_t cap1, cap2;
+    int32_t *status;
+    // direct = 1 (T <= 128): phase 1 reads all T token rows of x for every touched expert (one
+    // row block per group, rows = T); the epilogue places each row through the position table
+    int32_t direct;
+};
+
+// Shared-memory scratch of build_tiles_block.
+struct TileBuildSmem {
+    int32_t pre1[kMaxExperts + 2], pre2[kMaxExperts + 2];
+};
+
+// Called by all threads of one block; cnt_s/off_s hold counts and offsets in shared memory.
+// Group order: the shared expert first (its tiles are always full), then experts 0..E-1.
+// Inside a group: 128-row block outermost, then output-feature block, then K slab.
+__device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const int32_t *cnt_s,
+                                                  const int32_t *off_s, TileBuildSmem &sm) {
+    const int groups = a.E + (a.has_shared ? 1 : 0);
+    auto group_of = [&](int slot) { return a.has_shared ? (slot == 0 ? a.E : slot - 1) : slot; };
+    auto rows_of = [&](int g) { return g == a.E ? a.T : cnt_s[g]; };
+    auto mblk1_of = [&](int g) {
+        const int r = rows_of(g);
+        return a.direct ? (r > 0 ? 1 : 0) : (r + kTileRows - 1) / kTileRows;
+    };
+    // tiles per group, then an exclusive scan over the (at most 129) groups by warp 0
+    const int n1_routed = (a.N1_routed + a.feat1 - 1) / a.feat1;
+    const int n1_shared = (a.N1_shared + a.feat1 - 1) / a.feat1;
+    const int n2 = (a.N2 + a.bn2 - 1) / a.bn2;
+    for (int sidx = threadIdx.x; sidx < groups; sidx += blockDim.x) {
+        const int g = group_of(sidx);
+        const int mblk = (rows_of(g) + kTileRows - 1) / kTileRows;
+        sm.pre1[sidx] = mblk1_of(g) * (g == a.E ? n1_shared : n1_routed);
+        sm.pre2[sidx] = mblk * n2 * (g == a.E ? a.ksplit_shared : a.ksplit_routed);
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        const int per = (groups + 31) / 32;
+        const int base = lane * per;
+        int s1 = 0, s2 = 0;
+        for (int i = 0; i < per; ++i)
+            if (base + i < groups) { s1 += sm.pre1[base + i]; s2 += sm.pre2[base + i]; }
+        int i1 = s1, i2 = s2;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v1 = __shfl_up_sync(0xffffffffu, i1, o), v2 = __shfl_up_sync(0xffffffffu, i2, o);
+            if (lane >= o) { i1 += v1; i2 += v2; }
+        }
+        int r1 = i1 - s1, r2 = i2 - s2;
+        for (int i = 0; i < per; ++i)
+            if (base + i < groups) {
+                const int c1 = sm.pre1[base + i], c2 = sm.pre2[base + i];
+                sm.pre1[base + i] = r1; sm.pre2[base + i] = r2;
+                r1 += c1; r2 += c2;
+            }
+        if (lane == 31) {
+            int t1 = i1, t2 = i2;
+            if (t1 > a.cap1 || t2 > a.cap2) { atomicOr(a.status, kStatusBadIndex); t1 = 0; t2 = 0; }
+            sm.pre1[groups] = t1; sm.pre2[groups] = t2;
+            a.n_tiles[0] = t1;
+            a.n_tiles[1] = t2;
+        }
+    }
+    __syncthreads();
+    for (int phase = 0; phase < 2; ++phase) {
+        const int32_t *pre = phase == 0 ? sm.pre1 : sm.pre2;
+        const int total = pre[groups];
+        for (int i = threadIdx.x; i < total; i += blockDim.x) {
+            int lo = 0, hi = groups - 1;
+            while (lo < hi) {                     // last slot with pre[slot] <= i
+                const int mid = (lo + hi + 1) >> 1;
+                if (pre[mid] <= i) lo = mid; else hi = mid - 1;
+            }
+            const int g = group_of(lo);
+            const int local = i - pre[lo];
+            const int rows = rows_of(g);
+            const int first = g == a.E ? 0 : off_s[g];
+            Tile t;
+            t.group = g; t.pad = 0;
+            if (phase == 0) {
+                const int n1 = g == a.E ? n1_shared : n1_routed;
+                const int m = local / n1, n = local % n1;
+                if (a.direct) {
+                    t.row0 = 0;
+                    t.rows = a.T;
+                } else {
+                    t.row0 = first + m * kTileRows;
+                    t.rows = min(kTileRows, rows - m * kTileRows);
+                }
+                t.n0 = n * a.feat1;
+                t.k0 = 0; t.klen = a.K1; t.slot = 0;
+                a.tiles1[i] = t;
+            } else {
+                const int ks = g == a.E ? a.ksplit_shared : a.ksplit_routed;
+                const int kchunk = g == a.E ? a.kchunk_shared : a.kchunk_routed;
+                const int K = g == a.E ? a.K2_shared : a.K2_routed;
+                const int m = local / (n2 * ks), rem = local % (n2 * ks);
+                const int n = rem / ks, sl = rem % ks;
+                t.row0 = first + m * kTileRows;
+                t.rows = min(kTileRows, rows - m * kTileRows);
+                t.n0 = n * a.bn2;
+                t.k0 = sl * kchunk;
+                t.klen = max(0, min(kchunk, K - sl * kchunk));
+                t.slot = sl;
+                a.tiles2[i] = t;
+            }
+        }
+    }
+}
+
+}  // namespace lexi
