@@ -363,6 +363,13 @@ def run_ours(args):
         cpu_baseline = {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                         "sample": f"first {n_tok} of the {T} tokens, one pass, {secs:.1f} s"}
 
+    # ---- whole stacks with uniform and per-layer k (rank 0 at N = 1)
+    stacks = []
+    if args.stacks and world == 1:
+        del layers, wsets
+        torch.cuda.empty_cache()
+        stacks = run_stacks(B, [n for n in args.stacks.split(",") if n], peaks, device, 50)
+
     if rank == 0:
         line = {
             "metric": "MoE layer tokens/s at per-layer top-k", "value": value, "unit": "tokens/s",
@@ -378,7 +385,7 @@ def run_ours(args):
                        "reasons": clocks.get("reasons", []), "samples": clocks.get("samples", 0)},
             "e2e": e2e, "gpu_launches": gpu_launches,
             "roofline": roof, "cpu_baseline": cpu_baseline,
-            "layer": main, "sweep": sweep,
+            "layer": main, "sweep": sweep, "stacks": stacks,
             "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
                       "bf16_tflops_burst": peaks["bf16_tflops"], "source": peaks["source"],
                       "nominal_hbm_gbs": NOMINAL_HBM_GBS, "nominal_bf16_tflops": NOMINAL_BF16_TFLOPS},
@@ -388,6 +395,79 @@ def run_ours(args):
     if dist:
         dist.destroy_process_group()
     return 0
+
+
+def stack_bytes_flops(wl, T, k_vec, touched_total, elem=2):
+    """Algorithmic bytes and flops of one stack pass; touched_total = sum over layers of experts hit."""
+    L = len(k_vec)
+    gate_vec = wl.d if wl.shared_gate else 0
+    w = touched_total * 3 * wl.d * wl.I + L * (3 * wl.d * wl.I_shared + wl.d * wl.E + gate_vec)
+    byts = w * elem + L * 2 * T * wl.d * elem
+    flops = sum(T * (k * 6 * wl.d * wl.I + 6 * wl.d * wl.I_shared + 2 * wl.d * wl.E) for k in k_vec)
+    return byts, flops
+
+
+def run_stacks(B, names, peaks, device, max_steps):
+    """Whole stacks (moe_stack_forward) with the pretrained uniform top-k and with the seeded
+    per-layer k vector, for every T of the workload.  Returns a list of report dicts."""
+    out = []
+    dtype = torch.bfloat16
+    for name in names:
+        wl = synth.WORKLOADS[name]
+        need = wl.L * layer_bytes(wl, 0, wl.E) * 1.15 + 4e9
+        free, _ = torch.cuda.mem_get_info(device)
+        if free < need:
+            out.append({"workload": name, "skipped": f"needs {need / 1e9:.0f} GB, {free / 1e9:.0f} GB free"})
+            continue
+        layers = [synth.make_layer(wl, l, dtype, device) for l in range(wl.L)]
+        structs = [B.make_weights(w) for w in layers]
+        k_lexi = synth.make_k_vector(wl)
+        Ts = list(wl.T_decode) + list(wl.T_prefill)
+        plan = B.MoEPlan(wl.d, wl.E, wl.I, max(Ts), wl.k_base, dtype, I_shared=wl.I_shared,
+                         shared_gate=wl.shared_gate)
+        for T in Ts:
+            x0 = synth.make_tokens(wl, T, dtype, device, seed=2)
+            h = torch.empty_like(x0)
+            for label, k_vec in (("uniform", [wl.k_base] * wl.L), ("per-layer", k_lexi)):
+                def one_pass():
+                    h.copy_(x0)        # every pass starts from the same residual stream
+                    plan.stack_forward(h, structs, k_vec, wl.renorm)
+                one_pass()                                             # warm-up
+                B.moe_plan_touched_experts(plan.handle)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                e0.record()
+                one_pass()
+                e1.record()
+                torch.cuda.synchronize()
+                one = e0.elapsed_time(e1)
+                touched = B.moe_plan_touched_experts(plan.handle)
+                steps = int(max(3, min(max_steps, 300.0 / max(one, 1e-3))))
+                for _ in range(3):
+                    one_pass()
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(steps):
+                    one_pass()
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / steps
+                B.moe_plan_touched_experts(plan.handle)
+                byts, flops = stack_bytes_flops(wl, T, k_vec, touched)
+                t = ms * 1e-3
+                t_nom = max(byts / (NOMINAL_HBM_GBS * 1e9), flops / (NOMINAL_BF16_TFLOPS * 1e12))
+                t_meas = max(byts / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops_sustained"] * 1e12))
+                out.append({"workload": name, "layers": wl.L, "T": T, "k": label, "sum_k": sum(k_vec),
+                            "touched_experts_total": touched, "steps": steps, "ms": ms,
+                            "tokens_per_s": T / t,
+                            "bound": "hbm" if byts / (peaks["hbm_gbs"] * 1e9) >= flops / (peaks["bf16_tflops_sustained"] * 1e12) else "tensor",
+                            "achieved_GBs": byts / t / 1e9, "achieved_TFLOPs": flops / t / 1e12,
+                            "frac_roof_nominal": t_nom / t, "frac_roof_measured": t_meas / t})
+        assert plan.device_status() == 0
+        plan.close()
+        del layers, structs
+        torch.cuda.empty_cache()
+    return out
 
 
 # (T, k) cases reported beside the headline, per workload
@@ -409,6 +489,8 @@ def main():
     ap.add_argument("--weight-sets", type=int, default=4)
     ap.add_argument("--no-sweep", dest="sweep", action="store_false")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stacks", default="olmoe,dsv2lite,mixtral",
+                    help="comma-separated stack workloads measured beside the headline ('' = none)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--ref-tokens", type=int, default=32)
     args = ap.parse_args()

@@ -230,6 +230,14 @@ enum { MOE_STAGE_ROUTER = 0, MOE_STAGE_DISPATCH = 1, MOE_STAGE_FFN1 = 2, MOE_STA
 int moe_plan_set_stage_timing(moe_plan_t *plan, int32_t enable);
 int moe_plan_stage_times(moe_plan_t *plan, float *ms, int32_t *n_calls);
 
+/*
+ * moe_plan_touched_experts (measurement aid): the number of routed experts that received at least
+ * one token, summed over the tensor-core layer calls since the last read; synchronises the stream,
+ * stores the sum in *total and resets it.  This is the U of the byte roofline: only the weights of
+ * touched experts have to be read.  (fp32 / SIMT calls are not counted.)
+ */
+int moe_plan_touched_experts(moe_plan_t *plan, int64_t *total, void *cuda_stream);
+
 /* Number of kernel launches this plan has issued since it was created. */
 uint64_t moe_plan_launch_count(const moe_plan_t *plan);
 

@@ -27,7 +27,7 @@ EXPORTS = (
     "moe_plan_get_schedule", "moe_layer_forward", "moe_layer_forward_host", "moe_stack_forward",
     "moe_route_from_logits", "moe_last_routing", "moe_device_status", "moe_plan_launch_count",
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
-    "moe_last_residual_f32", "moe_dispatch_tables_static",
+    "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
 
@@ -79,6 +79,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_last_routing.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.moe_device_status.argtypes = [vp, vp]
     lib.moe_last_residual_f32.argtypes = [vp, vp, i32, vp]
+    lib.moe_plan_touched_experts.argtypes = [vp, P(ctypes.c_int64), vp]
     lib.moe_dispatch_tables_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     lib.moe_plan_set_stage_timing.argtypes = [vp, i32]
     lib.moe_plan_stage_times.argtypes = [vp, P(ctypes.c_float), P(i32)]
@@ -238,6 +239,14 @@ def moe_last_routing(plan: int, T: int, k_l: int, E: int, device, stream=None):
                                            offsets.data_ptr(), perm.data_ptr(), logits.data_ptr(),
                                            _stream(stream)))
     return idx, wts, counts, offsets, perm, logits
+
+
+def moe_plan_touched_experts(plan: int, stream=None) -> int:
+    """Sum over the tensor-core layer calls since the last read of the experts that got tokens."""
+    n = ctypes.c_int64()
+    _check("moe_plan_touched_experts",
+           load_library().moe_plan_touched_experts(plan, ctypes.byref(n), _stream(stream)))
+    return int(n.value)
 
 
 def moe_plan_set_stage_timing(plan: int, enable: bool) -> None:

@@ -393,6 +393,7 @@ void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs 
     tb.cap1 = (int)tc_max_tiles(c, 1); tb.cap2 = (int)tc_max_tiles(c, 2);
     tb.status = ws.status;
     tb.direct = direct ? 1 : 0;
+    tb.stats = ws.stats;
 }
 
 int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, const FfnArgs &a,

@@ -55,6 +55,7 @@ struct Workspace {
     Tile    *tiles2 = nullptr;     // phase-2 tile list
     int32_t *n_tiles = nullptr;    // [2] tile counts
     int32_t *ticket = nullptr;     // block-arrival counter of the fused small-T front end
+    int32_t *stats = nullptr;      // [4] counters read by moe_plan_touched_experts
     int32_t *pos = nullptr;        // [E, 128] direct mode: output row of (expert, token) or -1
 };
 

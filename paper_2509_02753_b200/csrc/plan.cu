@@ -230,10 +230,11 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
     ok = ok && ws_alloc(p, &ws.n_tiles, (size_t)4);
     ok = ok && ws_alloc(p, &ws.ticket, (size_t)4 + kFrontMaxTokens);
     ok = ok && ws_alloc(p, &ws.pos, (size_t)c.E * kFrontMaxTokens);
+    ok = ok && ws_alloc(p, &ws.stats, (size_t)4);
     if (ok && cudaMallocHost(&p->status_host, sizeof(int32_t)) != cudaSuccess) { cudaGetLastError(); ok = false; }
     if (ok) {
         ok = cudaMemset(ws.status, 0, 16) == cudaSuccess && cudaMemset(ws.ticket, 0, sizeof(int32_t) * (4 + kFrontMaxTokens)) == cudaSuccess &&
-             cudaMemset(ws.n_tiles, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
+             cudaMemset(ws.n_tiles, 0, 16) == cudaSuccess && cudaMemset(ws.stats, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
     if (!ok) {
         cudaGetLastError();
@@ -409,6 +410,19 @@ int moe_last_residual_f32(moe_plan_t *p, float *h_f32, int32_t T, void *cuda_str
         cudaGetLastError();
         return MOE_ERR_CUDA;
     }
+    return MOE_OK;
+}
+
+int moe_plan_touched_experts(moe_plan_t *p, int64_t *total, void *cuda_stream) {
+    if (!p || !total) return MOE_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(p->status_host, p->ws.stats, sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemsetAsync(p->ws.stats, 0, sizeof(int32_t), s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    *total = *p->status_host;
     return MOE_OK;
 }
 

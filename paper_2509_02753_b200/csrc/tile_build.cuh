@@ -18,6 +18,7 @@ struct TileBuildArgs {
     // direct = 1 (T <= 128): phase 1 reads all T token rows of x for every touched expert (one
     // row block per group, rows = T); the epilogue places each row through the position table
     int32_t direct;
+    int32_t *stats;   // stats[0] += number of routed experts that received at least one token
 };
 
 // Shared-memory scratch of build_tiles_block.
@@ -44,6 +45,7 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
     for (int sidx = threadIdx.x; sidx < groups; sidx += blockDim.x) {
         const int g = group_of(sidx);
         const int mblk = (rows_of(g) + kTileRows - 1) / kTileRows;
+        if (a.stats && g != a.E && rows_of(g) > 0) atomicAdd(a.stats, 1);
         sm.pre1[sidx] = mblk1_of(g) * (g == a.E ? n1_shared : n1_routed);
         sm.pre2[sidx] = mblk * n2 * (g == a.E ? a.ksplit_shared : a.ksplit_routed);
     }

@@ -32,6 +32,10 @@ class Workload:
     router_bias_std: float = 0.0   # per-expert logit bias (skewed load)
     w_std: float = 0.02
     w_down_std: Optional[float] = None   # None -> w_std
+    # stacks: down projections drawn with std (2 L fan_in)^-1/2 (depth- and fan-in-scaled residual
+    # branches).  With std 0.02 the plain residual chain h <- h + MoE(h) of the DeepSeek- and
+    # Mixtral-shaped stacks overflows to inf within 6-10 layers, which turns every logit into NaN.
+    residual_init: bool = False
     k_lo: int = 1          # range of the per-layer k vector
     k_hi: int = 1
     k_budget: int = 0      # sum of the per-layer k vector
@@ -49,15 +53,15 @@ WORKLOADS: Dict[str, Workload] = {
                        shared_gate=True, renorm=False, router_bias_std=0.5,
                        k_lo=1, k_hi=4, k_budget=4, T_decode=(1, 8, 64), T_prefill=(2048, 8192)),
     # OLMoE-1B-7B-shaped stack: 16 layers, 64 experts, top-8, k_l in {2..8}, mean 5
-    "olmoe": Workload("olmoe", d=2048, E=64, I=1024, k_base=8, L=16, renorm=False,
+    "olmoe": Workload("olmoe", d=2048, E=64, I=1024, k_base=8, L=16, renorm=False, residual_init=True,
                       k_lo=2, k_hi=8, k_budget=80, T_decode=(1, 32), T_prefill=(4096,)),
     # DeepSeek-V2-Lite-shaped stack: 26 MoE layers, 64 experts, top-6, two ungated shared
     # experts of 1408 each (held as one of 2816), k_l in {2..6}, mean 4
     "dsv2lite": Workload("dsv2lite", d=2048, E=64, I=1408, k_base=6, L=26, I_shared=2816,
-                         shared_gate=False, renorm=False, router_bias_std=0.5,
+                         shared_gate=False, renorm=False, router_bias_std=0.5, residual_init=True,
                          k_lo=2, k_hi=6, k_budget=104, T_decode=(1, 64), T_prefill=(8192,)),
     # Mixtral-8x7B-shaped stack: 32 layers, 8 experts, top-2, half the layers at k = 1
-    "mixtral": Workload("mixtral", d=4096, E=8, I=14336, k_base=2, L=32, renorm=True,
+    "mixtral": Workload("mixtral", d=4096, E=8, I=14336, k_base=2, L=32, renorm=True, residual_init=True,
                         k_lo=1, k_hi=2, k_budget=48, T_decode=(1, 16, 256),
                         T_prefill=(4096, 16384)),
 }
@@ -89,6 +93,10 @@ def make_layer(wl: Workload, layer: int, dtype: torch.dtype, device="cpu", seed:
     """Weights of one MoE layer as a dict of tensors on ``device``."""
     s = lambda name: _seed(seed, wl.name, layer, name)
     dn = wl.w_down_std if wl.w_down_std is not None else wl.w_std
+    dn_s = dn
+    if wl.residual_init:
+        dn = (2.0 * wl.L * wl.I) ** -0.5
+        dn_s = (2.0 * wl.L * wl.I_shared) ** -0.5 if wl.I_shared > 0 else dn
     w: Dict[str, Optional[torch.Tensor]] = {
         "router_W": _normal((wl.E, wl.d), wl.w_std, s("router_W"), dtype, device),
         "router_bias": None,
@@ -103,7 +111,7 @@ def make_layer(wl: Workload, layer: int, dtype: torch.dtype, device="cpu", seed:
     if wl.I_shared > 0:
         w["Ws_gate"] = _normal((wl.I_shared, wl.d), wl.w_std, s("Ws_gate"), dtype, device)
         w["Ws_up"] = _normal((wl.I_shared, wl.d), wl.w_std, s("Ws_up"), dtype, device)
-        w["Ws_down"] = _normal((wl.d, wl.I_shared), dn, s("Ws_down"), dtype, device)
+        w["Ws_down"] = _normal((wl.d, wl.I_shared), dn_s, s("Ws_down"), dtype, device)
         if wl.shared_gate:
             w["w_s"] = _normal((wl.d,), wl.w_std, s("w_s"), dtype, device)
     return w
