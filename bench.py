@@ -26,7 +26,7 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
-from paper_2509_02753_b200 import synth  # noqa: E402
+from paper_2509_02753_b200 import replicas, synth  # noqa: E402
 
 NOMINAL_HBM_GBS = 8000.0      # "about 8 TB/s" of the target statement
 NOMINAL_BF16_TFLOPS = 2250.0  # dense bf16 peak of a B200
@@ -289,12 +289,9 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else {}
     gpu_launches = run_case.launches
     assert plan.device_status() == 0, "device status word set during the timed region"
-    if dist:
-        t = torch.tensor([ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms, tokens_done = replicas.aggregate(ms, T * args.steps, dist, device)
     ms_per_step = ms / args.steps
-    value = world * T * args.steps / (ms * 1e-3)
+    value = tokens_done / (ms * 1e-3)
     main = case_report(B, plan, wl, T, k, ms_per_step, stages, peaks, device)
 
     # ---- dominant kernel: the gate/up grouped GEMM (phase 1), timed by CUDA events on the stream
@@ -331,12 +328,9 @@ def run_ours(args):
     if barrier:
         barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if dist:
-        t = torch.tensor([e2e_ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms, e2e_tokens = replicas.aggregate(e2e_ms, T * args.steps, dist, device)
     bytes_io = T * wl.d * 2
-    e2e = {"value": world * T * args.steps / (e2e_ms * 1e-3), "unit": "tokens/s",
+    e2e = {"value": e2e_tokens / (e2e_ms * 1e-3), "unit": "tokens/s",
            "h2d_bytes_per_step": bytes_io, "d2h_bytes_per_step": bytes_io,
            "ms_per_step": e2e_ms / args.steps}
 
