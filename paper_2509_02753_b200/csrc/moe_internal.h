@@ -83,6 +83,8 @@ inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 bloc
 }
 #endif
 
+struct TileBuildArgs;
+
 // ---- launchers (each returns the cudaError_t of its launches) -------------------------
 
 struct RouterArgs {
@@ -101,9 +103,14 @@ struct DispatchArgs {
     const int32_t *topk_idx; int T, k, E;
     int32_t *counts, *offsets, *perm, *inv_perm, *part_hist; int32_t *status;
 };
-cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches);
+// tiles != NULL (and a call of at most kBlockDispatchPairs pairs): one block does the dispatch and then builds the
+// tensor-core tile lists; returns with both done.  Otherwise the three-kernel dispatch only.
+cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained = false,
+                            const TileBuildArgs *tiles = nullptr);
+constexpr int kBlockDispatchPairs = 8192;
 cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k, int d, int dtype,
-                          void *x_perm, cudaStream_t s, uint64_t *launches);
+                          void *x_perm, cudaStream_t s, uint64_t *launches, bool chained = false,
+                          const TileBuildArgs *tiles = nullptr);   // tiles: also build the tile lists
 
 struct FfnArgs {
     int dtype, T, k, d, E, I, I_s;

@@ -99,9 +99,9 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
     TcSchedule sc{};
     if (sched != MOE_SCHED_SIMT) tc_make_schedule(c, ws, fa, sched, direct, &sc);
 
+    ra.chained = chained;
+    fa.chained = chained && sched != MOE_SCHED_SIMT;
     if (direct) {
-        ra.chained = chained;
-        fa.chained = chained;
         FrontArgs fr{ra, ws.counts, ws.offsets, ws.perm, ws.inv_perm, ws.pos, ws.ticket, sc.tb};
         if ((err = launch_decode_front(fr, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
         mark(1);
@@ -114,9 +114,15 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
         mark(1);
         DispatchArgs da{ws.topk_idx, T, k, c.E, ws.counts, ws.offsets, ws.perm, ws.inv_perm,
                         ws.part_hist, ws.status};
-        if ((err = launch_dispatch(da, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
-        if ((err = launch_gather(x, ws.perm, T * k, k, c.d, c.dtype, ws.x_perm, s, &p->launches)) != cudaSuccess)
+        const bool fuse_tiles = sched != MOE_SCHED_SIMT && T * k <= kBlockDispatchPairs;
+        if ((err = launch_dispatch(da, s, &p->launches, chained, fuse_tiles ? &sc.tb : nullptr)) != cudaSuccess)
             return MOE_ERR_CUDA;
+        // larger calls: the tile lists are built by a few extra blocks of the gather launch
+        const bool tiles_in_gather = sched != MOE_SCHED_SIMT && !fuse_tiles;
+        if ((err = launch_gather(x, ws.perm, T * k, k, c.d, c.dtype, ws.x_perm, s, &p->launches, chained,
+                                 tiles_in_gather ? &sc.tb : nullptr)) != cudaSuccess)
+            return MOE_ERR_CUDA;
+        sc.tiles_built = fuse_tiles || tiles_in_gather;
     }
 
     CombineArgs ca{};
@@ -125,7 +131,7 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
     ca.gamma = (c.I_shared > 0 && c.shared_gate) ? ws.gamma : nullptr;
     ca.o = ws.o; ca.o_s = c.I_shared > 0 ? ws.o_s : nullptr;
     ca.routed_scale = c.routed_scale; ca.y = y; ca.h_run = ws.h_run; ca.mode = mode;
-    ca.chained = direct && chained;
+    ca.chained = chained;
     if (sched == MOE_SCHED_SIMT) {
         if ((err = launch_ffn_simt(fa, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
         ca.o_is_f32 = 1; ca.o_slabs = 1; ca.o_slab_stride = 0; ca.os_slabs = 1; ca.os_slab_stride = 0;

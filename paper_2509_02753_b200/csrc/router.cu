@@ -18,6 +18,8 @@ namespace lexi {
 // ---------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256) router_token_kernel(RouterArgs a) {
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ float smem[];
     float *xs = smem;                 // [d]
     float *zs = smem + a.d;           // [E + 1]
@@ -78,6 +80,8 @@ constexpr int kRtChunk = 64;
 
 template <typename T>
 __global__ void __launch_bounds__(256) router_tile_kernel(RouterArgs a) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float xs[kRtTokens][kRtChunk + 1];
     __shared__ float ws[kMaxExperts][kRtChunk + 1];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -159,21 +163,22 @@ __global__ void __launch_bounds__(256) route_logits_kernel(const float *logits, 
 cudaError_t launch_router(const RouterArgs &a, cudaStream_t s, uint64_t *launches) {
     if (a.T <= 0) return cudaSuccess;
     const bool small = a.T <= 512;
+    cudaError_t e;
     if (small) {
         const size_t smem = (size_t)(a.d + a.E + 1) * sizeof(float);
         if (a.dtype == MOE_BF16)
-            router_token_kernel<__nv_bfloat16><<<a.T, 256, smem, s>>>(a);
+            e = launch_chained(router_token_kernel<__nv_bfloat16>, dim3(a.T), dim3(256), smem, s, a.chained, a);
         else
-            router_token_kernel<float><<<a.T, 256, smem, s>>>(a);
+            e = launch_chained(router_token_kernel<float>, dim3(a.T), dim3(256), smem, s, a.chained, a);
     } else {
         const int grid = (a.T + kRtTokens - 1) / kRtTokens;
         if (a.dtype == MOE_BF16)
-            router_tile_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(a);
+            e = launch_chained(router_tile_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, s, a.chained, a);
         else
-            router_tile_kernel<float><<<grid, 256, 0, s>>>(a);
+            e = launch_chained(router_tile_kernel<float>, dim3(grid), dim3(256), 0, s, a.chained, a);
     }
     ++*launches;
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_route_from_logits(const float *logits, int T, int E, int k, int renorm,

@@ -33,9 +33,8 @@ struct RouterTcParams {
 __global__ void __launch_bounds__(192, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const __grid_constant__ CUtensorMap map_ws, const RouterTcParams p) {
+    pdl_trigger();
     const int n_tiles = (p.T + 127) / 128;
-    if ((int)blockIdx.x >= n_tiles) return;
-
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -62,6 +61,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = *slot_ptr;
     const int nk = (p.d + kBK - 1) / kBK;
+    pdl_wait();          // x may be the previous layer's output
 
     if (warp == 0) {
         if (lane == 0) {
@@ -218,9 +218,10 @@ cudaError_t launch_router_tc(const TcState *st, const RouterArgs &a, int sm_coun
                      a.logits, a.topk_idx, a.topk_w, a.gamma, a.status};
     const int n_tiles = (a.T + 127) / 128;
     const int grid = n_tiles < sm_count ? n_tiles : sm_count;
-    router_tc_kernel<<<grid, 192, kRSmem, s>>>(mx, mw, mg, p);
+    const cudaError_t e = launch_chained(router_tc_kernel, dim3(grid), dim3(192), (size_t)kRSmem, s, a.chained,
+                                         mx, mw, mg, p);
     ++*launches;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace lexi

@@ -29,8 +29,11 @@ struct TileBuildSmem {
 // Called by all threads of one block; cnt_s/off_s hold counts and offsets in shared memory.
 // Group order: the shared expert first (its tiles are always full), then experts 0..E-1.
 // Inside a group: 128-row block outermost, then output-feature block, then K slab.
+// Several blocks may share the work: block `rank` of `n_blocks` writes every n_blocks-th stripe of
+// the lists (each block recomputes the small prefix); rank 0 publishes the tile counts.
 __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const int32_t *cnt_s,
-                                                  const int32_t *off_s, TileBuildSmem &sm) {
+                                                  const int32_t *off_s, TileBuildSmem &sm,
+                                                  int rank = 0, int n_blocks = 1) {
     const int groups = a.E + (a.has_shared ? 1 : 0);
     auto group_of = [&](int slot) { return a.has_shared ? (slot == 0 ? a.E : slot - 1) : slot; };
     auto rows_of = [&](int g) { return g == a.E ? a.T : cnt_s[g]; };
@@ -45,7 +48,7 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
     for (int sidx = threadIdx.x; sidx < groups; sidx += blockDim.x) {
         const int g = group_of(sidx);
         const int mblk = (rows_of(g) + kTileRows - 1) / kTileRows;
-        if (a.stats && g != a.E && rows_of(g) > 0) atomicAdd(a.stats, 1);
+        if (rank == 0 && a.stats && g != a.E && rows_of(g) > 0) atomicAdd(a.stats, 1);
         sm.pre1[sidx] = mblk1_of(g) * (g == a.E ? n1_shared : n1_routed);
         sm.pre2[sidx] = mblk * n2 * (g == a.E ? a.ksplit_shared : a.ksplit_routed);
     }
@@ -74,15 +77,17 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
             int t1 = i1, t2 = i2;
             if (t1 > a.cap1 || t2 > a.cap2) { atomicOr(a.status, kStatusBadIndex); t1 = 0; t2 = 0; }
             sm.pre1[groups] = t1; sm.pre2[groups] = t2;
-            a.n_tiles[0] = t1;
-            a.n_tiles[1] = t2;
+            if (rank == 0) {
+                a.n_tiles[0] = t1;
+                a.n_tiles[1] = t2;
+            }
         }
     }
     __syncthreads();
     for (int phase = 0; phase < 2; ++phase) {
         const int32_t *pre = phase == 0 ? sm.pre1 : sm.pre2;
         const int total = pre[groups];
-        for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        for (int i = rank * blockDim.x + threadIdx.x; i < total; i += n_blocks * blockDim.x) {
             int lo = 0, hi = groups - 1;
             while (lo < hi) {                     // last slot with pre[slot] <= i
                 const int mid = (lo + hi + 1) >> 1;
