@@ -42,9 +42,18 @@ struct TcParams {
     int32_t pos_stride;
 };
 
+// Phase-2 tiles of the prefill schedule pass their fp32 output through a per-warp staging buffer
+// (32 rows x 32 columns, row pitch 36 floats) so that global stores are row-contiguous.
+constexpr int kStagePitch = 36;
+constexpr int kStageBytes = 4 * 32 * kStagePitch * 4;
+
+template <int PHASE, int BN, typename OutT>
+__host__ __device__ constexpr bool tc_staged_out() { return PHASE == 2 && BN == 256 && sizeof(OutT) == 4; }
+
 template <int A_ROWS, int BN, int STAGES>
-constexpr int tc_smem_bytes() {
-    return STAGES * (A_ROWS * 128 + BN * 128) + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int tc_smem_bytes(bool staged) {
+    return STAGES * (A_ROWS * 128 + BN * 128) + 1024 /* alignment slack */ + 256 /* barriers */ +
+           (staged ? kStageBytes : 0);
 }
 
 __device__ __forceinline__ float silu_mul(float g, float u) {
@@ -202,6 +211,38 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
                             *reinterpret_cast<uint4 *>(out + c + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
                     }
                 }
+            } else if constexpr (tc_staged_out<PHASE, BN, OutT>()) {
+                // each lane parks its row's 32 columns in shared memory; the warp then writes them
+                // out four rows per instruction, 128 contiguous bytes per row
+                float *stg = reinterpret_cast<float *>(smem_raw + (bar_base + 256u - raw)) + q * 32 * kStagePitch;
+                OutT *wbase = reinterpret_cast<OutT *>(shared ? p.out_shared : p.out_routed) +
+                              (size_t)t.slot * (shared ? p.slab_stride_shared : p.slab_stride_routed) +
+                              (size_t)(t.row0 + q * 32) * N + t.n0;
+                const int rows_here = t.rows - q * 32;       // valid rows among this warp's 32
+                const int rr0 = lane >> 3, cc = 4 * (lane & 7);
+#pragma unroll 1
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t v0[16], v1[16];
+                    tmem_ld16(taddr + c, v0);
+                    tmem_ld16(taddr + c + 16, v1);
+                    tmem_ld_wait();
+                    uint4 *wr = reinterpret_cast<uint4 *>(stg + lane * kStagePitch);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        wr[i] = make_uint4(v0[4 * i], v0[4 * i + 1], v0[4 * i + 2], v0[4 * i + 3]);
+                        wr[4 + i] = make_uint4(v1[4 * i], v1[4 * i + 1], v1[4 * i + 2], v1[4 * i + 3]);
+                    }
+                    __syncwarp();
+                    const bool col_ok = t.n0 + c + cc + 4 <= N;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int rr = 4 * j + rr0;
+                        const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * kStagePitch + cc);
+                        if (rr < rows_here && col_ok)
+                            *reinterpret_cast<uint4 *>(wbase + (size_t)rr * N + c + cc) = val;
+                    }
+                    __syncwarp();
+                }
             } else {
 #pragma unroll 1
                 for (int c = 0; c < BN; c += 16) {
@@ -302,7 +343,7 @@ size_t decode_row_cap(const moe_config_t &c) {
 template <int PHASE, int BN, int A_ROWS, int STAGES, int MIN_CTAS, typename OutT>
 cudaError_t launch_tc(const CUtensorMap *maps, const TcParams &p, int grid, cudaStream_t s, bool chained) {
     auto kern = ffn_tc_kernel<PHASE, BN, A_ROWS, STAGES, MIN_CTAS, OutT>;
-    constexpr int smem = tc_smem_bytes<A_ROWS, BN, STAGES>();
+    constexpr int smem = tc_smem_bytes<A_ROWS, BN, STAGES>(tc_staged_out<PHASE, BN, OutT>());
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
