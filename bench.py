@@ -357,6 +357,34 @@ def run_ours(args):
         cpu_baseline = {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                         "sample": f"first {n_tok} of the {T} tokens, one pass, {secs:.1f} s"}
 
+    # ---- Stage 1 (Algorithm 1) on this layer: all k from one expert pass vs one layer call per k
+    stage1 = None
+    if args.sweep and world == 1:
+        Tp = min(2048, max_T)
+        xp = synth.make_tokens(wl, Tp, dtype, device, seed=3)
+        yp = torch.empty_like(xp)
+        kb = wl.k_base
+        for _ in range(3):
+            plan.profile_layer(xp, wsets[0], kb, wl.renorm)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        e0.record()
+        for i in range(reps):
+            plan.profile_layer(xp, wsets[i % n_sets], kb, wl.renorm)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_prof = e0.elapsed_time(e1) / reps
+        e0.record()
+        for i in range(reps):
+            for kk in list(range(1, kb + 1)) + [kb]:       # |T| perturbed passes + the base pass
+                B.moe_layer_forward(plan.handle, xp, wsets[i % n_sets], kk, wl.renorm, yp)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_alg1 = e0.elapsed_time(e1) / reps
+        stage1 = {"T": Tp, "k_base": kb, "ms_per_sample_prefix_sums": ms_prof,
+                  "ms_per_sample_one_call_per_k": ms_alg1, "speedup": ms_alg1 / ms_prof,
+                  "samples_tokens_per_s": Tp / (ms_prof * 1e-3)}
+
     # ---- whole stacks with uniform and per-layer k (rank 0 at N = 1)
     stacks = []
     if args.stacks and world == 1:
@@ -379,7 +407,7 @@ def run_ours(args):
                        "reasons": clocks.get("reasons", []), "samples": clocks.get("samples", 0)},
             "e2e": e2e, "gpu_launches": gpu_launches,
             "roofline": roof, "cpu_baseline": cpu_baseline,
-            "layer": main, "sweep": sweep, "stacks": stacks,
+            "layer": main, "sweep": sweep, "stacks": stacks, "stage1": stage1,
             "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
                       "bf16_tflops_burst": peaks["bf16_tflops"], "source": peaks["source"],
                       "nominal_hbm_gbs": NOMINAL_HBM_GBS, "nominal_bf16_tflops": NOMINAL_BF16_TFLOPS},

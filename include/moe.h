@@ -160,6 +160,22 @@ int moe_stack_forward(moe_plan_t *plan, void *h, const moe_layer_weights_t *laye
                       void *cuda_stream);
 
 /*
+ * moe_profile_layer: one Monte-Carlo sample of the paper's Stage 1 (Algorithm 1, "Per Layer Top-k
+ * Perturbation Loss Computation") for ALL k of the search space {1..k_base} at once:
+ *
+ *     delta[k-1] = || f_moe(X; k) - f_moe(X; k_base) ||_F        k = 1 .. k_base  (delta[k_base-1] = 0)
+ *
+ * Algorithm 1 runs the module once per k; because the top-k sets are nested in k, this call runs
+ * the experts once at k_base and forms every f_moe(X; k) from prefix sums over the slot outputs
+ * (in fp32, before any rounding of y).  x [T, d] device is the sample X (the caller draws it,
+ * X ~ N(0,1) in the paper, and averages delta over its iterations).  delta: HOST array of k_base
+ * doubles.  base_norm (host, may be NULL) receives || f_moe(X; k_base) ||_F.
+ * Synchronises the stream.  Errors: INVALID_ARG, ALIGN, CUDA.
+ */
+int moe_profile_layer(moe_plan_t *plan, const void *x, const moe_layer_weights_t *w, int32_t T,
+                      int32_t k_base, int32_t renorm, double *delta, double *base_norm, void *cuda_stream);
+
+/*
  * moe_route_from_logits (test hook): TopK + Softmax + dispatch tables from logits the
  * caller supplies, so that routing can be compared bit for bit (Section 2's TopK[.] and
  * Softmax).  logits [T, E] fp32 device.  Outputs, device, any may be NULL:

@@ -28,6 +28,7 @@ EXPORTS = (
     "moe_route_from_logits", "moe_last_routing", "moe_device_status", "moe_plan_launch_count",
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
     "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts",
+    "moe_profile_layer",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
 
@@ -80,6 +81,8 @@ def load_library() -> ctypes.CDLL:
     lib.moe_device_status.argtypes = [vp, vp]
     lib.moe_last_residual_f32.argtypes = [vp, vp, i32, vp]
     lib.moe_plan_touched_experts.argtypes = [vp, P(ctypes.c_int64), vp]
+    lib.moe_profile_layer.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, P(ctypes.c_double),
+                                      P(ctypes.c_double), vp]
     lib.moe_dispatch_tables_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     lib.moe_plan_set_stage_timing.argtypes = [vp, i32]
     lib.moe_plan_stage_times.argtypes = [vp, P(ctypes.c_float), P(i32)]
@@ -193,6 +196,19 @@ def moe_stack_forward(plan: int, h: torch.Tensor, layers: Sequence[moe_layer_wei
                                             h.shape[0], _stream(stream)))
 
 
+def moe_profile_layer(plan: int, x: torch.Tensor, w: moe_layer_weights_t, k_base: int, renorm: bool,
+                      stream=None):
+    """One sample of Algorithm 1 for every k: (list of ||f(X;k) - f(X;k_base)||_F for k = 1..k_base,
+    ||f(X;k_base)||_F)."""
+    assert x.is_cuda and x.is_contiguous()
+    delta = (ctypes.c_double * k_base)()
+    base = ctypes.c_double()
+    _check("moe_profile_layer",
+           load_library().moe_profile_layer(plan, x.data_ptr(), ctypes.byref(w), x.shape[0], k_base,
+                                            int(renorm), delta, ctypes.byref(base), _stream(stream)))
+    return [float(v) for v in delta], float(base.value)
+
+
 def moe_route_from_logits(plan: int, logits: torch.Tensor, k_l: int, renorm: bool, stream=None):
     """Returns (topk_idx [T,k], topk_w [T,k], counts [E], offsets [E+1], perm [T*k]) on the device."""
     assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
@@ -245,6 +261,7 @@ def moe_plan_touched_experts(plan: int, stream=None) -> int:
     """Sum over the tensor-core layer calls since the last read of the experts that got tokens."""
     n = ctypes.c_int64()
     _check("moe_plan_touched_experts",
+    "moe_profile_layer",
            load_library().moe_plan_touched_experts(plan, ctypes.byref(n), _stream(stream)))
     return int(n.value)
 
@@ -314,6 +331,9 @@ class MoEPlan:
     def stack_forward(self, h, layers, k_vec, renorm, stream=None):
         moe_stack_forward(self.handle, h, layers, k_vec, renorm, stream)
         return h
+
+    def profile_layer(self, x, w, k_base, renorm, stream=None):
+        return moe_profile_layer(self.handle, x, w, k_base, renorm, stream)
 
     def route_from_logits(self, logits, k_l, renorm, stream=None):
         return moe_route_from_logits(self.handle, logits, k_l, renorm, stream)

@@ -138,6 +138,124 @@ cudaError_t launch_combine(const CombineArgs &a, cudaStream_t s, uint64_t *launc
     return e;
 }
 
+// ---------------------------------------------------------------------------------------
+// Stage-1 profiling (paper, Algorithm 1): Delta_k = || f_moe(X; k) - f_moe(X; k_base) ||_F for every
+// k <= k_base from ONE pass of the experts at k_base.  The top-k sets are nested in k (slot j holds
+// the j-th largest logit), so with the slot outputs o_j of the k_base pass
+//     Y_k = s_r * sum_{j<k} g_j^(k) o_j + shared,   g_j^(k) = p_j            (no renormalisation)
+//                                                   g_j^(k) = p_j / sum_{i<k} p_i   (renormalised)
+// and the shared term cancels in the difference.  p_j are full-softmax entries (the router runs
+// without renormalisation for this call).  Each block reduces its squared differences per k and
+// writes them to partial[block][k]; a second kernel adds the blocks in a fixed order in double.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float block_sum_256(float v, float *scratch) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < 8; ++w) t += scratch[w];
+    return t;      // valid in thread 0
+}
+
+template <typename OT>
+__global__ void __launch_bounds__(256) profile_kernel(CombineArgs a, int renorm, float *partial) {
+    __shared__ float scratch[8];
+    pdl_trigger();
+    pdl_wait();
+    const int vec_per_row = a.d / 4;
+    const size_t n_vec = (size_t)a.T * vec_per_row;
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    const bool on = i < n_vec;
+    const int t = on ? (int)(i / vec_per_row) : 0;
+    const int c = on ? (int)(i % vec_per_row) * 4 : 0;
+    const OT *o = (const OT *)a.o;
+    auto slot_out = [&](int j) {
+        const int r = a.inv_perm[(size_t)t * a.k + j];
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sl = 0; sl < a.o_slabs; ++sl) {
+            const float4 w = ld4(o + (size_t)sl * a.o_slab_stride + (size_t)r * a.d + c);
+            v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+        }
+        return v;
+    };
+    // f(X; k_base): numerator and gate mass over all k_base slots
+    float4 S = make_float4(0.f, 0.f, 0.f, 0.f);
+    float P = 0.f;
+    for (int j = 0; j < a.k; ++j) {
+        const float pj = a.topk_w[(size_t)t * a.k + j];
+        const float4 v = slot_out(j);
+        S.x = fmaf(pj, v.x, S.x); S.y = fmaf(pj, v.y, S.y); S.z = fmaf(pj, v.z, S.z); S.w = fmaf(pj, v.w, S.w);
+        P += pj;
+    }
+    const float sb = a.routed_scale / (renorm ? P : 1.0f);
+    // explicit roundings (no fused multiply-subtract below), so that the k = k_base prefix, which
+    // repeats these operations term by term, differs from Yb by exactly zero
+    const float4 Yb = make_float4(__fmul_rn(S.x, sb), __fmul_rn(S.y, sb), __fmul_rn(S.z, sb), __fmul_rn(S.w, sb));
+    // norm of the base output, shared expert included
+    float4 full = Yb;
+    if (a.o_s) {
+        const float gm = a.gamma ? a.gamma[t] : 1.0f;
+        const OT *os = (const OT *)a.o_s + (size_t)t * a.d + c;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sl = 0; sl < a.os_slabs; ++sl) {
+            const float4 w = ld4(os + (size_t)sl * a.os_slab_stride);
+            v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+        }
+        full.x = fmaf(gm, v.x, full.x); full.y = fmaf(gm, v.y, full.y);
+        full.z = fmaf(gm, v.z, full.z); full.w = fmaf(gm, v.w, full.w);
+    }
+    float sq = on ? full.x * full.x + full.y * full.y + full.z * full.z + full.w * full.w : 0.f;
+    float tot = block_sum_256(sq, scratch);
+    if (threadIdx.x == 0) partial[(size_t)blockIdx.x * (a.k + 1) + a.k] = tot;
+    // prefixes: k = 1 .. k_base (the last one reproduces the base sum term by term: difference 0)
+    S = make_float4(0.f, 0.f, 0.f, 0.f);
+    P = 0.f;
+    for (int kk = 1; kk <= a.k; ++kk) {
+        const float pj = a.topk_w[(size_t)t * a.k + kk - 1];
+        const float4 v = slot_out(kk - 1);
+        S.x = fmaf(pj, v.x, S.x); S.y = fmaf(pj, v.y, S.y); S.z = fmaf(pj, v.z, S.z); S.w = fmaf(pj, v.w, S.w);
+        P += pj;
+        const float sk = a.routed_scale / (renorm ? P : 1.0f);
+        const float dx = __fmul_rn(S.x, sk) - Yb.x, dy = __fmul_rn(S.y, sk) - Yb.y;
+        const float dz = __fmul_rn(S.z, sk) - Yb.z, dw = __fmul_rn(S.w, sk) - Yb.w;
+        sq = on ? dx * dx + dy * dy + dz * dz + dw * dw : 0.f;
+        tot = block_sum_256(sq, scratch);
+        if (threadIdx.x == 0) partial[(size_t)blockIdx.x * (a.k + 1) + kk - 1] = tot;
+    }
+}
+
+// out[b] = sum over blocks of partial[block][b], fixed order, double.
+__global__ void __launch_bounds__(256) profile_reduce_kernel(const float *partial, int n_blocks, int width,
+                                                             double *out) {
+    __shared__ double sh[256];
+    const int b = blockIdx.x;
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < n_blocks; i += 256) acc += (double)partial[(size_t)i * width + b];
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) out[b] = sh[0];
+}
+
+cudaError_t launch_profile(const CombineArgs &a, int renorm, float *partial, double *sums, cudaStream_t s,
+                           uint64_t *launches) {
+    if (a.T <= 0) return cudaSuccess;
+    const size_t n_vec = (size_t)a.T * (a.d / 4);
+    const int grid = (int)((n_vec + 255) / 256);
+    if (a.o_is_f32) profile_kernel<float><<<grid, 256, 0, s>>>(a, renorm, partial);
+    else profile_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(a, renorm, partial);
+    profile_reduce_kernel<<<a.k + 1, 256, 0, s>>>(partial, grid, a.k + 1, sums);
+    *launches += 2;
+    return cudaGetLastError();
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) widen_kernel(const T *src, float *dst, size_t n) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;

@@ -55,6 +55,8 @@ struct Workspace {
     Tile    *tiles2 = nullptr;     // phase-2 tile list
     int32_t *n_tiles = nullptr;    // [2] tile counts
     int32_t *ticket = nullptr;     // block-arrival counter of the fused small-T front end
+    float   *prof_partial = nullptr;  // Stage-1 profiling: per-block partial sums
+    double  *prof_sums = nullptr;     // [max_k + 1]
     int32_t *stats = nullptr;      // [4] counters read by moe_plan_touched_experts
     int32_t *pos = nullptr;        // [E, 128] direct mode: output row of (expert, token) or -1
 };
@@ -136,6 +138,11 @@ struct CombineArgs {
     bool chained;
 };
 cudaError_t launch_combine(const CombineArgs &a, cudaStream_t s, uint64_t *launches);
+
+// Stage-1 profiling: sums[k-1] = sum of squares of f(X;k) - f(X;k_base) for k = 1..a.k, sums[a.k] =
+// sum of squares of f(X;k_base); partial holds ceil(T*d/1024) * (a.k+1) floats.
+cudaError_t launch_profile(const CombineArgs &a, int renorm, float *partial, double *sums, cudaStream_t s,
+                           uint64_t *launches);
 
 cudaError_t launch_widen(const void *src, float *dst, size_t n, int dtype, cudaStream_t s,
                          uint64_t *launches);

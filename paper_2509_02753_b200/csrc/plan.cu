@@ -1,5 +1,6 @@
 // C ABI of the library (include/moe.h): plan, workspace, and the host-side sequencing of the
 // kernels of one MoE layer and of a stack of layers with a per-layer k vector.
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -71,6 +72,7 @@ int pick_schedule(const moe_plan *p, int T, int k) {
     return ((int64_t)T * k < (int64_t)16 * p->cfg.E) ? MOE_SCHED_DECODE : MOE_SCHED_PREFILL;
 }
 
+// mode 3: Stage-1 profiling (no y; sums of squared differences go to ws.prof_sums).
 // mode 0: y = MoE(x).  mode 1: h_run += MoE(x), y = round(h_run) (y may be x).  mode 2: y += MoE(x), y == x.
 int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, int k, int renorm,
                void *y, int mode, cudaStream_t s) {
@@ -84,7 +86,7 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
     mark(0);
 
     RouterArgs ra{x, w->router_W, w->router_bias, (c.I_shared > 0 && c.shared_gate) ? w->w_s : nullptr,
-                  T, c.d, c.E, k, renorm, c.dtype, ws.logits, ws.topk_idx, ws.topk_w, ws.gamma,
+                  T, c.d, c.E, k, mode == 3 ? 0 : renorm, c.dtype, ws.logits, ws.topk_idx, ws.topk_w, ws.gamma,
                   ws.status, false};
     // kernels of a small decode call are chained as programmatic dependents (not while stage
     // events are being recorded between them)
@@ -143,7 +145,11 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
         ca.os_slabs = lay.os_slabs; ca.os_slab_stride = lay.os_slab_stride;
     }
     mark(4);
-    if ((err = launch_combine(ca, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
+    if (mode == 3)
+        err = launch_profile(ca, renorm, ws.prof_partial, ws.prof_sums, s, &p->launches);
+    else
+        err = launch_combine(ca, s, &p->launches);
+    if (err != cudaSuccess) return MOE_ERR_CUDA;
     mark(5);
     p->last_T = T;
     p->last_k = k;
@@ -237,6 +243,8 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
     ok = ok && ws_alloc(p, &ws.ticket, (size_t)4 + kFrontMaxTokens);
     ok = ok && ws_alloc(p, &ws.pos, (size_t)c.E * kFrontMaxTokens);
     ok = ok && ws_alloc(p, &ws.stats, (size_t)4);
+    ok = ok && ws_alloc(p, &ws.prof_partial, (((size_t)c.max_T * c.d / 4 + 255) / 256) * (c.max_k + 1));
+    ok = ok && ws_alloc(p, &ws.prof_sums, (size_t)c.max_k + 1);
     if (ok && cudaMallocHost(&p->status_host, sizeof(int32_t)) != cudaSuccess) { cudaGetLastError(); ok = false; }
     if (ok) {
         ok = cudaMemset(ws.status, 0, 16) == cudaSuccess && cudaMemset(ws.ticket, 0, sizeof(int32_t) * (4 + kFrontMaxTokens)) == cudaSuccess &&
@@ -342,6 +350,27 @@ int moe_layer_forward_host(moe_plan_t *p, const void *x_host, const moe_layer_we
         cudaGetLastError();
         return MOE_ERR_CUDA;
     }
+    return MOE_OK;
+}
+
+int moe_profile_layer(moe_plan_t *p, const void *x, const moe_layer_weights_t *w, int32_t T, int32_t k_base,
+                      int32_t renorm, double *delta, double *base_norm, void *cuda_stream) {
+    if (!p || !x || !delta) return MOE_ERR_INVALID_ARG;
+    if (T < 1 || T > p->cfg.max_T || k_base < 1 || k_base > p->cfg.max_k) return MOE_ERR_INVALID_ARG;
+    if (!aligned16(x)) return MOE_ERR_ALIGN;
+    int rc = check_weights(p, w);
+    if (rc != MOE_OK) return rc;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    rc = layer_impl(p, x, w, T, k_base, renorm ? 1 : 0, nullptr, 3, s);
+    if (rc != MOE_OK) return rc;
+    double sums[kMaxExperts + 1];
+    if (cudaMemcpyAsync(sums, p->ws.prof_sums, sizeof(double) * (k_base + 1), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    for (int k = 0; k < k_base; ++k) delta[k] = sqrt(sums[k]);
+    if (base_norm) *base_norm = sqrt(sums[k_base]);
     return MOE_OK;
 }
 

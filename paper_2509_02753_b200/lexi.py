@@ -1,0 +1,42 @@
+"""Stage 1 of LExI on the CUDA path: the per-layer top-k perturbation profile (paper, Algorithm 1).
+
+Thin driver: draws the Monte-Carlo samples X ~ N(0,1)^{B x L x H} with torch's generator on the
+device (or takes them from the caller), hands each to ``moe_profile_layer`` and averages.  All
+arithmetic on X runs in the library's kernels.
+"""
+from __future__ import annotations
+
+from typing import Dict, Iterable, Optional
+
+import torch
+
+from . import binding as B
+
+
+def perturbation_profile(plan: B.MoEPlan, weights: B.moe_layer_weights_t, k_base: int, renorm: bool, *,
+                         batch: int = 16, seq_len: int = 128, n_iter: int = 8, seed: int = 0,
+                         samples: Optional[Iterable[torch.Tensor]] = None) -> Dict[int, float]:
+    """Average over the samples of ||f_moe(X; k) - f_moe(X; k_base)||_F for k = 1..k_base.
+
+    ``samples``: optional iterable of [T, H] CUDA tensors (T <= the plan's max_T); otherwise n_iter
+    samples of batch * seq_len tokens are drawn from N(0,1) with the given seed.
+    Returns {k: mean Delta_k}; by construction the entry for k_base is exactly 0.
+    """
+    if samples is None:
+        g = torch.Generator(device="cuda")
+        g.manual_seed(seed)
+
+        def draw():
+            for _ in range(n_iter):
+                x = torch.empty((batch * seq_len, plan.d), dtype=torch.float32, device="cuda")
+                x.normal_(0.0, 1.0, generator=g)
+                yield x.to(plan.dtype)
+        samples = draw()
+    total = [0.0] * k_base
+    n = 0
+    for x in samples:
+        delta, _ = plan.profile_layer(x, weights, k_base, renorm)
+        total = [a + b for a, b in zip(total, delta)]
+        n += 1
+    assert n > 0, "no samples"
+    return {k + 1: total[k] / n for k in range(k_base)}

@@ -1,0 +1,69 @@
+"""Stage 1 (Algorithm 1) on the GPU against the oracle's literal Algorithm 1: the oracle runs the
+layer once per k and takes the Frobenius norm of the difference; the library runs the experts once
+at k_base and forms every f(X; k) from prefix sums.
+
+Tolerance: both outputs of a difference carry the bf16 path's error (h is rounded to bf16, about
+3e-3 of ||Y||_F in Frobenius norm), so |Delta_gpu - Delta_ref| <= 1e-2 ||Y_base||_F for bf16 and
+1e-4 ||Y_base||_F for fp32; Delta(k_base) must be exactly 0."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as orc
+from paper_2509_02753_b200 import binding as B
+from paper_2509_02753_b200 import lexi, synth
+
+from parity import oracle_weights
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(wl, T, dtype, k_base, renorm, sched=None):
+    w_host = synth.make_layer(wl, 0, dtype, "cpu")
+    w_dev = {k: (None if v is None else v.cuda()) for k, v in w_host.items()}
+    x = synth.make_tokens(wl, T, dtype, "cpu")
+    ref = orc.perturbation_profile(x, oracle_weights(w_host), k_base, list(range(1, k_base + 1)), renorm,
+                                   shared_gate=wl.shared_gate)
+    base = orc.moe_layer(x, oracle_weights(w_host), k_base, renorm, shared_gate=wl.shared_gate).y
+    base_norm = float(np.sqrt((base ** 2).sum()))
+    with B.MoEPlan(wl.d, wl.E, wl.I, T, k_base, dtype, I_shared=wl.I_shared, shared_gate=wl.shared_gate) as plan:
+        if sched is not None:
+            plan.set_schedule(sched)
+        delta, bn = plan.profile_layer(x.cuda(), B.make_weights(w_dev), k_base, renorm)
+        assert plan.device_status() == 0
+    tol = (1e-2 if dtype == torch.bfloat16 else 1e-4) * base_norm
+    assert delta[k_base - 1] == 0.0 and ref[k_base] == 0.0
+    for k in range(1, k_base):
+        assert abs(delta[k - 1] - ref[k]) <= tol, (k, delta[k - 1], ref[k], tol)
+        assert delta[k - 1] > 0
+    assert abs(bn - base_norm) <= tol
+    return delta, ref
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("renorm", [True, False])
+def test_profile_tiny_layer(dtype, renorm):
+    _case(synth.WORKLOADS["tiny"], 64, dtype, 2, renorm)
+
+
+@pytest.mark.parametrize("T,sched", [(24, None), (300, B.MOE_SCHED_PREFILL), (300, B.MOE_SCHED_DECODE),
+                                     (300, B.MOE_SCHED_SIMT)])
+@pytest.mark.parametrize("renorm", [True, False])
+def test_profile_with_shared_expert_and_six_slots(T, sched, renorm):
+    wl = synth.Workload("prof", d=256, E=16, I=256, k_base=6, L=1, I_shared=256, shared_gate=True,
+                        router_bias_std=0.3)
+    _case(wl, T, torch.bfloat16, 6, renorm, sched)
+
+
+def test_stage1_driver_averages_samples():
+    wl = synth.WORKLOADS["tiny"]
+    w_host = synth.make_layer(wl, 0, torch.bfloat16, "cpu")
+    w_dev = {k: (None if v is None else v.cuda()) for k, v in w_host.items()}
+    xs = [synth.make_tokens(wl, 48, torch.bfloat16, "cpu", seed=s) for s in (1, 2, 3)]
+    refs = [orc.perturbation_profile(x, oracle_weights(w_host), 2, [1, 2], True) for x in xs]
+    with B.MoEPlan(wl.d, wl.E, wl.I, 2048, 2, torch.bfloat16) as plan:
+        got = lexi.perturbation_profile(plan, B.make_weights(w_dev), 2, True, samples=[x.cuda() for x in xs])
+        drawn = lexi.perturbation_profile(plan, B.make_weights(w_dev), 2, True, batch=4, seq_len=64, n_iter=3)
+    mean1 = float(np.mean([r[1] for r in refs]))
+    assert got[2] == 0.0 and abs(got[1] - mean1) <= 2e-2 * mean1
+    assert drawn[2] == 0.0 and drawn[1] > 0
