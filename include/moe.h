@@ -176,6 +176,27 @@ int moe_profile_layer(moe_plan_t *plan, const void *x, const moe_layer_weights_t
                       int32_t k_base, int32_t renorm, double *delta, double *base_norm, void *cuda_stream);
 
 /*
+ * Stage 2 of LExI (Algorithm 2, "Evolutionary Top-k Allocation Optimization with Proxy"): pick
+ * k = (k_1..k_L), sum_j k_j = budget, k_min <= k_j <= k_max, minimising phi(k) = sum_j D_j(k_j).
+ * Host functions, no GPU work.  D: HOST table [L, k_max], D[j * k_max + (k-1)] = D_j(k) from Stage 1.
+ * k_out: HOST [L].  phi_out (may be NULL): the loss of the returned allocation.
+ *
+ * moe_lexi_allocate_exact: the constrained minimum itself (phi is separable: dynamic programme over
+ * layer and budget).  moe_lexi_allocate_evolutionary: the search of Algorithm 2 - population of n_pop
+ * feasible members, g_max generations of tournament selection (size `tournament`), uniform
+ * crossover, zero-sum +-1 mutation with probability eta_mut, projection back to the constraints,
+ * the child joins the population; returns the best member.  Its random numbers are read, in program
+ * order, from the caller's stream rnd[0..n_rnd) of uniform uint32 (about 2 * tournament + L + 4 per
+ * generation plus budget per initial member); a stream that runs out is an error.
+ * Errors: INVALID_ARG (also for an infeasible budget).
+ */
+int moe_lexi_allocate_exact(const double *D, int32_t L, int32_t k_max, int32_t k_min, int32_t budget,
+                            int32_t *k_out, double *phi_out);
+int moe_lexi_allocate_evolutionary(const double *D, int32_t L, int32_t k_max, int32_t k_min, int32_t budget,
+                                   int32_t n_pop, int32_t g_max, double eta_mut, int32_t tournament,
+                                   const uint32_t *rnd, int64_t n_rnd, int32_t *k_out, double *phi_out);
+
+/*
  * moe_route_from_logits (test hook): TopK + Softmax + dispatch tables from logits the
  * caller supplies, so that routing can be compared bit for bit (Section 2's TopK[.] and
  * Softmax).  logits [T, E] fp32 device.  Outputs, device, any may be NULL:

@@ -28,7 +28,7 @@ EXPORTS = (
     "moe_route_from_logits", "moe_last_routing", "moe_device_status", "moe_plan_launch_count",
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
     "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts",
-    "moe_profile_layer",
+    "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
 
@@ -83,6 +83,10 @@ def load_library() -> ctypes.CDLL:
     lib.moe_plan_touched_experts.argtypes = [vp, P(ctypes.c_int64), vp]
     lib.moe_profile_layer.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, P(ctypes.c_double),
                                       P(ctypes.c_double), vp]
+    dbl_p, i32_p = P(ctypes.c_double), P(i32)
+    lib.moe_lexi_allocate_exact.argtypes = [dbl_p, i32, i32, i32, i32, i32_p, dbl_p]
+    lib.moe_lexi_allocate_evolutionary.argtypes = [dbl_p, i32, i32, i32, i32, i32, i32, ctypes.c_double, i32,
+                                                   P(ctypes.c_uint32), ctypes.c_int64, i32_p, dbl_p]
     lib.moe_dispatch_tables_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     lib.moe_plan_set_stage_timing.argtypes = [vp, i32]
     lib.moe_plan_stage_times.argtypes = [vp, P(ctypes.c_float), P(i32)]
@@ -209,6 +213,40 @@ def moe_profile_layer(plan: int, x: torch.Tensor, w: moe_layer_weights_t, k_base
     return [float(v) for v in delta], float(base.value)
 
 
+def _stage2_table(D):
+    import numpy as np
+    D = np.ascontiguousarray(np.asarray(D, dtype=np.float64))
+    assert D.ndim == 2
+    return D, D.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def moe_lexi_allocate_exact(D, k_min: int, budget: int):
+    """Stage 2, exact optimum.  D [L, k_max] with D[j, k-1] = D_j(k).  Returns (k list, phi)."""
+    D, dp = _stage2_table(D)
+    L, k_max = D.shape
+    k = (ctypes.c_int32 * L)()
+    phi = ctypes.c_double()
+    _check("moe_lexi_allocate_exact",
+           load_library().moe_lexi_allocate_exact(dp, L, k_max, k_min, budget, k, ctypes.byref(phi)))
+    return list(k), float(phi.value)
+
+
+def moe_lexi_allocate_evolutionary(D, k_min: int, budget: int, rnd, *, n_pop: int = 32, g_max: int = 2000,
+                                   eta_mut: float = 0.3, tournament: int = 3):
+    """Stage 2, Algorithm 2's evolutionary search.  rnd: uint32 array, the random stream it consumes."""
+    import numpy as np
+    D, dp = _stage2_table(D)
+    L, k_max = D.shape
+    rnd = np.ascontiguousarray(np.asarray(rnd, dtype=np.uint32))
+    k = (ctypes.c_int32 * L)()
+    phi = ctypes.c_double()
+    _check("moe_lexi_allocate_evolutionary",
+           load_library().moe_lexi_allocate_evolutionary(
+               dp, L, k_max, k_min, budget, n_pop, g_max, eta_mut, tournament,
+               rnd.ctypes.data_as(ctypes.POINTER(ctypes.c_uint32)), rnd.size, k, ctypes.byref(phi)))
+    return list(k), float(phi.value)
+
+
 def moe_route_from_logits(plan: int, logits: torch.Tensor, k_l: int, renorm: bool, stream=None):
     """Returns (topk_idx [T,k], topk_w [T,k], counts [E], offsets [E+1], perm [T*k]) on the device."""
     assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
@@ -261,7 +299,7 @@ def moe_plan_touched_experts(plan: int, stream=None) -> int:
     """Sum over the tensor-core layer calls since the last read of the experts that got tokens."""
     n = ctypes.c_int64()
     _check("moe_plan_touched_experts",
-    "moe_profile_layer",
+    "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
            load_library().moe_plan_touched_experts(plan, ctypes.byref(n), _stream(stream)))
     return int(n.value)
 
