@@ -289,6 +289,211 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
     }
 }
 
+// ------------------------------------------------------------------ CTA-pair variant (prefill)
+// Tile = 256 token rows x 256 weight rows, worked on by the two CTAs of a cluster of 2 with
+// tcgen05.mma.cta_group::2: CTA r holds rows 128r..128r+127 of the tile (A and D) and half of B
+// (phase 1: CTA 0 the 128 gate rows, CTA 1 the 128 up rows; phase 2: 128 rows of W_down each), so a
+// stage costs 32 KB of loads per CTA instead of 48 KB.  CTA 0 issues all MMAs once both CTAs' loads
+// have landed (both count their bytes on CTA 0's "full" mbarrier); tcgen05.commit multicasts the
+// "stage free" and "accumulator ready" arrivals to both CTAs; both epilogues release the accumulator
+// on CTA 0's "empty" mbarrier.  No multicast loads.  Waits are bounded as in the 1-CTA kernel.
+constexpr int kPairStages = 6;
+constexpr int kPairABytes = 128 * 128, kPairBBytes = 128 * 128;
+
+template <int PHASE>
+constexpr int pair_smem_bytes() {
+    return kPairStages * (kPairABytes + kPairBBytes) + 1024 + 256 + (PHASE == 2 ? kStageBytes : 0);
+}
+
+template <int PHASE, typename OutT>
+__global__ void __launch_bounds__(192, 1)
+ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_constant__ CUtensorMap mapA_shared,
+                   const __grid_constant__ CUtensorMap mapB0_routed, const __grid_constant__ CUtensorMap mapB1_routed,
+                   const __grid_constant__ CUtensorMap mapB0_shared, const __grid_constant__ CUtensorMap mapB1_shared,
+                   const TcParams p) {
+    constexpr int BN = 256, STAGES = kPairStages, A_BYTES = kPairABytes, B_BYTES = kPairBBytes;
+    constexpr int TMEM_COLS = 2 * BN;
+    pdl_trigger();
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const uint32_t a_base = base;
+    const uint32_t b_base = base + STAGES * A_BYTES;
+    const uint32_t bar_base = b_base + STAGES * B_BYTES;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+    const uint32_t slot_addr = bar_base + 8u * (2 * STAGES + 4);
+    volatile uint32_t *slot_ptr = reinterpret_cast<volatile uint32_t *>(smem_raw + (slot_addr - raw));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();          // 0: issues the MMAs
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 256); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(slot_addr, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();          // the peer's barriers exist before anything is sent to them
+    tc_fence_after();
+    const uint32_t tmem_base = *slot_ptr;
+    pdl_wait();
+    const int n_tiles = *p.n_tiles;
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (one lane, both CTAs)
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            Tile t_next = pair_id < n_tiles ? p.tiles[pair_id] : Tile{};
+            for (int tile = pair_id; ok && tile < n_tiles; tile += n_pairs) {
+                const Tile t = t_next;
+                if (tile + n_pairs < n_tiles) t_next = p.tiles[tile + n_pairs];
+                const bool shared = t.group == p.E;
+                const CUtensorMap *mA = shared ? &mapA_shared : &mapA_routed;
+                // this CTA's half of B: phase 1 -> gate rows (CTA 0) or up rows (CTA 1) of the same
+                // features; phase 2 -> rows n0 + 128 rank of W_down
+                const CUtensorMap *mB = PHASE == 1 ? (rank == 0 ? (shared ? &mapB0_shared : &mapB0_routed)
+                                                                : (shared ? &mapB1_shared : &mapB1_routed))
+                                                   : (shared ? &mapB0_shared : &mapB0_routed);
+                const int b_row = PHASE == 1 ? t.n0 : t.n0 + 128 * (int)rank;
+                const int grp = shared ? 0 : t.group;
+                const int a_row = t.row0 + 128 * (int)rank;
+                const int nk = (t.klen + kBK - 1) / kBK;
+                for (int kc = 0; kc < nk; ++kc, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, p.status)) { ok = false; break; }
+                    const uint32_t full0 = full_bar(s) & kPeerBitMask;      // CTA 0 counts both CTAs' bytes
+                    if (rank == 0) mbar_expect_tx(full_bar(s), 2 * (A_BYTES + B_BYTES));
+                    const int k = t.k0 + kc * kBK;
+                    tma_load_3d_pair(a_base + s * A_BYTES, mA, full0, k, a_row, 0);
+                    tma_load_3d_pair(b_base + s * B_BYTES, mB, full0, k, b_row, grp);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (CTA 0 only)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16_m(256, BN);
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            int klen_next = pair_id < n_tiles ? p.tiles[pair_id].klen : 0;
+            for (int tile = pair_id; ok && tile < n_tiles; tile += n_pairs, ++tcount) {
+                const int nk = (klen_next + kBK - 1) / kBK;
+                if (tile + n_pairs < n_tiles) klen_next = p.tiles[tile + n_pairs].klen;
+                const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(buf), bph ^ 1u, p.status)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kc = 0; kc < nk; ++kc, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t a_desc = make_kmajor_sw128_desc(a_base + s * A_BYTES);
+                    const uint64_t b_desc = make_kmajor_sw128_desc(b_base + s * B_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < kBK / 16; ++kk)
+                        umma_bf16_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kc | kk) != 0);
+                    umma_commit_pair(empty_bar(s));
+                }
+                if (ok) umma_commit_pair(tfull_bar(buf));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+        const int q = warp & 3;
+        const int row_in_cta = q * 32 + lane;                    // row of this CTA's 128
+        const int row_in_tile = 128 * (int)rank + row_in_cta;    // row of the 256-row tile
+        uint32_t tcount = 0;
+        Tile t_next = pair_id < n_tiles ? p.tiles[pair_id] : Tile{};
+        for (int tile = pair_id; tile < n_tiles; tile += n_pairs, ++tcount) {
+            const Tile t = t_next;
+            if (tile + n_pairs < n_tiles) t_next = p.tiles[tile + n_pairs];
+            const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
+            const bool shared = t.group == p.E;
+            const int N = shared ? p.N_shared : p.N_routed;
+            const bool row_ok = row_in_tile < t.rows;
+            const bool got = mbar_wait(tfull_bar(buf), bph, p.status);
+            if (!__all_sync(0xffffffffu, got)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
+            OutT *obase = reinterpret_cast<OutT *>(shared ? p.out_shared : p.out_routed) +
+                          (size_t)t.slot * (shared ? p.slab_stride_shared : p.slab_stride_routed);
+            if (PHASE == 1) {
+                OutT *out = obase + (size_t)(t.row0 + row_in_tile) * N + t.n0;
+#pragma unroll 1
+                for (int c = 0; c < BN / 2; c += 16) {
+                    uint32_t g[16], u[16];
+                    tmem_ld16(taddr + c, g);
+                    tmem_ld16(taddr + BN / 2 + c, u);
+                    tmem_ld_wait();
+                    uint32_t packed[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        packed[i] = pack_bf16(silu_mul(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
+                                              silu_mul(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1])));
+                    if (row_ok) {
+                        if (t.n0 + c + 8 <= N)
+                            *reinterpret_cast<uint4 *>(out + c) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                        if (t.n0 + c + 16 <= N)
+                            *reinterpret_cast<uint4 *>(out + c + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                    }
+                }
+            } else {
+                float *stg = reinterpret_cast<float *>(smem_raw + (bar_base + 256u - raw)) + q * 32 * kStagePitch;
+                OutT *wbase = obase + (size_t)(t.row0 + 128 * (int)rank + q * 32) * N + t.n0;
+                const int rows_here = t.rows - 128 * (int)rank - q * 32;
+                const int rr0 = lane >> 3, cc = 4 * (lane & 7);
+#pragma unroll 1
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t v0[16], v1[16];
+                    tmem_ld16(taddr + c, v0);
+                    tmem_ld16(taddr + c + 16, v1);
+                    tmem_ld_wait();
+                    uint4 *wr = reinterpret_cast<uint4 *>(stg + lane * kStagePitch);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        wr[i] = make_uint4(v0[4 * i], v0[4 * i + 1], v0[4 * i + 2], v0[4 * i + 3]);
+                        wr[4 + i] = make_uint4(v1[4 * i], v1[4 * i + 1], v1[4 * i + 2], v1[4 * i + 3]);
+                    }
+                    __syncwarp();
+                    const bool col_ok = t.n0 + c + cc + 4 <= N;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int rr = 4 * j + rr0;
+                        const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * kStagePitch + cc);
+                        if (rr < rows_here && col_ok)
+                            *reinterpret_cast<uint4 *>(wbase + (size_t)rr * N + c + cc) = val;
+                    }
+                    __syncwarp();
+                }
+            }
+            tc_fence_before();
+            mbar_arrive_cta0(tempty_bar(buf));       // both CTAs' epilogues free the buffer on CTA 0
+        }
+    }
+
+    // ---------------------------------------------------------------- common exit
+    __syncwarp();
+    if (*reinterpret_cast<volatile int32_t *>(p.status) & kStatusTimeout) {
+        for (int i = 0; i < 256; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();          // neither CTA leaves while the other may still reach into it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
 // ------------------------------------------------------------------ tile lists
 __global__ void __launch_bounds__(1024) build_tiles_kernel(TileBuildArgs a) {
     pdl_trigger();
@@ -354,6 +559,36 @@ cudaError_t launch_tc(const CUtensorMap *maps, const TcParams &p, int grid, cuda
                           maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], p);
 }
 
+template <int PHASE, typename OutT>
+cudaError_t launch_tc_pair(const CUtensorMap *maps, const TcParams &p, int max_pairs, cudaStream_t s, bool chained) {
+    auto kern = ffn_tc_pair_kernel<PHASE, OutT>;
+    constexpr int smem = pair_smem_bytes<PHASE>();
+    static int max_clusters = -1;
+    cudaLaunchConfig_t cfg{};
+    cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    if (max_clusters < 0) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        cfg.gridDim = dim3(2 * 74);
+        cfg.numAttrs = 1;
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+        if (e != cudaSuccess) return e;
+        if (n < 1) return cudaErrorInvalidConfiguration;
+        max_clusters = n;
+    }
+    const int clusters = max_pairs < max_clusters ? (max_pairs < 1 ? 1 : max_pairs) : max_clusters;
+    cfg.gridDim = dim3(2 * clusters);
+    cfg.numAttrs = chained ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, kern, maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], p);
+}
+
 }  // namespace
 
 bool tc_encode_bf16_map(const TcState *st, void *map, const void *ptr, uint64_t K, uint64_t rows,
@@ -416,6 +651,9 @@ void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs 
     TcSchedule &sc = *out;
     sc.decode = decode;
     sc.direct = direct;
+    // LEXI_PREFILL_2CTA=1: the prefill GEMMs run on CTA pairs (256-row tiles, cta_group::2)
+    static const bool pair_env = getenv("LEXI_PREFILL_2CTA") != nullptr;
+    sc.pair = !decode && !direct && pair_env;
     const int dec_bn = decode_bn_override() ? decode_bn_override() : 128;
     sc.bn1 = decode ? dec_bn : 256;       // phase-1 tile: bn1/2 gate rows + bn1/2 up rows
     sc.bn2 = decode ? dec_bn : 256;
@@ -442,6 +680,7 @@ void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs 
     tb.cap1 = (int)tc_max_tiles(c, 1); tb.cap2 = (int)tc_max_tiles(c, 2);
     tb.status = ws.status;
     tb.direct = direct ? 1 : 0;
+    tb.tile_rows = sc.pair ? 2 * kTileRows : kTileRows;
     tb.stats = ws.stats;
 }
 
@@ -469,9 +708,10 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
     ok = ok && encode_map(st, &m2[0], a.h, a.I, pairs_alloc + 128, 1, a_rows);
     ok = ok && encode_map(st, &m2[1], has_shared ? a.h_s : a.h, has_shared ? a.I_s : a.I,
                           has_shared ? (size_t)c.max_T + 128 : pairs_alloc + 128, 1, a_rows);
-    ok = ok && encode_map(st, &m2[2], a.W_down, a.I, a.d, a.E, bn2);
+    ok = ok && encode_map(st, &m2[2], a.W_down, a.I, a.d, a.E, sc.pair ? 128 : bn2);
     m2[3] = m2[2];
-    ok = ok && encode_map(st, &m2[4], has_shared ? a.Ws_down : a.W_down, has_shared ? a.I_s : a.I, a.d, 1, bn2);
+    ok = ok && encode_map(st, &m2[4], has_shared ? a.Ws_down : a.W_down, has_shared ? a.I_s : a.I, a.d, 1,
+                          sc.pair ? 128 : bn2);
     m2[5] = m2[4];
     if (!ok) return MOE_ERR_CUDA;
 
@@ -524,6 +764,15 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
             else LEXI_DECODE_PAIR(128, 128, 3, 2);
         }
 #undef LEXI_DECODE_PAIR
+        layout->o_is_f32 = 1;
+    } else if (sc.pair) {
+        const int rows_t = 2 * kTileRows;
+        const int pr = rows / rows_t + (rows < a.E ? rows : a.E), ps = has_shared ? ceil_div(a.T, rows_t) : 0;
+        const int pairs1 = pr * ceil_div(a.I, 128) + ps * ceil_div(has_shared ? a.I_s : 1, 128);
+        const int pairs2 = (pr + ps) * ceil_div(a.d, 256);
+        e1 = launch_tc_pair<1, __nv_bfloat16>(m1, p1, pairs1, s, ch);
+        if (a.mid_event) cudaEventRecord(a.mid_event, s);
+        e2 = launch_tc_pair<2, float>(m2, p2, pairs2, s, ch);
         layout->o_is_f32 = 1;
     } else {
         e1 = launch_tc<1, 256, 128, 4, 1, __nv_bfloat16>(m1, p1, grid1, s, ch);

@@ -39,6 +39,7 @@ cudaError_t launch_router_tc(const TcState *st, const RouterArgs &a, int sm_coun
 // Tile shapes, split-K factors and the tile-list recipe of one call.
 struct TcSchedule {
     bool decode = false, direct = false;
+    bool pair = false;           // prefill GEMMs on CTA pairs (256-row tiles)
     bool tiles_built = false;    // the tile lists were already built by the dispatch or front-end kernel
     int bn1 = 256, bn2 = 256, a_rows = 128, ks_r = 1, ks_s = 1, kchunk_r = 64, kchunk_s = 64;
     TileBuildArgs tb{};

@@ -18,6 +18,7 @@ struct TileBuildArgs {
     // direct = 1 (T <= 128): phase 1 reads all T token rows of x for every touched expert (one
     // row block per group, rows = T); the epilogue places each row through the position table
     int32_t direct;
+    int32_t tile_rows;   // rows of one tile: 128, or 256 when a CTA pair shares a tile
     int32_t *stats;   // stats[0] += number of routed experts that received at least one token
 };
 
@@ -39,7 +40,7 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
     auto rows_of = [&](int g) { return g == a.E ? a.T : cnt_s[g]; };
     auto mblk1_of = [&](int g) {
         const int r = rows_of(g);
-        return a.direct ? (r > 0 ? 1 : 0) : (r + kTileRows - 1) / kTileRows;
+        return a.direct ? (r > 0 ? 1 : 0) : (r + a.tile_rows - 1) / a.tile_rows;
     };
     // tiles per group, then an exclusive scan over the (at most 129) groups by warp 0
     const int n1_routed = (a.N1_routed + a.feat1 - 1) / a.feat1;
@@ -47,7 +48,7 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
     const int n2 = (a.N2 + a.bn2 - 1) / a.bn2;
     for (int sidx = threadIdx.x; sidx < groups; sidx += blockDim.x) {
         const int g = group_of(sidx);
-        const int mblk = (rows_of(g) + kTileRows - 1) / kTileRows;
+        const int mblk = (rows_of(g) + a.tile_rows - 1) / a.tile_rows;
         if (rank == 0 && a.stats && g != a.E && rows_of(g) > 0) atomicAdd(a.stats, 1);
         sm.pre1[sidx] = mblk1_of(g) * (g == a.E ? n1_shared : n1_routed);
         sm.pre2[sidx] = mblk * n2 * (g == a.E ? a.ksplit_shared : a.ksplit_routed);
@@ -106,8 +107,8 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
                     t.row0 = 0;
                     t.rows = a.T;
                 } else {
-                    t.row0 = first + m * kTileRows;
-                    t.rows = min(kTileRows, rows - m * kTileRows);
+                    t.row0 = first + m * a.tile_rows;
+                    t.rows = min(a.tile_rows, rows - m * a.tile_rows);
                 }
                 t.n0 = n * a.feat1;
                 t.k0 = 0; t.klen = a.K1; t.slot = 0;
@@ -118,8 +119,8 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
                 const int K = g == a.E ? a.K2_shared : a.K2_routed;
                 const int m = local / (n2 * ks), rem = local % (n2 * ks);
                 const int n = rem / ks, sl = rem % ks;
-                t.row0 = first + m * kTileRows;
-                t.rows = min(kTileRows, rows - m * kTileRows);
+                t.row0 = first + m * a.tile_rows;
+                t.rows = min(a.tile_rows, rows - m * a.tile_rows);
                 t.n0 = n * a.bn2;
                 t.k0 = sl * kchunk;
                 t.klen = max(0, min(kchunk, K - sl * kchunk));
