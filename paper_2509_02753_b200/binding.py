@@ -299,7 +299,6 @@ def moe_plan_touched_experts(plan: int, stream=None) -> int:
     """Sum over the tensor-core layer calls since the last read of the experts that got tokens."""
     n = ctypes.c_int64()
     _check("moe_plan_touched_experts",
-    "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
            load_library().moe_plan_touched_experts(plan, ctypes.byref(n), _stream(stream)))
     return int(n.value)
 

@@ -211,7 +211,7 @@ def test_olmoe_and_deepseek_shaped_layers(name, T, k):
         assert info["excluded"] < 0.05
 
 
-@pytest.mark.parametrize("T,k", [(1, 2), (16, 1), (256, 2)])
+@pytest.mark.parametrize("T,k", [(1, 2), (16, 1), (256, 2), (4096, 2)])
 def test_mixtral_shaped_layer(T, k):
     """d=4096, E=8, I=14336, renormalised gates; 16 sampled tokens."""
     wl = synth.WORKLOADS["mixtral"]
