@@ -391,6 +391,36 @@ def run_ours(args):
                   "ms_per_sample_one_call_per_k": ms_alg1, "speedup": ms_alg1 / ms_prof,
                   "samples_tokens_per_s": Tp / (ms_prof * 1e-3)}
 
+    # ---- the paper's comparison (Section 3, Fig. 2) on shapes: expert pruning keeps k and shrinks E or
+    #      I, LExI keeps the weights and lowers k.  Same layer, decode (T=64) and prefill (T=8192).
+    pruning = []
+    if args.sweep and world == 1 and wl.name == "qwen15":
+        def timed(plan_p, ws_p, wl_p, Tp, kp):
+            xp = synth.make_tokens(wl_p, Tp, dtype, device, seed=4)
+            yp = torch.empty_like(xp)
+            ms_p, _ = run_case(B, plan_p, wl_p, ws_p, xp, yp, kp, 20, 5, False)
+            return ms_p / 20
+        for label, wl_p, kp in ([("baseline k=4", wl, 4), ("LExI k=3", wl, 3), ("LExI k=2", wl, 2)] +
+                                [(f"inter-pruned {int(f * 1000) / 10:g}% (E={synth.pruned(wl, 'inter', f).E}), k=4",
+                                  synth.pruned(wl, "inter", f), 4) for f in (0.125, 0.25, 0.5)] +
+                                [(f"intra-pruned {int(f * 1000) / 10:g}% (I={synth.pruned(wl, 'intra', f).I}), k=4",
+                                  synth.pruned(wl, "intra", f), 4) for f in (0.125, 0.25, 0.5)]):
+            if wl_p is wl:
+                plan_p, ws_p = plan, wsets
+            else:
+                lay_p = [synth.make_layer(wl_p, l, dtype, device) for l in range(2)]
+                ws_p = [B.make_weights(w) for w in lay_p]
+                plan_p = B.MoEPlan(wl_p.d, wl_p.E, wl_p.I, 8192, wl_p.k_base, dtype, I_shared=wl_p.I_shared,
+                                   shared_gate=wl_p.shared_gate)
+            row = {"variant": label}
+            for Tp in (64, 8192):
+                row[f"tokens_per_s_T{Tp}"] = Tp / (timed(plan_p, ws_p, wl_p, Tp, kp) * 1e-3)
+            pruning.append(row)
+            if wl_p is not wl:
+                plan_p.close()
+                del lay_p, ws_p
+                torch.cuda.empty_cache()
+
     # ---- whole stacks with uniform and per-layer k (rank 0 at N = 1)
     stacks = []
     if args.stacks and world == 1:
@@ -413,7 +443,7 @@ def run_ours(args):
                        "reasons": clocks.get("reasons", []), "samples": clocks.get("samples", 0)},
             "e2e": e2e, "gpu_launches": gpu_launches,
             "roofline": roof, "cpu_baseline": cpu_baseline,
-            "layer": main, "sweep": sweep, "stacks": stacks, "stage1": stage1,
+            "layer": main, "sweep": sweep, "stacks": stacks, "stage1": stage1, "pruning_shapes": pruning,
             "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
                       "bf16_tflops_burst": peaks["bf16_tflops"], "source": peaks["source"],
                       "nominal_hbm_gbs": NOMINAL_HBM_GBS, "nominal_bf16_tflops": NOMINAL_BF16_TFLOPS},

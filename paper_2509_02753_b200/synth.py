@@ -67,6 +67,22 @@ WORKLOADS: Dict[str, Workload] = {
 }
 
 
+def pruned(wl: Workload, kind: str, fraction: float) -> Workload:
+    """The shape an expert-pruning method leaves behind (Section 3, "Inter and Intra Expert
+    Pruning"): ``inter`` removes that fraction of the experts of every layer (and their router
+    rows), ``intra`` that fraction of each expert's FFN intermediate size; the number of active
+    experts per token stays k_base.  Only the shape is modelled (which experts or channels a
+    method would drop needs calibration data and trained weights); sizes are rounded down to a
+    multiple of 8 for the intermediate size."""
+    import dataclasses
+    assert kind in ("inter", "intra") and 0.0 <= fraction < 1.0
+    if kind == "inter":
+        E = max(wl.k_base, int(round(wl.E * (1.0 - fraction))))
+        return dataclasses.replace(wl, name=f"{wl.name}-inter{int(fraction * 1000)}", E=E)
+    I = max(8, int(wl.I * (1.0 - fraction)) // 8 * 8)
+    return dataclasses.replace(wl, name=f"{wl.name}-intra{int(fraction * 1000)}", I=I)
+
+
 def _seed(base: int, *parts) -> int:
     s = "/".join(str(p) for p in (base,) + parts)
     return zlib.crc32(s.encode()) & 0x7FFFFFFF

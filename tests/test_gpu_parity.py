@@ -211,6 +211,21 @@ def test_olmoe_and_deepseek_shaped_layers(name, T, k):
         assert info["excluded"] < 0.05
 
 
+@pytest.mark.parametrize("kind,frac,T", [("inter", 0.125, 64), ("inter", 0.5, 2048), ("intra", 0.125, 64),
+                                           ("intra", 0.125, 2048), ("intra", 0.5, 8)])
+def test_pruning_shaped_qwen_layers(kind, frac, T):
+    """Shapes left by 12.5-50 % inter/intra expert pruning: E' = 52 / 30, I' = 1232 (not a multiple
+    of 64: the K tail of the down projection is zero-filled by TMA) / 704."""
+    wl = synth.pruned(synth.WORKLOADS["qwen15"], kind, frac)
+    w = synth.make_layer(wl, 0, torch.bfloat16, DEV)
+    w_host = synth.to_host(w)
+    x = synth.make_tokens(wl, T, torch.bfloat16, DEV)
+    toks = None if T <= 64 else np.random.default_rng(T).choice(T, 40, replace=False)
+    with _plan(wl, T, 4, torch.bfloat16) as plan:
+        check_layer(plan, x, w, 4, False, shared_gate=True, tokens=toks, w_host=w_host)
+        check_layer(plan, x, w, 2, False, shared_gate=True, tokens=toks, w_host=w_host)
+
+
 @pytest.mark.parametrize("T,k", [(1, 2), (16, 1), (256, 2), (4096, 2)])
 def test_mixtral_shaped_layer(T, k):
     """d=4096, E=8, I=14336, renormalised gates; 16 sampled tokens."""

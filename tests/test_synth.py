@@ -61,3 +61,14 @@ def test_tensors_are_seeded_and_shaped():
     x = synth.make_tokens(wl, 64, torch.bfloat16)
     assert x.shape == (64, 256) and x.dtype == torch.bfloat16
     assert abs(float(x.float().std()) - 1.0) < 0.05
+
+
+def test_pruned_shapes_follow_the_papers_percentages():
+    """12.5 / 25 / 50 % inter pruning removes that share of the experts, intra that share of the FFN size."""
+    q = synth.WORKLOADS["qwen15"]
+    assert [synth.pruned(q, "inter", f).E for f in (0.125, 0.25, 0.5)] == [52, 45, 30]
+    assert [synth.pruned(q, "intra", f).I for f in (0.125, 0.25, 0.5)] == [1232, 1056, 704]
+    m = synth.WORKLOADS["mixtral"]
+    assert [synth.pruned(m, "inter", f).E for f in (0.125, 0.25, 0.5)] == [7, 6, 4]
+    p = synth.pruned(q, "intra", 0.25)
+    assert (p.E, p.k_base, p.d, p.I_shared) == (q.E, q.k_base, q.d, q.I_shared)
