@@ -249,6 +249,15 @@ int moe_last_routing(moe_plan_t *plan, int32_t *topk_idx, float *topk_w, int32_t
 int moe_last_residual_f32(moe_plan_t *plan, float *h_f32, int32_t T, void *cuda_stream);
 
 /*
+ * moe_debug_wait_timeout (test hook for the failure path): launches a one-block kernel whose only
+ * work is the library's bounded mbarrier wait on a barrier that nothing arrives on, with a limit of
+ * limit_us microseconds (1 .. 1,000,000).  The wait gives up, the kernel returns normally and the
+ * device status word carries the time-out, which the next moe_device_status reports as
+ * MOE_ERR_TIMEOUT; the context stays usable.  Errors: INVALID_ARG, CUDA.
+ */
+int moe_debug_wait_timeout(moe_plan_t *plan, int32_t limit_us, void *cuda_stream);
+
+/*
  * moe_device_status: synchronises the stream, reads and clears the device status word.
  * Returns MOE_OK, MOE_ERR_TIMEOUT, MOE_ERR_DEVICE_CHECK or MOE_ERR_CUDA.
  */

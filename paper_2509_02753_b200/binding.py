@@ -28,7 +28,7 @@ EXPORTS = (
     "moe_route_from_logits", "moe_last_routing", "moe_device_status", "moe_plan_launch_count",
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
     "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts",
-    "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
+    "moe_debug_wait_timeout", "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
 
@@ -79,6 +79,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_route_from_logits.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.moe_last_routing.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.moe_device_status.argtypes = [vp, vp]
+    lib.moe_debug_wait_timeout.argtypes = [vp, i32, vp]
     lib.moe_last_residual_f32.argtypes = [vp, vp, i32, vp]
     lib.moe_plan_touched_experts.argtypes = [vp, P(ctypes.c_int64), vp]
     lib.moe_profile_layer.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, P(ctypes.c_double),
@@ -321,6 +322,12 @@ def moe_last_residual_f32(plan: int, T: int, d: int, device="cuda", stream=None)
     _check("moe_last_residual_f32",
            load_library().moe_last_residual_f32(plan, out.data_ptr(), T, _stream(stream)))
     return out
+
+
+def moe_debug_wait_timeout(plan: int, limit_us: int, stream=None) -> None:
+    """Runs the bounded device-side wait on a barrier nobody signals; see moe_device_status."""
+    _check("moe_debug_wait_timeout",
+           load_library().moe_debug_wait_timeout(plan, limit_us, _stream(stream)))
 
 
 def moe_device_status(plan: int, stream=None) -> int:

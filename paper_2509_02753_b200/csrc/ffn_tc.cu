@@ -76,7 +76,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
     static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM columns: power of two");
     static_assert(STAGES * B_BYTES >= 128 * 128, "the 128-row operand read must stay inside the allocation");
 
-    pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -102,8 +101,27 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *slot_ptr;
+    // Phase 2 only: the tile lists were finished two kernels ago (phase 1 lets its successor start
+    // only after its own wait), and weights never change, so the weight halves of the first stages
+    // of this CTA's first tile are requested before waiting for phase 1; h follows after the wait.
+    int preloaded = 0;
+    if (PHASE == 2 && threadIdx.x == 0) {
+        const int nt = *p.n_tiles;
+        if ((int)blockIdx.x < nt) {
+            const Tile t = p.tiles[blockIdx.x];
+            const bool shared = t.group == p.E;
+            const int nk = (t.klen + kBK - 1) / kBK;
+            preloaded = nk < STAGES ? nk : STAGES;
+            for (int kc = 0; kc < preloaded; ++kc) {
+                mbar_expect_tx(full_bar(kc), A_BYTES + B_BYTES);
+                tma_load_3d(b_base + kc * B_BYTES, shared ? &mapB0_shared : &mapB0_routed, full_bar(kc),
+                            t.k0 + kc * kBK, t.n0, shared ? 0 : t.group);
+            }
+        }
+    }
     // everything above overlaps the tail of the previous kernel; its results are needed from here on
     pdl_wait();
+    pdl_trigger();
     const int n_tiles = *p.n_tiles;
 
     if (warp == 0) {
@@ -124,9 +142,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
                 for (int kc = 0; kc < nk; ++kc, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
+                    const int k = t.k0 + kc * kBK;
+                    if (PHASE == 2 && (int)it < preloaded) {     // weights of this stage are already on their way
+                        tma_load_3d(a_base + s * A_BYTES, mA, full_bar(s), k, t.row0, 0);
+                        continue;
+                    }
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, p.status)) { ok = false; break; }
                     mbar_expect_tx(full_bar(s), A_BYTES + B_BYTES);
-                    const int k = t.k0 + kc * kBK;
                     tma_load_3d(a_base + s * A_BYTES, mA, full_bar(s), k, t.row0, 0);
                     if (PHASE == 1) {
                         tma_load_3d(b_base + s * B_BYTES, mB0, full_bar(s), k, t.n0, grp);
@@ -313,7 +335,6 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
                    const TcParams p) {
     constexpr int BN = 256, STAGES = kPairStages, A_BYTES = kPairABytes, B_BYTES = kPairBBytes;
     constexpr int TMEM_COLS = 2 * BN;
-    pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -342,6 +363,7 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
     tc_fence_after();
     const uint32_t tmem_base = *slot_ptr;
     pdl_wait();
+    pdl_trigger();
     const int n_tiles = *p.n_tiles;
     const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
@@ -494,6 +516,18 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
     }
 }
 
+// One thread waits on an mbarrier that nothing will ever arrive on, with a short limit: the same
+// bounded wait as in the GEMM kernels, used by the test of the time-out path.
+__global__ void wait_probe_kernel(int32_t *status, unsigned long long limit_ns) {
+    __shared__ unsigned long long bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(b, 0, status, limit_ns);
+    }
+}
+
 // ------------------------------------------------------------------ tile lists
 __global__ void __launch_bounds__(1024) build_tiles_kernel(TileBuildArgs a) {
     pdl_trigger();
@@ -624,6 +658,11 @@ size_t tc_max_tiles(const moe_config_t &c, int phase) {
         return mblk_routed * ceil_div(c.I, 32) + mblk_shared * ceil_div(c.I_shared > 0 ? c.I_shared : 32, 32) + 1;
     return mblk_routed * ceil_div(c.d, 64) * slabs_for(c.I) +
            mblk_shared * ceil_div(c.d, 64) * (c.I_shared > 0 ? slabs_for(c.I_shared) : 1) + 1;
+}
+
+cudaError_t launch_wait_probe(int32_t *status, unsigned long long limit_ns, cudaStream_t s) {
+    wait_probe_kernel<<<1, 32, 0, s>>>(status, limit_ns);
+    return cudaGetLastError();
 }
 
 int tc_state_init(TcState *st, const moe_config_t &c) {

@@ -28,6 +28,7 @@ size_t tc_o_elems(const moe_config_t &c, int slabs);     // fp32-sized elements 
 size_t tc_os_elems(const moe_config_t &c, int slabs);    // ... `o_s`
 size_t tc_max_tiles(const moe_config_t &c, int phase);   // capacity of a tile list
 int    tc_state_init(TcState *st, const moe_config_t &c);
+cudaError_t launch_wait_probe(int32_t *status, unsigned long long limit_ns, cudaStream_t s);
 // Encodes a TMA tensor map (into the 128-byte CUtensorMap at `map`) of a bf16 tensor
 // [groups, rows, K] with K contiguous: box 64 x box_rows x 1, 128-byte swizzle, zero fill outside.
 bool   tc_encode_bf16_map(const TcState *st, void *map, const void *ptr, uint64_t K, uint64_t rows,

@@ -461,6 +461,16 @@ int moe_plan_touched_experts(moe_plan_t *p, int64_t *total, void *cuda_stream) {
     return MOE_OK;
 }
 
+int moe_debug_wait_timeout(moe_plan_t *p, int32_t limit_us, void *cuda_stream) {
+    if (!p || limit_us < 1 || limit_us > 1000000) return MOE_ERR_INVALID_ARG;
+    if (launch_wait_probe(p->ws.status, (unsigned long long)limit_us * 1000ull, (cudaStream_t)cuda_stream) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    ++p->launches;
+    return MOE_OK;
+}
+
 int moe_device_status(moe_plan_t *p, void *cuda_stream) {
     if (!p) return MOE_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)cuda_stream;

@@ -153,6 +153,19 @@ def test_zero_tokens_is_a_no_op_and_bad_arguments_are_refused():
         B.MoEPlan(250, 8, 512, 8, 2, torch.bfloat16)                 # d not a multiple of 8
 
 
+def test_bounded_wait_reports_a_timeout_and_leaves_the_context_usable():
+    """Failure path without a fault: a device-side wait that nothing satisfies gives up after its
+    limit, the status word says so, and the next layer call on the same plan is correct."""
+    wl = synth.WORKLOADS["tiny"]
+    w, x, w_host = _small(wl, 64, torch.bfloat16)
+    with _plan(wl, 64, 2, torch.bfloat16) as plan:
+        assert plan.device_status() == 0
+        B.moe_debug_wait_timeout(plan.handle, 500)
+        assert plan.device_status() == -6            # MOE_ERR_TIMEOUT
+        assert plan.device_status() == 0             # the read cleared it
+        check_layer(plan, x, w, 2, True, w_host=w_host)
+
+
 def test_two_calls_are_bit_identical():
     """Algorithm 1 relies on Delta(k_base) = 0: the same call twice gives the same bits."""
     wl = _custom("det", d=256, E=16, I=384, I_shared=256)
