@@ -91,6 +91,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
+        tma_prefetch_map(&mapA_routed); tma_prefetch_map(&mapA_shared);
+        tma_prefetch_map(&mapB0_routed); tma_prefetch_map(&mapB0_shared);
+        if (PHASE == 1) { tma_prefetch_map(&mapB1_routed); tma_prefetch_map(&mapB1_shared); }
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 128); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -122,6 +125,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
     // everything above overlaps the tail of the previous kernel; its results are needed from here on
     pdl_wait();
     pdl_trigger();
+    // the tile count and this CTA's first tile record are independent loads (the record lies inside
+    // the list's allocation whether or not it is valid); every role starts from them
+    const Tile first_tile = p.tiles[blockIdx.x];
     const int n_tiles = *p.n_tiles;
 
     if (warp == 0) {
@@ -129,7 +135,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            Tile t_next = (int)blockIdx.x < n_tiles ? p.tiles[blockIdx.x] : Tile{};
+            Tile t_next = first_tile;
             for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
                 const Tile t = t_next;       // the next tile's record is fetched while this one streams
                 if (tile + (int)gridDim.x < n_tiles) t_next = p.tiles[tile + gridDim.x];
@@ -165,7 +171,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
             constexpr uint32_t idesc = make_idesc_bf16(BN);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            int klen_next = (int)blockIdx.x < n_tiles ? p.tiles[blockIdx.x].klen : 0;
+            int klen_next = first_tile.klen;
             for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++tcount) {
                 const int nk = (klen_next + kBK - 1) / kBK;
                 if (tile + (int)gridDim.x < n_tiles) klen_next = p.tiles[tile + gridDim.x].klen;
@@ -193,7 +199,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
         const int q = warp & 3;                  // TMEM lane quarter this warp may read
         const int row_in_tile = q * 32 + lane;
         uint32_t tcount = 0;
-        Tile t_next = (int)blockIdx.x < n_tiles ? p.tiles[blockIdx.x] : Tile{};
+        Tile t_next = first_tile;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
             const Tile t = t_next;
             if (tile + (int)gridDim.x < n_tiles) t_next = p.tiles[tile + gridDim.x];
