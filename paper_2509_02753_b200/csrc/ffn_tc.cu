@@ -338,7 +338,14 @@ __global__ void __launch_bounds__(192, 1)
 ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_constant__ CUtensorMap mapA_shared,
                    const __grid_constant__ CUtensorMap mapB0_routed, const __grid_constant__ CUtensorMap mapB1_routed,
                    const __grid_constant__ CUtensorMap mapB0_shared, const __grid_constant__ CUtensorMap mapB1_shared,
+                   const __grid_constant__ CUtensorMap mapG64_routed, const __grid_constant__ CUtensorMap mapU64_routed,
+                   const __grid_constant__ CUtensorMap mapG64_shared, const __grid_constant__ CUtensorMap mapU64_shared,
                    const TcParams p) {
+    // Half-height tiles (Tile::pad = 1, at most 128 valid rows): the pair issues M = 128 MMAs, 64 rows
+    // per CTA.  Then each CTA's accumulator holds its 64 rows twice over the lanes: lanes 0-63 carry
+    // output columns 0-127 (B rows of CTA 0), lanes 64-127 columns 128-255 (B rows of CTA 1), both in
+    // TMEM columns 0-127.  Phase 1 therefore gives each CTA 64 gate rows followed by 64 up rows of the
+    // same 64 features (mapG64/mapU64, 64-row boxes), so that gate and up of a feature meet in a thread.
     constexpr int BN = 256, STAGES = kPairStages, A_BYTES = kPairABytes, B_BYTES = kPairBBytes;
     constexpr int TMEM_COLS = 2 * BN;
     extern __shared__ uint8_t smem_raw[];
@@ -383,6 +390,7 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
                 const Tile t = t_next;
                 if (tile + n_pairs < n_tiles) t_next = p.tiles[tile + n_pairs];
                 const bool shared = t.group == p.E;
+                const bool half = t.pad != 0;
                 const CUtensorMap *mA = shared ? &mapA_shared : &mapA_routed;
                 // this CTA's half of B: phase 1 -> gate rows (CTA 0) or up rows (CTA 1) of the same
                 // features; phase 2 -> rows n0 + 128 rank of W_down
@@ -391,7 +399,7 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
                                                    : (shared ? &mapB0_shared : &mapB0_routed);
                 const int b_row = PHASE == 1 ? t.n0 : t.n0 + 128 * (int)rank;
                 const int grp = shared ? 0 : t.group;
-                const int a_row = t.row0 + 128 * (int)rank;
+                const int a_row = t.row0 + (half ? 64 : 128) * (int)rank;
                 const int nk = (t.klen + kBK - 1) / kBK;
                 for (int kc = 0; kc < nk; ++kc, ++it) {
                     const int s = it % STAGES;
@@ -401,20 +409,28 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
                     if (rank == 0) mbar_expect_tx(full_bar(s), 2 * (A_BYTES + B_BYTES));
                     const int k = t.k0 + kc * kBK;
                     tma_load_3d_pair(a_base + s * A_BYTES, mA, full0, k, a_row, 0);
-                    tma_load_3d_pair(b_base + s * B_BYTES, mB, full0, k, b_row, grp);
+                    if (PHASE == 1 && half) {
+                        const int f = t.n0 + 64 * (int)rank;      // this CTA's 64 features: gate rows, then up rows
+                        tma_load_3d_pair(b_base + s * B_BYTES, shared ? &mapG64_shared : &mapG64_routed, full0, k, f, grp);
+                        tma_load_3d_pair(b_base + s * B_BYTES + B_BYTES / 2, shared ? &mapU64_shared : &mapU64_routed,
+                                         full0, k, f, grp);
+                    } else {
+                        tma_load_3d_pair(b_base + s * B_BYTES, mB, full0, k, b_row, grp);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (CTA 0 only)
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16_m(256, BN);
+            constexpr uint32_t idesc_full = make_idesc_bf16_m(256, BN), idesc_half = make_idesc_bf16_m(128, BN);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            int klen_next = pair_id < n_tiles ? p.tiles[pair_id].klen : 0;
+            Tile t_next = pair_id < n_tiles ? p.tiles[pair_id] : Tile{};
             for (int tile = pair_id; ok && tile < n_tiles; tile += n_pairs, ++tcount) {
-                const int nk = (klen_next + kBK - 1) / kBK;
-                if (tile + n_pairs < n_tiles) klen_next = p.tiles[tile + n_pairs].klen;
+                const int nk = (t_next.klen + kBK - 1) / kBK;
+                const uint32_t idesc = t_next.pad ? idesc_half : idesc_full;
+                if (tile + n_pairs < n_tiles) t_next = p.tiles[tile + n_pairs];
                 const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(buf), bph ^ 1u, p.status)) { ok = false; break; }
                 tc_fence_after();
@@ -437,8 +453,7 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
         const int q = warp & 3;
-        const int row_in_cta = q * 32 + lane;                    // row of this CTA's 128
-        const int row_in_tile = 128 * (int)rank + row_in_cta;    // row of the 256-row tile
+        const int row_in_cta = q * 32 + lane;                    // TMEM lane of this thread
         uint32_t tcount = 0;
         Tile t_next = pair_id < n_tiles ? p.tiles[pair_id] : Tile{};
         for (int tile = pair_id; tile < n_tiles; tile += n_pairs, ++tcount) {
@@ -446,7 +461,12 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
             if (tile + n_pairs < n_tiles) t_next = p.tiles[tile + n_pairs];
             const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
             const bool shared = t.group == p.E;
+            const bool half = t.pad != 0;
             const int N = shared ? p.N_shared : p.N_routed;
+            // full tile: lane = row of this CTA's 128, all 256 columns.  Half tile: lane % 64 = row of
+            // this CTA's 64, lane / 64 picks output columns 0-127 or 128-255 (TMEM columns 0-127 both).
+            const int cb = half ? (row_in_cta >> 6) : 0;
+            const int row_in_tile = half ? 64 * (int)rank + (row_in_cta & 63) : 128 * (int)rank + row_in_cta;
             const bool row_ok = row_in_tile < t.rows;
             const bool got = mbar_wait(tfull_bar(buf), bph, p.status);
             if (!__all_sync(0xffffffffu, got)) break;
@@ -455,12 +475,14 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
             OutT *obase = reinterpret_cast<OutT *>(shared ? p.out_shared : p.out_routed) +
                           (size_t)t.slot * (shared ? p.slab_stride_shared : p.slab_stride_routed);
             if (PHASE == 1) {
-                OutT *out = obase + (size_t)(t.row0 + row_in_tile) * N + t.n0;
+                const int feats = half ? 64 : 128;               // features this thread finishes
+                const int f0 = t.n0 + 64 * cb;
+                OutT *out = obase + (size_t)(t.row0 + row_in_tile) * N + f0;
 #pragma unroll 1
-                for (int c = 0; c < BN / 2; c += 16) {
+                for (int c = 0; c < feats; c += 16) {
                     uint32_t g[16], u[16];
                     tmem_ld16(taddr + c, g);
-                    tmem_ld16(taddr + BN / 2 + c, u);
+                    tmem_ld16(taddr + feats + c, u);
                     tmem_ld_wait();
                     uint32_t packed[8];
 #pragma unroll
@@ -468,19 +490,23 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
                         packed[i] = pack_bf16(silu_mul(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
                                               silu_mul(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1])));
                     if (row_ok) {
-                        if (t.n0 + c + 8 <= N)
+                        if (f0 + c + 8 <= N)
                             *reinterpret_cast<uint4 *>(out + c) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                        if (t.n0 + c + 16 <= N)
+                        if (f0 + c + 16 <= N)
                             *reinterpret_cast<uint4 *>(out + c + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
                     }
                 }
             } else {
                 float *stg = reinterpret_cast<float *>(smem_raw + (bar_base + 256u - raw)) + q * 32 * kStagePitch;
-                OutT *wbase = obase + (size_t)(t.row0 + 128 * (int)rank + q * 32) * N + t.n0;
-                const int rows_here = t.rows - 128 * (int)rank - q * 32;
+                // this warp's 32 rows of the tile and its first output column
+                const int warp_row0 = half ? 64 * (int)rank + 32 * (q & 1) : 128 * (int)rank + 32 * q;
+                const int col0 = t.n0 + (half ? 128 * (q >> 1) : 0);
+                const int cols = half ? 128 : BN;
+                OutT *wbase = obase + (size_t)(t.row0 + warp_row0) * N + col0;
+                const int rows_here = t.rows - warp_row0;
                 const int rr0 = lane >> 3, cc = 4 * (lane & 7);
 #pragma unroll 1
-                for (int c = 0; c < BN; c += 32) {
+                for (int c = 0; c < cols; c += 32) {
                     uint32_t v0[16], v1[16];
                     tmem_ld16(taddr + c, v0);
                     tmem_ld16(taddr + c + 16, v1);
@@ -492,7 +518,7 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
                         wr[4 + i] = make_uint4(v1[4 * i], v1[4 * i + 1], v1[4 * i + 2], v1[4 * i + 3]);
                     }
                     __syncwarp();
-                    const bool col_ok = t.n0 + c + cc + 4 <= N;
+                    const bool col_ok = col0 + c + cc + 4 <= N;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const int rr = 4 * j + rr0;
@@ -626,7 +652,8 @@ cudaError_t launch_tc_pair(const CUtensorMap *maps, const TcParams &p, int max_p
     const int clusters = max_pairs < max_clusters ? (max_pairs < 1 ? 1 : max_pairs) : max_clusters;
     cfg.gridDim = dim3(2 * clusters);
     cfg.numAttrs = chained ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, kern, maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], p);
+    return cudaLaunchKernelEx(&cfg, kern, maps[0], maps[1], maps[2], maps[3], maps[4], maps[5],
+                              maps[6], maps[7], maps[8], maps[9], p);
 }
 
 }  // namespace
@@ -743,7 +770,7 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
     const int bn1 = sc.bn1, bn2 = sc.bn2, a_rows = sc.a_rows, ks_r = sc.ks_r, ks_s = sc.ks_s;
 
     // ---- tensor maps
-    CUtensorMap m1[6], m2[6];
+    CUtensorMap m1[10], m2[10];
     bool ok = true;
     const void *dummy = a.x;   // maps of an absent shared expert are never dereferenced
     if (sc.direct) ok = ok && encode_map(st, &m1[0], a.x, a.d, a.T, 1, a_rows);   // every group reads x itself
@@ -761,6 +788,14 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
     ok = ok && encode_map(st, &m2[4], has_shared ? a.Ws_down : a.W_down, has_shared ? a.I_s : a.I, a.d, 1,
                           sc.pair ? 128 : bn2);
     m2[5] = m2[4];
+    // 64-row weight boxes for the half-height tiles of the CTA-pair kernel (phase 1 only)
+    if (sc.pair) {
+        ok = ok && encode_map(st, &m1[6], a.W_gate, a.d, a.I, a.E, 64);
+        ok = ok && encode_map(st, &m1[7], a.W_up, a.d, a.I, a.E, 64);
+        ok = ok && encode_map(st, &m1[8], has_shared ? a.Ws_gate : dummy, a.d, has_shared ? a.I_s : a.T, 1, 64);
+        ok = ok && encode_map(st, &m1[9], has_shared ? a.Ws_up : dummy, a.d, has_shared ? a.I_s : a.T, 1, 64);
+        for (int i = 6; i < 10; ++i) m2[i] = m2[2];
+    }
     if (!ok) return MOE_ERR_CUDA;
 
     // ---- tile lists (already built by the fused front end in direct mode)

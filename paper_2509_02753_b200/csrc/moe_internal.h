@@ -29,7 +29,7 @@ struct __align__(16) Tile {
     int32_t k0;        // first element of the reduction range
     int32_t klen;      // length of the reduction range
     int32_t slot;      // which partial-sum slab of the output this tile writes (split-K)
-    int32_t pad;
+    int32_t pad;       // CTA-pair lists: 1 = at most 128 rows, run as a half-height tile
 };
 
 struct Workspace {

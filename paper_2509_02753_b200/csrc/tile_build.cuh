@@ -112,6 +112,9 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
                 }
                 t.n0 = n * a.feat1;
                 t.k0 = 0; t.klen = a.K1; t.slot = 0;
+                // pair mode: a last block of at most 128 rows is marked so that the pair runs it as a
+                // 128-row MMA (64 rows per CTA) instead of a 256-row one
+                t.pad = (a.tile_rows > kTileRows && t.rows <= kTileRows) ? 1 : 0;
                 a.tiles1[i] = t;
             } else {
                 const int ks = g == a.E ? a.ksplit_shared : a.ksplit_routed;
@@ -125,6 +128,7 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
                 t.k0 = sl * kchunk;
                 t.klen = max(0, min(kchunk, K - sl * kchunk));
                 t.slot = sl;
+                t.pad = (a.tile_rows > kTileRows && t.rows <= kTileRows) ? 1 : 0;
                 a.tiles2[i] = t;
             }
         }
