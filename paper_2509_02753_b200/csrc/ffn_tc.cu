@@ -723,11 +723,11 @@ void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs 
     TcSchedule &sc = *out;
     sc.decode = decode;
     sc.direct = direct;
-    // Prefill with at least 384 rows per expert on average: the GEMMs run on CTA pairs (256-row tiles,
-    // cta_group::2); below that the padding of 256-row tiles costs more than the pairs gain.
+    // Prefill with at least 128 rows per expert on average: the GEMMs run on CTA pairs (256-row tiles,
+    // cta_group::2, leftovers as half-height tiles); below that the 1-CTA kernel measured faster.
     // LEXI_PREFILL_2CTA=0 / =1 forces the choice.
     static const char *pair_env = getenv("LEXI_PREFILL_2CTA");
-    const bool pair_auto = (int64_t)a.T * a.k >= (int64_t)384 * a.E;
+    const bool pair_auto = (int64_t)a.T * a.k >= (int64_t)128 * a.E;
     sc.pair = !decode && !direct && (pair_env ? pair_env[0] == '1' : pair_auto);
     const int dec_bn = decode_bn_override() ? decode_bn_override() : 128;
     sc.bn1 = decode ? dec_bn : 256;       // phase-1 tile: bn1/2 gate rows + bn1/2 up rows
