@@ -136,8 +136,11 @@ int moe_layer_forward(moe_plan_t *plan, const void *x, const moe_layer_weights_t
  * moe_layer_forward_host: the same call for callers that hold x and y in HOST memory
  * (pinned memory makes the copies asynchronous).  Copies x to the device, runs
  * moe_layer_forward, copies y back, all on the given stream; weights stay on the device.
- * The staging buffers belong to the plan.  Does not synchronise: wait on the stream
- * before reading y_host.
+ * The staging buffers belong to the plan.  Calls of 4096 tokens or more are cut into 2 (4 from
+ * 16384) token chunks whose copies run on two side streams of the plan and overlap the kernels of
+ * the neighbouring chunks; the given stream waits for the last copy, so, as for a single chunk:
+ * does not synchronise, wait on the stream before reading y_host.  After such a call
+ * moe_last_routing describes the last chunk only.
  */
 int moe_layer_forward_host(moe_plan_t *plan, const void *x_host, const moe_layer_weights_t *w,
                            int32_t T, int32_t k_l, int32_t renorm, void *y_host,

@@ -21,6 +21,9 @@ struct moe_plan {
     int32_t forced_schedule = MOE_SCHED_AUTO;
     int32_t last_T = 0, last_k = 0;
     int32_t *status_host = nullptr;   // pinned
+    // host-buffer entry point: copy streams and events of its token-chunk pipeline
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_out = nullptr, ev_in[4] = {}, ev_done[4] = {};
     int sm_count = 148;
     bool use_tc_router = true;   // cleared by MOE_SCHED_SIMT so that schedule stays tensor-core free
     bool use_direct = true;      // fused front end + direct-x gate/up GEMM for small decode calls
@@ -267,6 +270,14 @@ int moe_plan_destroy(moe_plan_t *p) {
     for (void *q : p->allocs) cudaFree(q);
     for (cudaEvent_t e : p->events) cudaEventDestroy(e);
     if (p->status_host) cudaFreeHost(p->status_host);
+    if (p->copy_in) cudaStreamDestroy(p->copy_in);
+    if (p->copy_out) cudaStreamDestroy(p->copy_out);
+    if (p->ev_start) cudaEventDestroy(p->ev_start);
+    if (p->ev_out) cudaEventDestroy(p->ev_out);
+    for (int c = 0; c < 4; ++c) {
+        if (p->ev_in[c]) cudaEventDestroy(p->ev_in[c]);
+        if (p->ev_done[c]) cudaEventDestroy(p->ev_done[c]);
+    }
     cudaGetLastError();
     delete p;
     return MOE_OK;
@@ -339,17 +350,62 @@ int moe_layer_forward_host(moe_plan_t *p, const void *x_host, const moe_layer_we
     if (rc != MOE_OK) return rc;
     if (T == 0) return MOE_OK;
     cudaStream_t s = (cudaStream_t)cuda_stream;
-    const size_t bytes = (size_t)T * p->cfg.d * elem_size(p->cfg.dtype);
-    if (cudaMemcpyAsync(p->ws.x_stage, x_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
-        cudaGetLastError();
-        return MOE_ERR_CUDA;
+    const size_t row_bytes = (size_t)p->cfg.d * elem_size(p->cfg.dtype);
+    // Tokens are independent, so a large call is cut into up to four chunks: the upload of chunk
+    // c+1 and the download of chunk c-1 (two side streams, both copy engines) overlap the kernels
+    // of chunk c on the caller's stream.  The caller's stream waits for the last download.
+    const int n_chunks = T >= 16384 ? 4 : (T >= 4096 ? 2 : 1);
+    if (n_chunks == 1) {
+        const size_t bytes = (size_t)T * row_bytes;
+        if (cudaMemcpyAsync(p->ws.x_stage, x_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+            cudaGetLastError();
+            return MOE_ERR_CUDA;
+        }
+        rc = layer_impl(p, p->ws.x_stage, w, T, k_l, renorm ? 1 : 0, p->ws.y_stage, 0, s);
+        if (rc != MOE_OK) return rc;
+        if (cudaMemcpyAsync(y_host, p->ws.y_stage, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+            cudaGetLastError();
+            return MOE_ERR_CUDA;
+        }
+        return MOE_OK;
     }
-    rc = layer_impl(p, p->ws.x_stage, w, T, k_l, renorm ? 1 : 0, p->ws.y_stage, 0, s);
-    if (rc != MOE_OK) return rc;
-    if (cudaMemcpyAsync(y_host, p->ws.y_stage, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
-        cudaGetLastError();
-        return MOE_ERR_CUDA;
+    if (!p->copy_in) {      // first chunked call: the side streams and events (no device memory)
+        bool ok = cudaStreamCreateWithFlags(&p->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&p->copy_out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p->ev_out, cudaEventDisableTiming) == cudaSuccess;
+        for (int c = 0; ok && c < 4; ++c)
+            ok = cudaEventCreateWithFlags(&p->ev_in[c], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&p->ev_done[c], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) { cudaGetLastError(); return MOE_ERR_CUDA; }
     }
+    const int per = ((T + n_chunks - 1) / n_chunks + 127) / 128 * 128;
+    bool ok = cudaEventRecord(p->ev_start, s) == cudaSuccess &&
+              cudaStreamWaitEvent(p->copy_in, p->ev_start, 0) == cudaSuccess &&
+              cudaStreamWaitEvent(p->copy_out, p->ev_start, 0) == cudaSuccess;
+    for (int c = 0; ok && c < n_chunks; ++c) {
+        const int t0 = c * per, tn = (T - t0 < per) ? T - t0 : per;
+        if (tn <= 0) break;
+        ok = cudaMemcpyAsync((char *)p->ws.x_stage + t0 * row_bytes, (const char *)x_host + t0 * row_bytes,
+                             tn * row_bytes, cudaMemcpyHostToDevice, p->copy_in) == cudaSuccess &&
+             cudaEventRecord(p->ev_in[c], p->copy_in) == cudaSuccess;
+    }
+    for (int c = 0; ok && c < n_chunks; ++c) {
+        const int t0 = c * per, tn = (T - t0 < per) ? T - t0 : per;
+        if (tn <= 0) break;
+        ok = cudaStreamWaitEvent(s, p->ev_in[c], 0) == cudaSuccess;
+        if (!ok) break;
+        rc = layer_impl(p, (char *)p->ws.x_stage + t0 * row_bytes, w, tn, k_l, renorm ? 1 : 0,
+                        (char *)p->ws.y_stage + t0 * row_bytes, 0, s);
+        if (rc != MOE_OK) return rc;
+        ok = cudaEventRecord(p->ev_done[c], s) == cudaSuccess &&
+             cudaStreamWaitEvent(p->copy_out, p->ev_done[c], 0) == cudaSuccess &&
+             cudaMemcpyAsync((char *)y_host + t0 * row_bytes, (char *)p->ws.y_stage + t0 * row_bytes,
+                             tn * row_bytes, cudaMemcpyDeviceToHost, p->copy_out) == cudaSuccess;
+    }
+    ok = ok && cudaEventRecord(p->ev_out, p->copy_out) == cudaSuccess &&
+         cudaStreamWaitEvent(s, p->ev_out, 0) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return MOE_ERR_CUDA; }
     return MOE_OK;
 }
 

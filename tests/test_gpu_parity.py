@@ -193,6 +193,24 @@ def test_host_buffer_entry_point_matches_device_entry_point():
         assert torch.equal(y_dev.cpu(), y_host)
 
 
+def test_chunked_host_entry_point_matches_device_entry_point():
+    """4096 tokens or more: the host-buffer call pipelines token chunks; tokens are independent, so
+    the result is the device call's, bit for bit."""
+    wl = _custom("hostpipe", d=256, E=8, I=256, I_shared=128, shared_gate=True)
+    w = B.make_weights(synth.make_layer(wl, 0, torch.bfloat16, DEV))
+    for T in (4500, 16500):
+        x = synth.make_tokens(wl, T, torch.bfloat16, "cpu").pin_memory()
+        y_host = torch.empty_like(x).pin_memory()
+        with _plan(wl, T, 2, torch.bfloat16) as plan:
+            y_dev = plan.layer_forward(x.to(DEV), w, 2, False)
+            for _ in range(2):
+                y_host.zero_()
+                B.moe_layer_forward_host(plan.handle, x, w, 2, False, y_host)
+                torch.cuda.synchronize()
+                assert torch.equal(y_dev.cpu(), y_host)
+            assert plan.device_status() == 0
+
+
 # --------------------------------------------------------------------------- model-shaped layers
 
 @pytest.mark.parametrize("T,k", [(1, 4), (8, 4), (64, 4), (64, 1), (2048, 4), (2048, 2), (8192, 4), (8192, 1)])
