@@ -593,16 +593,6 @@ bool encode_map(const TcState *st, CUtensorMap *m, const void *ptr, uint64_t K, 
 }
 
 int ceil_div(int a, int b) { return (a + b - 1) / b; }
-// LEXI_DECODE_BN=64|128 overrides the weight-tile height of the decode schedule (tuning aid).
-int decode_bn_override() {
-    static int v = -1;
-    if (v < 0) {
-        const char *e = getenv("LEXI_DECODE_BN");
-        const int n = e ? atoi(e) : 0;
-        v = (n == 64 || n == 128) ? n : 0;
-    }
-    return v;
-}
 int clampi(int v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : v); }
 int slabs_for(int K) { return clampi(ceil_div(K, 1024), 1, 8); }
 size_t decode_row_cap(const moe_config_t &c) {
@@ -729,9 +719,8 @@ void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs 
     static const char *pair_env = getenv("LEXI_PREFILL_2CTA");
     const bool pair_auto = (int64_t)a.T * a.k >= (int64_t)128 * a.E;
     sc.pair = !decode && !direct && (pair_env ? pair_env[0] == '1' : pair_auto);
-    const int dec_bn = decode_bn_override() ? decode_bn_override() : 128;
-    sc.bn1 = decode ? dec_bn : 256;       // phase-1 tile: bn1/2 gate rows + bn1/2 up rows
-    sc.bn2 = decode ? dec_bn : 256;
+    sc.bn1 = decode ? 128 : 256;          // phase-1 tile: bn1/2 gate rows + bn1/2 up rows
+    sc.bn2 = decode ? 128 : 256;
     sc.a_rows = 128;
     if (decode) sc.a_rows = a.T <= 32 ? 32 : (a.T <= 64 ? 64 : 128);
     int ks_r = 1, ks_s = 1;
@@ -811,7 +800,7 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
     const int mblk_shared = has_shared ? ceil_div(a.T, kTileRows) : 0;
     const int max1 = mblk_routed * ceil_div(a.I, bn1 / 2) + mblk_shared * ceil_div(has_shared ? a.I_s : 1, bn1 / 2);
     const int max2 = mblk_routed * ceil_div(a.d, bn2) * ks_r + mblk_shared * ceil_div(a.d, bn2) * ks_s;
-    const int ctas_per_sm = decode ? (bn1 == 64 ? 3 : 2) : 1;
+    const int ctas_per_sm = decode ? 2 : 1;
     const int grid1 = clampi(max1, 1, sm_count * ctas_per_sm);
     const int grid2 = clampi(max2, 1, sm_count * ctas_per_sm);
 
@@ -837,15 +826,9 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
         e2 = launch_tc<2, BN_, AR_, ST_, CTAS_, float>(m2, p2, grid2, s, ch);                      \
     } while (0)
     if (decode) {
-        if (bn1 == 64) {
-            if (a_rows == 32) LEXI_DECODE_PAIR(64, 32, 6, 3);
-            else if (a_rows == 64) LEXI_DECODE_PAIR(64, 64, 4, 3);
-            else LEXI_DECODE_PAIR(64, 128, 3, 3);
-        } else {
-            if (a_rows == 32) LEXI_DECODE_PAIR(128, 32, 5, 2);
-            else if (a_rows == 64) LEXI_DECODE_PAIR(128, 64, 4, 2);
-            else LEXI_DECODE_PAIR(128, 128, 3, 2);
-        }
+        if (a_rows == 32) LEXI_DECODE_PAIR(128, 32, 5, 2);
+        else if (a_rows == 64) LEXI_DECODE_PAIR(128, 64, 4, 2);
+        else LEXI_DECODE_PAIR(128, 128, 3, 2);
 #undef LEXI_DECODE_PAIR
         layout->o_is_f32 = 1;
     } else if (sc.pair) {
