@@ -13,7 +13,11 @@
 //               tile's MMAs overlap), SwiGLU or plain store
 // Decode schedule: BN = 128, small activation box (32/64/128 rows), K split into slabs so that
 // enough CTAs stream disjoint weight slices to saturate HBM; two CTAs per SM.
-// Prefill schedule: BN = 256, four 48 KB stages, one CTA per SM, all 512 TMEM columns.
+// Prefill schedule: BN = 256, four 48 KB stages, one CTA per SM, all 512 TMEM columns; from 128 rows
+// per expert on, the CTA-pair kernel below (256-row tiles shared by a cluster of two CTAs through
+// tcgen05.mma.cta_group::2, six 32 KB stages per CTA, leftover blocks as half-height tiles).
+// Small decode calls read x itself in phase 1 and place rows through a position table; phase 2
+// requests the weights of its first stages before it waits for phase 1 (launches are chained).
 //
 // Every mbarrier wait is bounded in time; a wait that runs out sets the status word and the CTA
 // leaves through the common exit (TMEM is always freed).
