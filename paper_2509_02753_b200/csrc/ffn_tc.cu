@@ -684,7 +684,7 @@ size_t tc_max_tiles(const moe_config_t &c, int phase) {
     if (phase == 1)
         return mblk_routed * ceil_div(c.I, 32) + mblk_shared * ceil_div(c.I_shared > 0 ? c.I_shared : 32, 32) + 1;
     return mblk_routed * ceil_div(c.d, 64) * slabs_for(c.I) +
-           mblk_shared * ceil_div(c.d, 64) * (c.I_shared > 0 ? slabs_for(c.I_shared) : 1) + 1;
+           mblk_shared * ceil_div(c.d, 64) * (c.I_shared > 0 ? slabs_for(c.I_shared) : 1) + 1 + kMaxBalanceTiles;
 }
 
 cudaError_t launch_wait_probe(int32_t *status, unsigned long long limit_ns, cudaStream_t s) {
@@ -710,7 +710,7 @@ int tc_state_init(TcState *st, const moe_config_t &c) {
 }
 
 void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs &a, int schedule,
-                      bool direct, TcSchedule *out) {
+                      bool direct, int sm_count, TcSchedule *out) {
     const bool decode = schedule == MOE_SCHED_DECODE;
     const int rows = a.T * a.k;
     const bool has_shared = a.I_s > 0;
@@ -749,6 +749,8 @@ void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs 
     tb.status = ws.status;
     tb.direct = direct ? 1 : 0;
     tb.tile_rows = sc.pair ? 2 * kTileRows : kTileRows;
+    // prefill: consumers of the phase-2 list (CTAs, or CTA pairs), for the balance of long shared tiles
+    tb.rr2 = (!decode && !direct && has_shared) ? (sc.pair ? sm_count / 2 : sm_count) : 0;
     tb.stats = ws.stats;
 }
 

@@ -46,7 +46,7 @@ struct TcSchedule {
     TileBuildArgs tb{};
 };
 void   tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs &a, int schedule,
-                        bool direct, TcSchedule *out);
+                        bool direct, int sm_count, TcSchedule *out);
 int    tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, const FfnArgs &a,
                       const TcSchedule &sc, int sm_count, cudaStream_t s, uint64_t *launches,
                       TcOutputLayout *layout);

@@ -102,7 +102,7 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
     const bool direct = sched == MOE_SCHED_DECODE && p->use_direct && T <= kFrontMaxTokens &&
                         T * k <= kFrontMaxPairs;
     TcSchedule sc{};
-    if (sched != MOE_SCHED_SIMT) tc_make_schedule(c, ws, fa, sched, direct, &sc);
+    if (sched != MOE_SCHED_SIMT) tc_make_schedule(c, ws, fa, sched, direct, p->sm_count, &sc);
 
     ra.chained = chained;
     fa.chained = chained && sched != MOE_SCHED_SIMT;

@@ -5,6 +5,8 @@
 
 namespace lexi {
 
+constexpr int kMaxBalanceTiles = 2048;   // most null tiles the balancing of list 2 may add
+
 struct TileBuildArgs {
     const int32_t *counts, *offsets;
     int32_t E, T, has_shared;
@@ -19,6 +21,10 @@ struct TileBuildArgs {
     // row block per group, rows = T); the epilogue places each row through the position table
     int32_t direct;
     int32_t tile_rows;   // rows of one tile: 128, or 256 when a CTA pair shares a tile
+    // rr2 > 0: list 2 is consumed round-robin by rr2 CTAs (or CTA pairs) and the shared expert's tiles
+    // reduce over a longer K than the routed ones; null tiles (rows = 0) are slipped in behind the
+    // shared tiles so that every consumer ends up with the same amount of work
+    int32_t rr2;
     int32_t *stats;   // stats[0] += number of routed experts that received at least one token
 };
 
@@ -76,19 +82,53 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
             }
         if (lane == 31) {
             int t1 = i1, t2 = i2;
-            if (t1 > a.cap1 || t2 > a.cap2) { atomicOr(a.status, kStatusBadIndex); t1 = 0; t2 = 0; }
+            if (t1 > a.cap1 || t2 + kMaxBalanceTiles > a.cap2) { atomicOr(a.status, kStatusBadIndex); t1 = 0; t2 = 0; }
             sm.pre1[groups] = t1; sm.pre2[groups] = t2;
-            if (rank == 0) {
-                a.n_tiles[0] = t1;
-                a.n_tiles[1] = t2;
-            }
         }
     }
     __syncthreads();
+    // Balance of list 2 (see rr2): S long shared tiles come first; if S is not a multiple of the
+    // consumer count C, consumers 0..rem-1 hold one long tile more.  The next (ratio-1) rounds
+    // therefore hand short tiles only to consumers rem..C-1 and null tiles to the others.
+    int bal_S = 0, bal_C = 0, bal_rem = 0, bal_rows = 0;
+    if (a.rr2 > 0 && a.has_shared && !a.direct && a.ksplit_shared == 1 && a.ksplit_routed == 1 &&
+        a.K2_shared > a.K2_routed && sm.pre2[groups] > 0) {
+        bal_S = groups > 1 ? sm.pre2[1] : sm.pre2[groups];
+        bal_C = a.rr2;
+        bal_rem = bal_S % bal_C;
+        bal_rows = bal_rem > 0 ? (a.K2_shared + a.K2_routed - 1) / a.K2_routed - 1 : 0;
+        if (bal_rows * bal_rem > kMaxBalanceTiles) bal_rows = 0;
+    }
+    const int extra2 = bal_rows * bal_rem;
+    if (rank == 0 && threadIdx.x == 0) {
+        a.n_tiles[0] = sm.pre1[groups];
+        a.n_tiles[1] = sm.pre2[groups] + extra2;
+    }
     for (int phase = 0; phase < 2; ++phase) {
         const int32_t *pre = phase == 0 ? sm.pre1 : sm.pre2;
-        const int total = pre[groups];
-        for (int i = rank * blockDim.x + threadIdx.x; i < total; i += n_blocks * blockDim.x) {
+        const int logical = pre[groups];
+        const int total = logical + (phase == 1 ? extra2 : 0);
+        for (int idx = rank * blockDim.x + threadIdx.x; idx < total; idx += n_blocks * blockDim.x) {
+            int i = idx;
+            if (phase == 1 && extra2 > 0 && idx >= bal_S) {
+                const int j = idx - bal_S;
+                int shorts;
+                bool null_tile = false;
+                if (j < bal_rows * bal_C) {
+                    const int qrow = j / bal_C, r = j % bal_C;
+                    null_tile = r >= bal_C - bal_rem;
+                    shorts = j - (qrow * bal_rem + max(0, r - (bal_C - bal_rem)));
+                } else {
+                    shorts = j - extra2;
+                }
+                i = bal_S + shorts;
+                if (null_tile || i >= logical) {
+                    Tile z;
+                    z.group = 0; z.row0 = 0; z.rows = 0; z.n0 = 0; z.k0 = 0; z.klen = 0; z.slot = 0; z.pad = 0;
+                    a.tiles2[idx] = z;
+                    continue;
+                }
+            }
             int lo = 0, hi = groups - 1;
             while (lo < hi) {                     // last slot with pre[slot] <= i
                 const int mid = (lo + hi + 1) >> 1;
@@ -115,7 +155,7 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
                 // pair mode: a last block of at most 128 rows is marked so that the pair runs it as a
                 // 128-row MMA (64 rows per CTA) instead of a 256-row one
                 t.pad = (a.tile_rows > kTileRows && t.rows <= kTileRows) ? 1 : 0;
-                a.tiles1[i] = t;
+                a.tiles1[idx] = t;
             } else {
                 const int ks = g == a.E ? a.ksplit_shared : a.ksplit_routed;
                 const int kchunk = g == a.E ? a.kchunk_shared : a.kchunk_routed;
@@ -129,7 +169,7 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
                 t.klen = max(0, min(kchunk, K - sl * kchunk));
                 t.slot = sl;
                 t.pad = (a.tile_rows > kTileRows && t.rows <= kTileRows) ? 1 : 0;
-                a.tiles2[i] = t;
+                a.tiles2[idx] = t;
             }
         }
     }
