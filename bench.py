@@ -309,7 +309,7 @@ def run_ours(args):
         roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = recorded_traffic(f"{wl.name}_T{T}_k{k}_ffn1")
-    pairs = main["schedule"] == "prefill" and T * k >= 128 * wl.E and os.environ.get("LEXI_PREFILL_2CTA", "1") != "0"
+    pairs = main["schedule"] == "prefill" and os.environ.get("LEXI_PREFILL_2CTA", "1") != "0"
     roof["kernel"] = ("ffn_tc_pair_kernel<phase 1> (gate/up GEMM + SwiGLU on CTA pairs)" if pairs
                       else "ffn_tc_kernel<phase 1> (gate/up GEMM + SwiGLU)")
     roof["launch_ms"] = stages.get("ffn1")

@@ -58,9 +58,10 @@ typedef enum {
     MOE_SCHED_AUTO    = 0,
     MOE_SCHED_SIMT    = 1,  /* CUDA-core FMA kernels; the only schedule for MOE_F32          */
     MOE_SCHED_DECODE  = 2,  /* tcgen05, narrow weight tiles + split-K: weight streaming      */
-    MOE_SCHED_PREFILL = 3   /* tcgen05, 128x256 tiles (256x256 on CTA pairs from 128 rows per
-                               expert; LEXI_PREFILL_2CTA=0/1 in the environment forces it),
+    MOE_SCHED_PREFILL = 3,  /* tcgen05, 256x256 tiles on CTA pairs (LEXI_PREFILL_2CTA=0 in the
+                               environment selects the 128x256 one-CTA kernel instead),
                                double-buffered TMEM accumulators                            */
+    MOE_SCHED_PREFILL_1CTA = 4  /* prefill on the one-CTA 128x256 kernel; never chosen by AUTO */
 } moe_schedule_t;
 
 /* Shapes fixed when the plan is made. */

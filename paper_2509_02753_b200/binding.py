@@ -19,8 +19,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "liblexi_moe.so")
 
 MOE_F32, MOE_BF16 = 0, 1
-MOE_SCHED_AUTO, MOE_SCHED_SIMT, MOE_SCHED_DECODE, MOE_SCHED_PREFILL = 0, 1, 2, 3
-SCHEDULE_NAMES = {0: "auto", 1: "simt", 2: "decode", 3: "prefill"}
+MOE_SCHED_AUTO, MOE_SCHED_SIMT, MOE_SCHED_DECODE, MOE_SCHED_PREFILL, MOE_SCHED_PREFILL_1CTA = 0, 1, 2, 3, 4
+SCHEDULE_NAMES = {0: "auto", 1: "simt", 2: "decode", 3: "prefill", 4: "prefill-1cta"}
 
 EXPORTS = (
     "moe_plan_create", "moe_plan_destroy", "moe_plan_workspace_bytes", "moe_plan_set_schedule",

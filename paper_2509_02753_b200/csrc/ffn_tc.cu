@@ -172,13 +172,16 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(BN);
+            // tiles of at most 64 rows run as M = 64 MMAs (half the tensor-core time); their 64 rows
+            // sit in lanes 0-15 of each 32-lane quarter of TMEM
+            constexpr uint32_t idesc128 = make_idesc_bf16(BN), idesc64 = make_idesc_bf16_m(64, BN);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            int klen_next = first_tile.klen;
+            Tile t_nx = first_tile;
             for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++tcount) {
-                const int nk = (klen_next + kBK - 1) / kBK;
-                if (tile + (int)gridDim.x < n_tiles) klen_next = p.tiles[tile + gridDim.x].klen;
+                const int nk = (t_nx.klen + kBK - 1) / kBK;
+                const uint32_t idesc = t_nx.rows <= 64 ? idesc64 : idesc128;
+                if (tile + (int)gridDim.x < n_tiles) t_nx = p.tiles[tile + gridDim.x];
                 const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(buf), bph ^ 1u, p.status)) { ok = false; break; }
                 tc_fence_after();
@@ -201,7 +204,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5)
         const int q = warp & 3;                  // TMEM lane quarter this warp may read
-        const int row_in_tile = q * 32 + lane;
         uint32_t tcount = 0;
         Tile t_next = first_tile;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
@@ -211,6 +213,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
             // everything that depends only on the tile record comes before the wait for its accumulator
             const bool shared = t.group == p.E;
             const int N = shared ? p.N_shared : p.N_routed;
+            // M = 128: lane = row.  M = 64 (rows <= 64): row 16 q + l lives in lane l < 16 of quarter q.
+            const bool small = t.rows <= 64;
+            const int row_in_tile = small ? (lane < 16 ? q * 16 + lane : 1 << 20) : q * 32 + lane;
             bool row_ok = row_in_tile < t.rows;
             int out_row = t.row0 + row_in_tile;
             if (p.pos != nullptr && !shared) {   // direct mode: the tile holds all tokens, keep the routed ones
@@ -247,10 +252,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
                 // each lane parks its row's 32 columns in shared memory; the warp then writes them
                 // out four rows per instruction, 128 contiguous bytes per row
                 float *stg = reinterpret_cast<float *>(smem_raw + (bar_base + 256u - raw)) + q * 32 * kStagePitch;
+                const int warp_row0 = small ? q * 16 : q * 32;        // first tile row held by this warp
                 OutT *wbase = reinterpret_cast<OutT *>(shared ? p.out_shared : p.out_routed) +
                               (size_t)t.slot * (shared ? p.slab_stride_shared : p.slab_stride_routed) +
-                              (size_t)(t.row0 + q * 32) * N + t.n0;
-                const int rows_here = t.rows - q * 32;       // valid rows among this warp's 32
+                              (size_t)(t.row0 + warp_row0) * N + t.n0;
+                const int rows_here = min(t.rows - warp_row0, small ? 16 : 32);   // valid rows of this warp
                 const int rr0 = lane >> 3, cc = 4 * (lane & 7);
 #pragma unroll 1
                 for (int c = 0; c < BN; c += 32) {
@@ -717,12 +723,12 @@ void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs 
     TcSchedule &sc = *out;
     sc.decode = decode;
     sc.direct = direct;
-    // Prefill with at least 128 rows per expert on average: the GEMMs run on CTA pairs (256-row tiles,
-    // cta_group::2, leftovers as half-height tiles); below that the 1-CTA kernel measured faster.
+    // Prefill: the GEMMs run on CTA pairs (256-row tiles, cta_group::2, leftovers as half-height
+    // tiles); measured at least as fast as the 1-CTA kernel from 68 rows per expert upwards.
     // LEXI_PREFILL_2CTA=0 / =1 forces the choice.
     static const char *pair_env = getenv("LEXI_PREFILL_2CTA");
-    const bool pair_auto = (int64_t)a.T * a.k >= (int64_t)128 * a.E;
-    sc.pair = !decode && !direct && (pair_env ? pair_env[0] == '1' : pair_auto);
+    const bool pair_auto = true;
+    sc.pair = !decode && !direct && schedule != MOE_SCHED_PREFILL_1CTA && (pair_env ? pair_env[0] == '1' : pair_auto);
     sc.bn1 = decode ? 128 : 256;          // phase-1 tile: bn1/2 gate rows + bn1/2 up rows
     sc.bn2 = decode ? 128 : 256;
     sc.a_rows = 128;

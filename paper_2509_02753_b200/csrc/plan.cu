@@ -287,8 +287,8 @@ uint64_t moe_plan_workspace_bytes(const moe_plan_t *p) { return p ? p->bytes : 0
 uint64_t moe_plan_launch_count(const moe_plan_t *p) { return p ? p->launches : 0; }
 
 int moe_plan_set_schedule(moe_plan_t *p, int32_t schedule) {
-    if (!p || schedule < MOE_SCHED_AUTO || schedule > MOE_SCHED_PREFILL) return MOE_ERR_INVALID_ARG;
-    if ((schedule == MOE_SCHED_DECODE || schedule == MOE_SCHED_PREFILL) &&
+    if (!p || schedule < MOE_SCHED_AUTO || schedule > MOE_SCHED_PREFILL_1CTA) return MOE_ERR_INVALID_ARG;
+    if ((schedule == MOE_SCHED_DECODE || schedule == MOE_SCHED_PREFILL || schedule == MOE_SCHED_PREFILL_1CTA) &&
         (p->cfg.dtype != MOE_BF16 || !tc_shape_ok(p->cfg)))
         return MOE_ERR_SHAPE;
     p->forced_schedule = schedule;

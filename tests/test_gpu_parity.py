@@ -36,7 +36,7 @@ def _plan(wl, max_T, max_k, dtype, routed_scale=1.0):
 
 def _schedules(plan):
     out = [B.MOE_SCHED_SIMT]
-    for s in (B.MOE_SCHED_DECODE, B.MOE_SCHED_PREFILL):
+    for s in (B.MOE_SCHED_DECODE, B.MOE_SCHED_PREFILL, B.MOE_SCHED_PREFILL_1CTA):
         try:
             plan.set_schedule(s)
             out.append(s)
