@@ -61,7 +61,13 @@ typedef enum {
     MOE_SCHED_PREFILL = 3,  /* tcgen05, 256x256 tiles on CTA pairs (LEXI_PREFILL_2CTA=0 in the
                                environment selects the 128x256 one-CTA kernel instead),
                                double-buffered TMEM accumulators                            */
-    MOE_SCHED_PREFILL_1CTA = 4  /* prefill on the one-CTA 128x256 kernel; never chosen by AUTO */
+    MOE_SCHED_PREFILL_1CTA = 4, /* prefill on the one-CTA 128x256 kernel; never chosen by AUTO */
+    MOE_SCHED_DECODE_FUSED = 5  /* bf16, at most 8 tokens: the whole layer (router to combine) in one
+                               cooperative launch that streams the touched experts' weights
+                               through mma.sync with the tokens in the N dimension; a call
+                               with more tokens falls back to MOE_SCHED_DECODE.  Needs d, I and
+                               I_shared to be multiples of 32 (else set_schedule -> SHAPE).
+                               The launch needs every SM of the device to itself while it runs. */
 } moe_schedule_t;
 
 /* Shapes fixed when the plan is made. */
@@ -129,7 +135,9 @@ int moe_plan_get_schedule(const moe_plan_t *plan, int32_t T, int32_t k_l);
  * histogram, prefix scan, stable permutation, gather of x into expert order), grouped
  * gate/up GEMM with SwiGLU, grouped down GEMM, weighted combine plus shared expert.
  * Schedule under MOE_SCHED_AUTO: SIMT for fp32; for bf16 DECODE when T * k_l < 16 * E
- * (fewer than 16 tokens per expert on average: weight streaming decides the time), else PREFILL.
+ * (fewer than 16 tokens per expert on average: weight streaming decides the time), else PREFILL;
+ * a DECODE call of at most 8 tokens runs as DECODE_FUSED where the shape allows it
+ * (LEXI_DECODE_FUSED=0 in the environment keeps such calls on the kernel chain).
  * Errors: INVALID_ARG, ALIGN, CUDA.
  */
 int moe_layer_forward(moe_plan_t *plan, const void *x, const moe_layer_weights_t *w,
@@ -253,6 +261,17 @@ int moe_last_routing(moe_plan_t *plan, int32_t *topk_idx, float *topk_w, int32_t
  * Errors: INVALID_ARG (also for fp32 plans, whose h is the residual stream itself).
  */
 int moe_last_residual_f32(moe_plan_t *plan, float *h_f32, int32_t T, void *cuda_stream);
+
+/*
+ * Debug hook of MOE_SCHED_DECODE_FUSED (the paper has no counterpart): with enable != 0 every
+ * later one-launch layer call records, per CTA, eight %globaltimer values in ns (start, logits
+ * sent, shared gate/up stream done, logits complete, routed, gate/up stream done, h' complete,
+ * end).  out_host (host memory, may be NULL) receives up to `capacity` values, [CTA][8], of the
+ * last stamped call after synchronising the stream; *n_ctas (may be NULL) the number of CTAs.
+ * Errors: INVALID_ARG (also when the plan's shape has no one-launch layer), CUDA.
+ */
+int moe_debug_fused_stamps(moe_plan_t *plan, int32_t enable, uint64_t *out_host, int32_t capacity,
+                           int32_t *n_ctas, void *cuda_stream);
 
 /*
  * moe_debug_wait_timeout (test hook for the failure path): launches a one-block kernel whose only

@@ -20,7 +20,8 @@ LIB_PATH = os.path.join(_PKG, "liblexi_moe.so")
 
 MOE_F32, MOE_BF16 = 0, 1
 MOE_SCHED_AUTO, MOE_SCHED_SIMT, MOE_SCHED_DECODE, MOE_SCHED_PREFILL, MOE_SCHED_PREFILL_1CTA = 0, 1, 2, 3, 4
-SCHEDULE_NAMES = {0: "auto", 1: "simt", 2: "decode", 3: "prefill", 4: "prefill-1cta"}
+MOE_SCHED_DECODE_FUSED = 5
+SCHEDULE_NAMES = {0: "auto", 1: "simt", 2: "decode", 3: "prefill", 4: "prefill-1cta", 5: "decode-fused"}
 
 EXPORTS = (
     "moe_plan_create", "moe_plan_destroy", "moe_plan_workspace_bytes", "moe_plan_set_schedule",
@@ -28,6 +29,7 @@ EXPORTS = (
     "moe_route_from_logits", "moe_last_routing", "moe_device_status", "moe_plan_launch_count",
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
     "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts",
+    "moe_debug_fused_stamps",
     "moe_debug_wait_timeout", "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
@@ -82,6 +84,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_debug_wait_timeout.argtypes = [vp, i32, vp]
     lib.moe_last_residual_f32.argtypes = [vp, vp, i32, vp]
     lib.moe_plan_touched_experts.argtypes = [vp, P(ctypes.c_int64), vp]
+    lib.moe_debug_fused_stamps.argtypes = [vp, i32, P(ctypes.c_uint64), i32, P(i32), vp]
     lib.moe_profile_layer.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, P(ctypes.c_double),
                                       P(ctypes.c_double), vp]
     dbl_p, i32_p = P(ctypes.c_double), P(i32)
@@ -302,6 +305,19 @@ def moe_plan_touched_experts(plan: int, stream=None) -> int:
     _check("moe_plan_touched_experts",
            load_library().moe_plan_touched_experts(plan, ctypes.byref(n), _stream(stream)))
     return int(n.value)
+
+
+def moe_debug_fused_stamps(plan: int, enable: bool, read: bool = False, stream=None):
+    """Switches the time stamps of the one-launch layer on or off; with read=True returns the last
+    stamped call's values as a list of per-CTA lists of eight ns values."""
+    lib = load_library()
+    n = ctypes.c_int32()
+    _check("moe_debug_fused_stamps", lib.moe_debug_fused_stamps(plan, int(enable), None, 0, ctypes.byref(n), _stream(stream)))
+    if not read:
+        return None
+    buf = (ctypes.c_uint64 * (n.value * 8))()
+    _check("moe_debug_fused_stamps", lib.moe_debug_fused_stamps(plan, int(enable), buf, n.value * 8, None, _stream(stream)))
+    return [[int(buf[c * 8 + i]) for i in range(8)] for c in range(n.value)]
 
 
 def moe_plan_set_stage_timing(plan: int, enable: bool) -> None:

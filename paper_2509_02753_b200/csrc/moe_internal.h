@@ -59,6 +59,13 @@ struct Workspace {
     double  *prof_sums = nullptr;     // [max_k + 1]
     int32_t *stats = nullptr;      // [4] counters read by moe_plan_touched_experts
     int32_t *pos = nullptr;        // [E, 128] direct mode: output row of (expert, token) or -1
+    // one-launch layer for calls of at most kFusedMaxTokens tokens (decode_fused.cu)
+    float   *f_part0 = nullptr;    // router logit partials, 128 floats per (16 rows, 128 columns) chunk
+    float   *f_parts = nullptr;    // [SMs][2] per-CTA partial sums of down-stream blocks split between CTAs
+    int32_t *f_tickets = nullptr;  // [d / 16] arrival counters of the down-stream blocks (zero between calls)
+    uint32_t *f_bar = nullptr;     // grid-barrier counter (only grows; reset by the host from time to time)
+    __nv_bfloat16 *f_hbuf = nullptr;  // [8, I_s + U_cap * I] gate-weighted hidden activations
+    unsigned long long *f_stamps = nullptr;   // [SMs, 8] %globaltimer stamps of the last stamped call
 };
 
 #ifdef __CUDACC__
@@ -143,6 +150,32 @@ cudaError_t launch_combine(const CombineArgs &a, cudaStream_t s, uint64_t *launc
 // sum of squares of f(X;k_base); partial holds ceil(T*d/1024) * (a.k+1) floats.
 cudaError_t launch_profile(const CombineArgs &a, int renorm, float *partial, double *sums, cudaStream_t s,
                            uint64_t *launches);
+
+// ---- one-launch layer for tiny decode calls (decode_fused.cu) ----------------------------
+constexpr int kFusedMaxTokens = 8;
+#ifndef LEXI_FUSED_WARPS
+#define LEXI_FUSED_WARPS 12
+#endif
+// warps per CTA (one CTA per SM).  12 leaves each thread 168 registers: two chunks of weights in
+// flight per warp without spills; 16 warps (128 registers, spills) measured 5-10 % slower.
+constexpr int kFusedWarps = LEXI_FUSED_WARPS;
+constexpr int kFusedThreads = kFusedWarps * 32;
+constexpr int kFusedMaxCtaBlocks = 512;   // row blocks of one stream that may fall to one CTA
+struct FusedArgs {
+    const void *x; __nv_bfloat16 *y; float *h_run; int mode;   // mode 0: y = MoE(x); 1: h_run += MoE(x), y = round(h_run)
+    const void *router_W; const float *router_bias; const void *w_s;   // w_s NULL: shared gate = 1
+    const void *W_gate, *W_up, *W_down, *Ws_gate, *Ws_up, *Ws_down;
+    int T, d, E, I, I_s, k, renorm;
+    float routed_scale;
+    float *logits; int32_t *topk_idx; float *topk_w; float *gamma;
+    int32_t *counts, *offsets, *perm, *inv_perm, *stats, *status;
+    float *part0, *parts; int32_t *tickets;   // logit partials; per-CTA partials and arrival counters of the down stream
+    uint32_t *bar; __nv_bfloat16 *hbuf; int hs;                       // hs: row pitch of hbuf
+    unsigned long long *stamps;                                       // NULL, or [grid, 8] time stamps (debug)
+};
+size_t fused_smem_bytes(int d);
+cudaError_t fused_prepare(int d);    // opts the kernel in to its shared-memory size (once per plan)
+cudaError_t launch_decode_fused(const FusedArgs &a, int sm_count, cudaStream_t s, uint64_t *launches);
 
 cudaError_t launch_widen(const void *src, float *dst, size_t n, int dtype, cudaStream_t s,
                          uint64_t *launches);

@@ -28,6 +28,11 @@ struct moe_plan {
     bool use_tc_router = true;   // cleared by MOE_SCHED_SIMT so that schedule stays tensor-core free
     bool use_direct = true;      // fused front end + direct-x gate/up GEMM for small decode calls
     bool use_pdl = true;         // programmatic dependent launch along the decode chain
+    bool fused_ok = false;       // the one-launch layer for <= kFusedMaxTokens tokens is available for this shape
+    bool use_fused = true;       // ... and chosen by MOE_SCHED_AUTO (LEXI_DECODE_FUSED=0 turns that off)
+    int fused_tk_total = 0, fused_hs = 0;
+    uint64_t fused_calls = 0;
+    bool fused_stamps = false;   // debug: later one-launch calls record time stamps
     TcState tc{};
     // stage timing: kMaxTimedCalls sets of MOE_N_STAGES + 1 events
     bool timing = false;
@@ -70,9 +75,43 @@ int check_weights(const moe_plan *p, const moe_layer_weights_t *w) {
 }
 
 int pick_schedule(const moe_plan *p, int T, int k) {
+    const bool fused_fits = p->fused_ok && T <= kFusedMaxTokens;
+    if (p->forced_schedule == MOE_SCHED_DECODE_FUSED) return fused_fits ? MOE_SCHED_DECODE_FUSED : MOE_SCHED_DECODE;
     if (p->forced_schedule != MOE_SCHED_AUTO) return p->forced_schedule;
     if (p->cfg.dtype != MOE_BF16 || !tc_shape_ok(p->cfg)) return MOE_SCHED_SIMT;
-    return ((int64_t)T * k < (int64_t)16 * p->cfg.E) ? MOE_SCHED_DECODE : MOE_SCHED_PREFILL;
+    if ((int64_t)T * k >= (int64_t)16 * p->cfg.E) return MOE_SCHED_PREFILL;
+    return (fused_fits && p->use_fused) ? MOE_SCHED_DECODE_FUSED : MOE_SCHED_DECODE;
+}
+
+// Whole layer in one cooperative launch (decode_fused.cu).
+int fused_layer(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, int k, int renorm, void *y,
+                int mode, cudaStream_t s) {
+    const moe_config_t &c = p->cfg;
+    Workspace &ws = p->ws;
+    // the barrier counter only grows; long before it could wrap it is put back to zero in stream order
+    if ((++p->fused_calls & 0xfffffu) == 0 && cudaMemsetAsync(ws.f_bar, 0, sizeof(uint32_t), s) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    FusedArgs fa{};
+    fa.x = x; fa.y = (__nv_bfloat16 *)y; fa.h_run = ws.h_run; fa.mode = mode;
+    fa.router_W = w->router_W; fa.router_bias = w->router_bias;
+    fa.w_s = (c.I_shared > 0 && c.shared_gate) ? w->w_s : nullptr;
+    fa.W_gate = w->W_gate; fa.W_up = w->W_up; fa.W_down = w->W_down;
+    fa.Ws_gate = w->Ws_gate; fa.Ws_up = w->Ws_up; fa.Ws_down = w->Ws_down;
+    fa.T = T; fa.d = c.d; fa.E = c.E; fa.I = c.I; fa.I_s = c.I_shared; fa.k = k; fa.renorm = renorm;
+    fa.routed_scale = c.routed_scale;
+    fa.logits = ws.logits; fa.topk_idx = ws.topk_idx; fa.topk_w = ws.topk_w; fa.gamma = ws.gamma;
+    fa.counts = ws.counts; fa.offsets = ws.offsets; fa.perm = ws.perm; fa.inv_perm = ws.inv_perm;
+    fa.stats = ws.stats; fa.status = ws.status;
+    fa.part0 = ws.f_part0; fa.parts = ws.f_parts; fa.tickets = ws.f_tickets;
+    fa.bar = ws.f_bar; fa.hbuf = ws.f_hbuf; fa.hs = p->fused_hs;
+    fa.stamps = p->fused_stamps ? ws.f_stamps : nullptr;
+    if (launch_decode_fused(fa, p->sm_count, s, &p->launches) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    return MOE_OK;
 }
 
 // mode 3: Stage-1 profiling (no y; sums of squared differences go to ws.prof_sums).
@@ -97,7 +136,17 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
     FfnArgs fa{c.dtype, T, k, c.d, c.E, c.I, c.I_shared, ws.counts, ws.offsets, x, ws.x_perm,
                w->W_gate, w->W_up, w->W_down, w->Ws_gate, w->Ws_up, w->Ws_down,
                ws.h, ws.h_s, ws.o, ws.o_s, false, ev ? ev[2] : nullptr, ev ? ev[3] : nullptr};
-    const int sched = pick_schedule(p, T, k);
+    int sched = pick_schedule(p, T, k);
+    if (sched == MOE_SCHED_DECODE_FUSED && (mode == 0 || mode == 1)) {
+        mark(1); mark(2);                 // the whole call is booked under the first GEMM stage
+        const int rc = fused_layer(p, x, w, T, k, renorm, y, mode, s);
+        if (rc != MOE_OK) return rc;
+        mark(3); mark(4); mark(5);
+        p->last_T = T;
+        p->last_k = k;
+        return MOE_OK;
+    }
+    if (sched == MOE_SCHED_DECODE_FUSED) sched = MOE_SCHED_DECODE;     // Stage-1 profiling needs the slot outputs
     // small decode calls: one fused front-end launch, and the gate/up GEMM reads x directly
     const bool direct = sched == MOE_SCHED_DECODE && p->use_direct && T <= kFrontMaxTokens &&
                         T * k <= kFrontMaxPairs;
@@ -260,6 +309,28 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
     }
     const int rc = tc_state_init(&p->tc, c);
     if (rc != MOE_OK) { moe_plan_destroy(p); return rc; }
+    // one-launch layer for tiny decode calls: scratch for its partial sums, arrival counters and h'
+    if (c.dtype == MOE_BF16 && tc_shape_ok(c) && c.d % 32 == 0 && c.I % 32 == 0 && c.I_shared % 32 == 0 &&
+        fused_smem_bytes(c.d) <= 160 * 1024 &&
+        ((c.E < kFusedMaxTokens * c.max_k ? c.E : kFusedMaxTokens * c.max_k) * (c.I / 8)) / sms + 2 <= kFusedMaxCtaBlocks &&
+        (c.I_shared / 8) / sms + 2 <= kFusedMaxCtaBlocks) {
+        const int ucap = c.E < kFusedMaxTokens * c.max_k ? c.E : kFusedMaxTokens * c.max_k;
+        p->fused_tk_total = c.d / 16;
+        p->fused_hs = c.I_shared + ucap * c.I;
+        bool fok = ws_alloc(p, &ws.f_part0, (size_t)((c.E + 15) / 16) * ((c.d + 127) / 128) * 128) &&
+                   ws_alloc(p, &ws.f_parts, (size_t)sms * 2 * 128) &&
+                   ws_alloc(p, &ws.f_tickets, (size_t)p->fused_tk_total) &&
+                   ws_alloc(p, &ws.f_bar, (size_t)4) &&
+                   ws_alloc(p, &ws.f_hbuf, (size_t)kFusedMaxTokens * p->fused_hs) &&
+                   ws_alloc(p, &ws.f_stamps, (size_t)sms * 8);
+        fok = fok && cudaMemset(ws.f_tickets, 0, sizeof(int32_t) * p->fused_tk_total) == cudaSuccess &&
+              cudaMemset(ws.f_bar, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess &&
+              fused_prepare(c.d) == cudaSuccess;
+        if (!fok) { cudaGetLastError(); moe_plan_destroy(p); return MOE_ERR_WORKSPACE; }
+        p->fused_ok = true;
+        const char *env = getenv("LEXI_DECODE_FUSED");
+        p->use_fused = !(env && env[0] == '0');
+    }
     *out = p;
     return MOE_OK;
 }
@@ -287,7 +358,8 @@ uint64_t moe_plan_workspace_bytes(const moe_plan_t *p) { return p ? p->bytes : 0
 uint64_t moe_plan_launch_count(const moe_plan_t *p) { return p ? p->launches : 0; }
 
 int moe_plan_set_schedule(moe_plan_t *p, int32_t schedule) {
-    if (!p || schedule < MOE_SCHED_AUTO || schedule > MOE_SCHED_PREFILL_1CTA) return MOE_ERR_INVALID_ARG;
+    if (!p || schedule < MOE_SCHED_AUTO || schedule > MOE_SCHED_DECODE_FUSED) return MOE_ERR_INVALID_ARG;
+    if (schedule == MOE_SCHED_DECODE_FUSED && !p->fused_ok) return MOE_ERR_SHAPE;
     if ((schedule == MOE_SCHED_DECODE || schedule == MOE_SCHED_PREFILL || schedule == MOE_SCHED_PREFILL_1CTA) &&
         (p->cfg.dtype != MOE_BF16 || !tc_shape_ok(p->cfg)))
         return MOE_ERR_SHAPE;
@@ -527,6 +599,23 @@ int moe_debug_wait_timeout(moe_plan_t *p, int32_t limit_us, void *cuda_stream) {
     return MOE_OK;
 }
 
+int moe_debug_fused_stamps(moe_plan_t *p, int32_t enable, uint64_t *out_host, int32_t capacity, int32_t *n_ctas,
+                           void *cuda_stream) {
+    if (!p || !p->fused_ok || capacity < 0) return MOE_ERR_INVALID_ARG;
+    p->fused_stamps = enable != 0;
+    if (n_ctas) *n_ctas = p->sm_count;
+    if (out_host && capacity > 0) {
+        const size_t n = (size_t)capacity < (size_t)p->sm_count * 8 ? (size_t)capacity : (size_t)p->sm_count * 8;
+        cudaStream_t s = (cudaStream_t)cuda_stream;
+        if (cudaMemcpyAsync(out_host, p->ws.f_stamps, n * sizeof(uint64_t), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) {
+            cudaGetLastError();
+            return MOE_ERR_CUDA;
+        }
+    }
+    return MOE_OK;
+}
+
 int moe_device_status(moe_plan_t *p, void *cuda_stream) {
     if (!p) return MOE_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)cuda_stream;
@@ -537,6 +626,12 @@ int moe_device_status(moe_plan_t *p, void *cuda_stream) {
         return MOE_ERR_CUDA;
     }
     const int32_t v = *p->status_host;
+    if ((v & kStatusTimeout) && p->fused_ok) {
+        // a one-launch layer that gave up may have left arrival counters behind
+        cudaMemsetAsync(p->ws.f_tickets, 0, sizeof(int32_t) * p->fused_tk_total, s);
+        cudaMemsetAsync(p->ws.f_bar, 0, sizeof(uint32_t), s);
+        cudaStreamSynchronize(s);
+    }
     if (v & kStatusTimeout) return MOE_ERR_TIMEOUT;
     if (v & kStatusBadIndex) return MOE_ERR_DEVICE_CHECK;
     return MOE_OK;

@@ -36,7 +36,7 @@ def _plan(wl, max_T, max_k, dtype, routed_scale=1.0):
 
 def _schedules(plan):
     out = [B.MOE_SCHED_SIMT]
-    for s in (B.MOE_SCHED_DECODE, B.MOE_SCHED_PREFILL, B.MOE_SCHED_PREFILL_1CTA):
+    for s in (B.MOE_SCHED_DECODE, B.MOE_SCHED_PREFILL, B.MOE_SCHED_PREFILL_1CTA, B.MOE_SCHED_DECODE_FUSED):
         try:
             plan.set_schedule(s)
             out.append(s)
@@ -267,6 +267,59 @@ def test_mixtral_shaped_layer(T, k):
     toks = None if T <= 16 else np.random.default_rng(T).choice(T, 16, replace=False)
     with _plan(wl, T, 2, torch.bfloat16) as plan:
         check_layer(plan, x, w, k, True, tokens=toks, w_host=w_host)
+
+
+# --------------------------------------------------------------------------- one-launch layer (T <= 8)
+
+@pytest.mark.parametrize("name,T,k,renorm", [
+    ("qwen15", 1, 4, False), ("qwen15", 1, 1, True), ("qwen15", 2, 3, False), ("qwen15", 3, 4, True),
+    ("qwen15", 7, 2, False), ("qwen15", 8, 4, False), ("olmoe", 1, 8, False), ("olmoe", 8, 8, False),
+    ("olmoe", 5, 3, False), ("dsv2lite", 1, 6, False), ("dsv2lite", 6, 6, False), ("mixtral", 1, 2, True),
+    ("mixtral", 8, 2, True), ("mixtral", 4, 1, True)])
+def test_one_launch_layer_for_at_most_8_tokens(name, T, k, renorm):
+    """Calls of at most 8 tokens run the whole layer in one cooperative launch; same checks as the
+    kernel chain, all tokens evaluated by the oracle, and the same bits on a repeated call."""
+    wl = synth.WORKLOADS[name]
+    w = synth.make_layer(wl, 2, torch.bfloat16, DEV)
+    w_host = synth.to_host(w)
+    x = synth.make_tokens(wl, T, torch.bfloat16, DEV)
+    with _plan(wl, 8, wl.k_base, torch.bfloat16) as plan:
+        assert plan.schedule_for(T, k) == B.MOE_SCHED_DECODE_FUSED
+        check_layer(plan, x, w, k, renorm, shared_gate=wl.shared_gate, w_host=w_host)
+        ws = B.make_weights(w)
+        a = plan.layer_forward(x, ws, k, renorm).clone()
+        plan.layer_forward(x, ws, 1, renorm)
+        b = plan.layer_forward(x, ws, k, renorm)
+        assert torch.equal(a, b)
+        assert plan.device_status() == 0
+        # the kernel chain gives the same layer within the output format's spacing
+        plan.set_schedule(B.MOE_SCHED_DECODE)
+        c = plan.layer_forward(x, ws, k, renorm)
+        rms = float(c.float().pow(2).mean().sqrt())
+        assert float((a.float() - c.float()).abs().max()) <= 4e-2 * rms
+
+
+def test_one_launch_layers_chained_in_a_stack():
+    """DeepSeek-V2-Lite-shaped stack (first 6 layers), T=8, per-layer k: every layer is one launch
+    that adds into the fp32 residual stream."""
+    wl = synth.WORKLOADS["dsv2lite"]
+    T, L = 8, 6
+    k_vec = [6, 2, 4, 3, 5, 2]
+    layers = [synth.make_layer(wl, l, torch.bfloat16, DEV) for l in range(L)]
+    structs = [B.make_weights(w) for w in layers]
+    x = synth.make_tokens(wl, T, torch.bfloat16, DEV)
+    ows = [oracle_weights(synth.to_host(w)) for w in layers]
+    h_ref, _, margins = orc.moe_stack(x.cpu(), ows, k_vec, wl.renorm, shared_gate=wl.shared_gate)
+    with _plan(wl, T, wl.k_base, torch.bfloat16) as plan:
+        assert plan.schedule_for(T, 6) == B.MOE_SCHED_DECODE_FUSED
+        h = x.clone()
+        plan.stack_forward(h, structs, k_vec, wl.renorm)
+        assert plan.device_status() == 0
+        h32 = plan.last_residual_f32(T).cpu().numpy()
+        safe = np.all(margins > 8e-3, axis=0)
+        assert safe.sum() >= 1, safe.sum()
+        assert rel_err(h32[safe], h_ref[safe]) <= TOL[torch.bfloat16]
+        assert_out_close(h.float().cpu().numpy()[safe], h_ref[safe], torch.bfloat16, "one-launch stack")
 
 
 # --------------------------------------------------------------------------- stack
