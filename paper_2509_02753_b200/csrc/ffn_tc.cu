@@ -724,10 +724,12 @@ void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs 
     sc.decode = decode;
     sc.direct = direct;
     // Prefill: the GEMMs run on CTA pairs (256-row tiles, cta_group::2, leftovers as half-height
-    // tiles); measured at least as fast as the 1-CTA kernel from 68 rows per expert upwards.
+    // tiles); measured at least as fast as the 1-CTA kernel from 64 rows per expert upwards.
     // LEXI_PREFILL_2CTA=0 / =1 forces the choice.
+    // Below 64 rows per expert the one-CTA 128x256 kernel measured 3-6 % faster (its tiles are half as
+    // tall, and the call is bound by the weight stream rather than by the tensor cores).
     static const char *pair_env = getenv("LEXI_PREFILL_2CTA");
-    const bool pair_auto = true;
+    const bool pair_auto = (long long)rows >= 64ll * a.E;
     sc.pair = !decode && !direct && schedule != MOE_SCHED_PREFILL_1CTA && (pair_env ? pair_env[0] == '1' : pair_auto);
     sc.bn1 = decode ? 128 : 256;          // phase-1 tile: bn1/2 gate rows + bn1/2 up rows
     sc.bn2 = decode ? 128 : 256;

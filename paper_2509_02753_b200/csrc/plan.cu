@@ -108,8 +108,11 @@ int fused_layer(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T,
     fa.bar = ws.f_bar; fa.hbuf = ws.f_hbuf; fa.hs = p->fused_hs;
     fa.stamps = p->fused_stamps ? ws.f_stamps : nullptr;
     if (launch_decode_fused(fa, p->sm_count, s, &p->launches) != cudaSuccess) {
+        // the grid did not fit the device at once (SMs taken away from this context, say): the
+        // kernel chain serves this and all later calls of the plan
         cudaGetLastError();
-        return MOE_ERR_CUDA;
+        p->fused_ok = false;
+        return MOE_ERR_NOT_IMPLEMENTED;
     }
     return MOE_OK;
 }
@@ -140,11 +143,13 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
     if (sched == MOE_SCHED_DECODE_FUSED && (mode == 0 || mode == 1)) {
         mark(1); mark(2);                 // the whole call is booked under the first GEMM stage
         const int rc = fused_layer(p, x, w, T, k, renorm, y, mode, s);
-        if (rc != MOE_OK) return rc;
-        mark(3); mark(4); mark(5);
-        p->last_T = T;
-        p->last_k = k;
-        return MOE_OK;
+        if (rc == MOE_OK) {
+            mark(3); mark(4); mark(5);
+            p->last_T = T;
+            p->last_k = k;
+            return MOE_OK;
+        }
+        if (rc != MOE_ERR_NOT_IMPLEMENTED) return rc;
     }
     if (sched == MOE_SCHED_DECODE_FUSED) sched = MOE_SCHED_DECODE;     // Stage-1 profiling needs the slot outputs
     // small decode calls: one fused front-end launch, and the gate/up GEMM reads x directly

@@ -257,7 +257,7 @@ def test_pruning_shaped_qwen_layers(kind, frac, T):
         check_layer(plan, x, w, 2, False, shared_gate=True, tokens=toks, w_host=w_host)
 
 
-@pytest.mark.parametrize("T,k", [(1, 2), (16, 1), (256, 2), (4096, 2)])
+@pytest.mark.parametrize("T,k", [(1, 2), (16, 1), (256, 2), (4096, 2), (16384, 1)])
 def test_mixtral_shaped_layer(T, k):
     """d=4096, E=8, I=14336, renormalised gates; 16 sampled tokens."""
     wl = synth.WORKLOADS["mixtral"]
@@ -297,6 +297,23 @@ def test_one_launch_layer_for_at_most_8_tokens(name, T, k, renorm):
         c = plan.layer_forward(x, ws, k, renorm)
         rms = float(c.float().pow(2).mean().sqrt())
         assert float((a.float() - c.float()).abs().max()) <= 4e-2 * rms
+
+
+def test_one_launch_layer_time_stamps_are_ordered():
+    """Debug hook: the eight per-CTA stamps of a stamped call never run backwards, and the spread of
+    the start stamps shows all CTAs of the cooperative grid running at once."""
+    wl = synth.WORKLOADS["qwen15"]
+    w = B.make_weights(synth.make_layer(wl, 0, torch.bfloat16, DEV))
+    x = synth.make_tokens(wl, 4, torch.bfloat16, DEV)
+    with _plan(wl, 8, 4, torch.bfloat16) as plan:
+        B.moe_debug_fused_stamps(plan.handle, True)
+        plan.layer_forward(x, w, 4, False)
+        st = np.array(B.moe_debug_fused_stamps(plan.handle, False, read=True), dtype=np.int64)
+        assert plan.device_status() == 0
+    assert st.shape[1] == 8 and st.shape[0] >= 1
+    assert np.all(np.diff(st, axis=1) >= 0)
+    assert st[:, 0].max() - st[:, 0].min() < 1_000_000          # all CTAs started within a millisecond
+    assert st[:, 7].max() - st[:, 0].min() < 50_000_000
 
 
 def test_one_launch_layers_chained_in_a_stack():
