@@ -158,6 +158,26 @@ int moe_layer_forward_host(moe_plan_t *plan, const void *x_host, const moe_layer
                            void *cuda_stream);
 
 /*
+ * Pipelined host-buffer calls, for callers that feed one batch after another from HOST memory
+ * (a serving loop): moe_host_pipeline_submit enqueues the upload of x_host, the layer and the
+ * download into y_host on three streams of the plan and returns at once with a ticket; up to two
+ * submissions are in flight (two pairs of staging buffers), so the upload of batch i+1 and the
+ * download of batch i-1 run beside the kernels of batch i.  A third submission first waits, on the
+ * host, for the download two tickets back.  moe_host_pipeline_wait(ticket) returns once that
+ * ticket's y_host is complete.  Tickets count up from 0 per plan.
+ *   x_host [T, d], y_host [T, d]: host memory (pinned for asynchronous copies), the caller's;
+ *   x_host must hold its data when submit is called and both must stay untouched until the
+ *   ticket has been waited for.  The weights must not change while tickets are in flight, and
+ *   no other call may use the plan meanwhile (the workspace is shared).  The second staging pair
+ *   (2 * max_T * d elements) and the streams are created by the first submission.
+ * Every batch is the layer call of moe_layer_forward (same schedule choice, same bits).
+ * Errors: INVALID_ARG, ALIGN, WORKSPACE, CUDA.
+ */
+int moe_host_pipeline_submit(moe_plan_t *plan, const void *x_host, const moe_layer_weights_t *w,
+                             int32_t T, int32_t k_l, int32_t renorm, void *y_host, int64_t *ticket);
+int moe_host_pipeline_wait(moe_plan_t *plan, int64_t ticket);
+
+/*
  * moe_stack_forward: L MoE modules in sequence, layer l with k_vec[l] active experts -
  * the deployment form of the allocation k* that Algorithm 2 returns:
  *

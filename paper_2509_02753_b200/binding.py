@@ -29,7 +29,7 @@ EXPORTS = (
     "moe_route_from_logits", "moe_last_routing", "moe_device_status", "moe_plan_launch_count",
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
     "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts",
-    "moe_debug_fused_stamps",
+    "moe_debug_fused_stamps", "moe_host_pipeline_submit", "moe_host_pipeline_wait",
     "moe_debug_wait_timeout", "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
@@ -85,6 +85,8 @@ def load_library() -> ctypes.CDLL:
     lib.moe_last_residual_f32.argtypes = [vp, vp, i32, vp]
     lib.moe_plan_touched_experts.argtypes = [vp, P(ctypes.c_int64), vp]
     lib.moe_debug_fused_stamps.argtypes = [vp, i32, P(ctypes.c_uint64), i32, P(i32), vp]
+    lib.moe_host_pipeline_submit.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, vp, P(ctypes.c_int64)]
+    lib.moe_host_pipeline_wait.argtypes = [vp, ctypes.c_int64]
     lib.moe_profile_layer.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, P(ctypes.c_double),
                                       P(ctypes.c_double), vp]
     dbl_p, i32_p = P(ctypes.c_double), P(i32)
@@ -191,6 +193,22 @@ def moe_layer_forward_host(plan: int, x_host: torch.Tensor, w: moe_layer_weights
            load_library().moe_layer_forward_host(plan, x_host.data_ptr(), ctypes.byref(w),
                                                  x_host.shape[0], k_l, int(renorm),
                                                  y_host.data_ptr(), _stream(stream)))
+
+
+def moe_host_pipeline_submit(plan: int, x_host: torch.Tensor, w: moe_layer_weights_t, k_l: int,
+                             renorm: bool, y_host: torch.Tensor) -> int:
+    """Enqueues upload, layer and download of one host-resident batch; returns its ticket."""
+    assert not x_host.is_cuda and not y_host.is_cuda
+    assert x_host.is_contiguous() and y_host.is_contiguous()
+    t = ctypes.c_int64()
+    _check("moe_host_pipeline_submit",
+           load_library().moe_host_pipeline_submit(plan, x_host.data_ptr(), ctypes.byref(w), x_host.shape[0],
+                                                   k_l, int(renorm), y_host.data_ptr(), ctypes.byref(t)))
+    return int(t.value)
+
+
+def moe_host_pipeline_wait(plan: int, ticket: int) -> None:
+    _check("moe_host_pipeline_wait", load_library().moe_host_pipeline_wait(plan, ticket))
 
 
 def moe_stack_forward(plan: int, h: torch.Tensor, layers: Sequence[moe_layer_weights_t],

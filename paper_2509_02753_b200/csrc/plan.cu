@@ -24,6 +24,14 @@ struct moe_plan {
     // host-buffer entry point: copy streams and events of its token-chunk pipeline
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_start = nullptr, ev_out = nullptr, ev_in[4] = {}, ev_done[4] = {};
+    // pipelined host-buffer calls (moe_host_pipeline_*): two slots of staging buffers, three streams
+    struct HostPipe {
+        bool ready = false;
+        cudaStream_t compute = nullptr, in = nullptr, out = nullptr;
+        void *x_stage[2] = {nullptr, nullptr}, *y_stage[2] = {nullptr, nullptr};
+        cudaEvent_t ev_in[2] = {}, ev_done[2] = {}, ev_out[2] = {};
+        int64_t submitted = 0;
+    } pipe;
     int sm_count = 148;
     bool use_tc_router = true;   // cleared by MOE_SCHED_SIMT so that schedule stays tensor-core free
     bool use_direct = true;      // fused front end + direct-x gate/up GEMM for small decode calls
@@ -346,6 +354,13 @@ int moe_plan_destroy(moe_plan_t *p) {
     for (void *q : p->allocs) cudaFree(q);
     for (cudaEvent_t e : p->events) cudaEventDestroy(e);
     if (p->status_host) cudaFreeHost(p->status_host);
+    if (p->pipe.ready) {
+        cudaStreamDestroy(p->pipe.compute); cudaStreamDestroy(p->pipe.in); cudaStreamDestroy(p->pipe.out);
+        for (int b = 0; b < 2; ++b) {
+            cudaEventDestroy(p->pipe.ev_in[b]); cudaEventDestroy(p->pipe.ev_done[b]); cudaEventDestroy(p->pipe.ev_out[b]);
+        }
+        cudaFree(p->pipe.x_stage[1]); cudaFree(p->pipe.y_stage[1]);     // slot 0 is the plan's own staging pair
+    }
     if (p->copy_in) cudaStreamDestroy(p->copy_in);
     if (p->copy_out) cudaStreamDestroy(p->copy_out);
     if (p->ev_start) cudaEventDestroy(p->ev_start);
@@ -483,6 +498,55 @@ int moe_layer_forward_host(moe_plan_t *p, const void *x_host, const moe_layer_we
     ok = ok && cudaEventRecord(p->ev_out, p->copy_out) == cudaSuccess &&
          cudaStreamWaitEvent(s, p->ev_out, 0) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    return MOE_OK;
+}
+
+int moe_host_pipeline_submit(moe_plan_t *p, const void *x_host, const moe_layer_weights_t *w, int32_t T,
+                             int32_t k_l, int32_t renorm, void *y_host, int64_t *ticket) {
+    if (!p || !x_host || !y_host || !ticket) return MOE_ERR_INVALID_ARG;
+    if (T < 1 || T > p->cfg.max_T || k_l < 1 || k_l > p->cfg.max_k) return MOE_ERR_INVALID_ARG;
+    int rc = check_weights(p, w);
+    if (rc != MOE_OK) return rc;
+    moe_plan::HostPipe &hp = p->pipe;
+    const size_t row_bytes = (size_t)p->cfg.d * elem_size(p->cfg.dtype);
+    if (!hp.ready) {                 // first submission: streams, events, the second staging pair
+        const size_t bytes = (size_t)p->cfg.max_T * row_bytes;
+        bool ok = cudaStreamCreateWithFlags(&hp.compute, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess;
+        for (int b = 0; ok && b < 2; ++b)
+            ok = cudaEventCreateWithFlags(&hp.ev_in[b], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.ev_done[b], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.ev_out[b], cudaEventDisableTiming) == cudaSuccess;
+        hp.x_stage[0] = p->ws.x_stage; hp.y_stage[0] = p->ws.y_stage;
+        ok = ok && cudaMalloc(&hp.x_stage[1], bytes) == cudaSuccess && cudaMalloc(&hp.y_stage[1], bytes) == cudaSuccess;
+        if (!ok) { cudaGetLastError(); return MOE_ERR_WORKSPACE; }
+        p->bytes += 2 * bytes;
+        hp.ready = true;
+    }
+    const int b = (int)(hp.submitted & 1);
+    // the slot's previous user (two submissions ago) must have delivered its result
+    if (hp.submitted >= 2 && cudaEventSynchronize(hp.ev_out[b]) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    const size_t bytes = (size_t)T * row_bytes;
+    bool ok = cudaMemcpyAsync(hp.x_stage[b], x_host, bytes, cudaMemcpyHostToDevice, hp.in) == cudaSuccess &&
+              cudaEventRecord(hp.ev_in[b], hp.in) == cudaSuccess &&
+              cudaStreamWaitEvent(hp.compute, hp.ev_in[b], 0) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    rc = layer_impl(p, hp.x_stage[b], w, T, k_l, renorm ? 1 : 0, hp.y_stage[b], 0, hp.compute);
+    if (rc != MOE_OK) return rc;
+    ok = cudaEventRecord(hp.ev_done[b], hp.compute) == cudaSuccess &&
+         cudaStreamWaitEvent(hp.out, hp.ev_done[b], 0) == cudaSuccess &&
+         cudaMemcpyAsync(y_host, hp.y_stage[b], bytes, cudaMemcpyDeviceToHost, hp.out) == cudaSuccess &&
+         cudaEventRecord(hp.ev_out[b], hp.out) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    *ticket = hp.submitted++;
+    return MOE_OK;
+}
+
+int moe_host_pipeline_wait(moe_plan_t *p, int64_t ticket) {
+    if (!p || ticket < 0 || !p->pipe.ready || ticket >= p->pipe.submitted) return MOE_ERR_INVALID_ARG;
+    if (ticket + 2 < p->pipe.submitted) return MOE_OK;      // its slot was reused: that submission waited for it
+    if (cudaEventSynchronize(p->pipe.ev_out[ticket & 1]) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
     return MOE_OK;
 }
 

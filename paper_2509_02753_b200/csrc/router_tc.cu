@@ -4,6 +4,9 @@
 //
 // Tile: 128 tokens (UMMA M) x 64 columns (UMMA N): columns 0..E-1 are the experts, column E is the
 // shared expert's gate vector w_s when the layer has one (so E + gate <= 64).  K = d in chunks of 64.
+// While 128-token tiles would leave SMs without a tile (T < 128 x SMs), tiles are 64 tokens (UMMA
+// M = 64: token 16 q + l of a tile sits in lane l < 16 of TMEM lane quarter q), so twice as many CTAs
+// share the reading of x.
 // Same role split as the expert GEMMs: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 epilogue with
 // two TMEM buffers.  Selection semantics equal the warp-shuffle router: fp32 logits (+ bias), larger
 // first, equal logits -> lower index; all waits are bounded.
@@ -25,6 +28,7 @@ constexpr int kRSmem = kRStages * (kRABytes + kRBBytes) + 1024 + 256;
 
 struct RouterTcParams {
     int T, d, E, k, renorm, has_gate;
+    int tile_m;            // tokens per tile: 128 or 64
     const float *bias;
     float *logits; int32_t *topk_idx; float *topk_w; float *gamma;
     int32_t *status;
@@ -34,7 +38,7 @@ __global__ void __launch_bounds__(192, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const __grid_constant__ CUtensorMap map_ws, const RouterTcParams p) {
     pdl_trigger();
-    const int n_tiles = (p.T + 127) / 128;
+    const int n_tiles = (p.T + p.tile_m - 1) / p.tile_m;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -67,7 +71,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (lane == 0) {
             // W_g is loaded with a box of exactly E rows and w_s as one more row behind it; rows
             // beyond are never written and only feed logit columns that are never read
-            const uint32_t tx = kRABytes + (uint32_t)p.E * 128u + (p.has_gate ? 128u : 0u);
+            const uint32_t tx = (uint32_t)p.tile_m * 128u + (uint32_t)p.E * 128u + (p.has_gate ? 128u : 0u);
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
@@ -76,7 +80,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     const uint32_t ph = (it / kRStages) & 1u;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, p.status)) { ok = false; break; }
                     mbar_expect_tx(full_bar(s), tx);
-                    tma_load_3d(a_base + s * kRABytes, &map_x, full_bar(s), kc * kBK, tile * 128, 0);
+                    tma_load_3d(a_base + s * kRABytes, &map_x, full_bar(s), kc * kBK, tile * p.tile_m, 0);
                     tma_load_3d(b_base + s * kRBBytes, &map_w, full_bar(s), kc * kBK, 0, 0);
                     if (p.has_gate)
                         tma_load_3d(b_base + s * kRBBytes + p.E * 128, &map_ws, full_bar(s), kc * kBK, 0, 0);
@@ -85,7 +89,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(kRN);
+            const uint32_t idesc = p.tile_m == 64 ? make_idesc_bf16_m(64, kRN) : make_idesc_bf16(kRN);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++tcount) {
@@ -110,7 +114,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         }
     } else {
         const int q = warp & 3;
-        const int row_in_tile = q * 32 + lane;
+        // M = 128: lane = row.  M = 64: row 16 q + l lives in lane l < 16 of quarter q.
+        const int row_in_tile = p.tile_m == 64 ? (lane < 16 ? q * 16 + lane : 1 << 20) : q * 32 + lane;
         uint32_t tcount = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
             const uint32_t buf = tcount & 1u, bph = (tcount >> 1) & 1u;
@@ -131,8 +136,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             tc_fence_before();
             mbar_arrive(tempty_bar(buf));
 
-            const int t = tile * 128 + row_in_tile;
-            if (t < p.T) {
+            const int t = tile * p.tile_m + row_in_tile;
+            if (row_in_tile < p.tile_m && t < p.T) {
                 float gate_logit = 0.f;
                 float m = -CUDART_INF_F;
 #pragma unroll
@@ -204,7 +209,8 @@ bool tc_router_supported(const TcState *st, const RouterArgs &a) {
 cudaError_t launch_router_tc(const TcState *st, const RouterArgs &a, int sm_count, cudaStream_t s,
                              uint64_t *launches) {
     CUtensorMap mx, mw, mg;
-    bool ok = tc_encode_bf16_map(st, &mx, a.x, a.d, a.T, 1, 128);
+    const int tile_m = (a.T + 127) / 128 >= sm_count ? 128 : 64;
+    bool ok = tc_encode_bf16_map(st, &mx, a.x, a.d, a.T, 1, tile_m);
     ok = ok && tc_encode_bf16_map(st, &mw, a.W, a.d, a.E, 1, a.E);
     ok = ok && tc_encode_bf16_map(st, &mg, a.w_s ? a.w_s : a.W, a.d, 1, 1, 1);
     if (!ok) return cudaErrorInvalidValue;
@@ -214,9 +220,9 @@ cudaError_t launch_router_tc(const TcState *st, const RouterArgs &a, int sm_coun
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    RouterTcParams p{a.T, a.d, a.E, a.k, a.renorm, a.w_s ? 1 : 0, a.bias,
+    RouterTcParams p{a.T, a.d, a.E, a.k, a.renorm, a.w_s ? 1 : 0, tile_m, a.bias,
                      a.logits, a.topk_idx, a.topk_w, a.gamma, a.status};
-    const int n_tiles = (a.T + 127) / 128;
+    const int n_tiles = (a.T + tile_m - 1) / tile_m;
     const int grid = n_tiles < sm_count ? n_tiles : sm_count;
     const cudaError_t e = launch_chained(router_tc_kernel, dim3(grid), dim3(192), (size_t)kRSmem, s, a.chained,
                                          mx, mw, mg, p);

@@ -64,6 +64,17 @@ WORKLOADS: Dict[str, Workload] = {
     "mixtral": Workload("mixtral", d=4096, E=8, I=14336, k_base=2, L=32, renorm=True, residual_init=True,
                         k_lo=1, k_hi=2, k_budget=48, T_decode=(1, 16, 256),
                         T_prefill=(4096, 16384)),
+    # The two remaining models of Table 1.  The paper prints layers, experts, top-k and FFN size but
+    # NO hidden size for them: d below is an ASSUMPTION (the hidden sizes of the public MiniCPM-2B
+    # and DeepSeek-VL2-Tiny model cards), as are the shared experts of the DeepSeek shape.
+    # MiniCPM-MoE-8x2B-shaped stack: 40 layers, 8 experts, top-2, budget 60 (one the paper evaluates)
+    "minicpm": Workload("minicpm", d=2304, E=8, I=5760, k_base=2, L=40, renorm=True, residual_init=True,
+                        k_lo=1, k_hi=2, k_budget=60, T_decode=(1, 16), T_prefill=(4096,)),
+    # DeepSeek-VL2-Tiny-shaped stack: 12 layers, 64 experts, top-6, two ungated shared experts of 896
+    # (held as one of 1792), budget 48
+    "dsvl2tiny": Workload("dsvl2tiny", d=1280, E=64, I=896, k_base=6, L=12, I_shared=1792,
+                          shared_gate=False, renorm=False, router_bias_std=0.5, residual_init=True,
+                          k_lo=2, k_hi=6, k_budget=48, T_decode=(1, 64), T_prefill=(4096,)),
 }
 
 

@@ -22,12 +22,17 @@ def _table1():
 def test_workload_shapes_match_table1():
     t = _table1()
     pairs = {"qwen15": "Qwen1.5-MoE-A2.7B", "olmoe": "OLMoE-1B-7B",
-             "dsv2lite": "DeepSeek-V2-Lite", "mixtral": "Mixtral-8x7B"}
+             "dsv2lite": "DeepSeek-V2-Lite", "mixtral": "Mixtral-8x7B",
+             "minicpm": "MiniCPM-MoE-8x2B", "dsvl2tiny": "DeepSeekVL2-Tiny"}
     for wl_name, paper_name in pairs.items():
         wl, row = synth.WORKLOADS[wl_name], t[paper_name]
         assert (wl.E, wl.k_base, wl.I) == (row["E"], row["k"], row["I"])
     assert synth.WORKLOADS["olmoe"].L == t["OLMoE-1B-7B"]["L"]
     assert synth.WORKLOADS["mixtral"].L == t["Mixtral-8x7B"]["L"]
+    assert synth.WORKLOADS["minicpm"].L == t["MiniCPM-MoE-8x2B"]["L"]
+    assert synth.WORKLOADS["dsvl2tiny"].L == t["DeepSeekVL2-Tiny"]["L"]
+    assert synth.WORKLOADS["minicpm"].k_budget in t["MiniCPM-MoE-8x2B"]["budgets"]
+    assert synth.WORKLOADS["dsvl2tiny"].k_budget in t["DeepSeekVL2-Tiny"]["budgets"]
     # DeepSeek-V2-Lite: 27 layers in the table, but its budgets are multiples of 26: first layer dense
     assert all(b % 26 == 0 for b in t["DeepSeek-V2-Lite"]["budgets"])
     assert synth.WORKLOADS["dsv2lite"].L == t["DeepSeek-V2-Lite"]["L"] - 1
@@ -37,7 +42,7 @@ def test_workload_shapes_match_table1():
 
 
 def test_k_vectors_meet_range_and_budget():
-    for name in ("olmoe", "dsv2lite", "mixtral", "qwen15", "tiny"):
+    for name in ("olmoe", "dsv2lite", "mixtral", "qwen15", "tiny", "minicpm", "dsvl2tiny"):
         wl = synth.WORKLOADS[name]
         k = synth.make_k_vector(wl, seed=0)
         assert len(k) == wl.L and sum(k) == wl.k_budget
