@@ -136,13 +136,17 @@ def _dtype_code(dtype: torch.dtype) -> int:
 
 
 def make_weights(w: Dict[str, Optional[torch.Tensor]]) -> moe_layer_weights_t:
-    """Packs a dict of contiguous CUDA tensors (keys as in ``moe_layer_weights_t``)."""
+    """Packs a dict of contiguous CUDA tensors (keys as in ``moe_layer_weights_t``).  The struct
+    holds raw pointers; the tensors are kept alive for as long as the returned object lives."""
     s = moe_layer_weights_t()
+    keep = []
     for name, _ in moe_layer_weights_t._fields_:
         t = w.get(name)
         if t is not None:
             assert t.is_cuda and t.is_contiguous(), name
+            keep.append(t)
         setattr(s, name, _ptr(t))
+    s._keepalive = keep
     return s
 
 
