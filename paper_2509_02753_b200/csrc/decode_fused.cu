@@ -756,8 +756,14 @@ size_t fused_smem_bytes(int d) {
 }
 
 cudaError_t fused_prepare(int d) {
-    return cudaFuncSetAttribute(decode_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)fused_smem_bytes(d));
+    // the attribute belongs to the kernel, not to a plan: it only ever grows, so that plans of
+    // different hidden sizes can live side by side
+    static int granted = 0;
+    const int need = (int)fused_smem_bytes(d);
+    if (need <= granted) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(decode_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, need);
+    if (e == cudaSuccess) granted = need;
+    return e;
 }
 
 cudaError_t launch_decode_fused(const FusedArgs &a, int sm_count, cudaStream_t s, uint64_t *launches) {

@@ -343,6 +343,23 @@ def test_one_launch_layer_for_at_most_8_tokens(name, T, k, renorm):
         assert float((a.float() - c.float()).abs().max()) <= 4e-2 * rms
 
 
+@pytest.mark.parametrize("d,E,I,I_s,gate,k,T", [(256, 128, 64, 0, False, 9, 8), (256, 127, 64, 96, True, 127, 2),
+                                               (4096, 8, 96, 0, False, 1, 7), (64, 3, 64, 96, False, 3, 8)])
+def test_one_launch_layer_on_extreme_shapes(d, E, I, I_s, gate, k, T):
+    """128 experts (eight 16-row router blocks, up to 64 touched experts), k = E, the smallest sizes the
+    kernel takes (two 32-element segments in its only chunk), a hidden size of 4096 with a tiny expert; two
+    plans of different hidden size alive at once."""
+    wl = _custom("fx", d=d, E=E, I=I, I_shared=I_s, shared_gate=gate, bias=0.3, k_base=k)
+    w, x, w_host = _small(wl, T, torch.bfloat16)
+    other = _custom("fy", d=512, E=4, I=64)
+    wo, xo, wo_host = _small(other, 3, torch.bfloat16)
+    with _plan(wl, 8, k, torch.bfloat16) as plan, _plan(other, 8, 2, torch.bfloat16) as plan2:
+        assert plan.schedule_for(T, k) == B.MOE_SCHED_DECODE_FUSED
+        check_layer(plan, x, w, k, True, shared_gate=gate, w_host=w_host)
+        check_layer(plan2, xo, wo, 2, False, w_host=wo_host)
+        check_layer(plan, x, w, max(1, k // 2), False, shared_gate=gate, w_host=w_host)
+
+
 def test_one_launch_layer_time_stamps_are_ordered():
     """Debug hook: the eight per-CTA stamps of a stamped call never run backwards, and the spread of
     the start stamps shows all CTAs of the cooperative grid running at once."""
