@@ -42,6 +42,8 @@ constexpr int kMaxPairsF = kFT * kMaxExperts;
 constexpr unsigned long long kBarrierLimitNs = 1000000000ull;
 constexpr uint32_t kPrefetchChunks = 4;  // chunks of its down-stream share a warp asks for ahead of the barrier
 
+static_assert(kFusedThreads >= kMaxExperts, "one thread per expert stages the router bias");
+
 enum { kPhShared1 = 0, kPhRouted1 = 1, kPh2 = 2 };
 
 struct FusedSmem {
@@ -509,6 +511,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_fused_kernel(const Fu
         }
     }
 
+    // router bias of expert tid: asked for before x is staged, like the gate vector
+    const float bias_v = (a.router_bias != nullptr && tid < E) ? a.router_bias[tid] : 0.f;
+
     // ---- x -> shared memory (rows >= T and the padding are zero)
     {
         const int vec_per_row = xstride / 8;
@@ -531,9 +536,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_fused_kernel(const Fu
         }
         if (tid == 0) sm.abort = 0;
         for (int i = tid; i < kFusedMaxCtaBlocks; i += kFusedThreads) sm.wticket[i] = 0;
-        for (int e = tid; e < kMaxExperts; e += kFusedThreads) {
-            sm.tokmask[e] = 0;
-            sm.bias[e] = (a.router_bias != nullptr && e < E) ? a.router_bias[e] : 0.f;
+        if (tid < kMaxExperts) {
+            sm.tokmask[tid] = 0;
+            sm.bias[tid] = bias_v;
         }
     }
     __syncthreads();
