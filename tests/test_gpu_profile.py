@@ -46,10 +46,11 @@ def test_profile_tiny_layer(dtype, renorm):
     _case(synth.WORKLOADS["tiny"], 64, dtype, 2, renorm)
 
 
-@pytest.mark.parametrize("T,sched", [(24, None), (300, B.MOE_SCHED_PREFILL), (300, B.MOE_SCHED_DECODE),
+@pytest.mark.parametrize("T,sched", [(6, None), (24, None), (300, B.MOE_SCHED_PREFILL), (300, B.MOE_SCHED_DECODE),
                                      (300, B.MOE_SCHED_SIMT)])
 @pytest.mark.parametrize("renorm", [True, False])
 def test_profile_with_shared_expert_and_six_slots(T, sched, renorm):
+    """T = 6 would be a one-launch layer call; profiling needs the slot outputs, so it runs the chain."""
     wl = synth.Workload("prof", d=256, E=16, I=256, k_base=6, L=1, I_shared=256, shared_gate=True,
                         router_bias_std=0.3)
     _case(wl, T, torch.bfloat16, 6, renorm, sched)
