@@ -170,8 +170,9 @@ int moe_layer_forward_host(moe_plan_t *plan, const void *x_host, const moe_layer
  *   ticket has been waited for.  The weights must not change while tickets are in flight, and
  *   no other call may use the plan meanwhile (the workspace is shared).  The second staging pair
  *   (2 * max_T * d elements) and the streams are created by the first submission.
- * Every batch is the layer call of moe_layer_forward (same schedule choice, same bits).
- * Errors: INVALID_ARG, ALIGN, WORKSPACE, CUDA.
+ * Every batch is the layer call of moe_layer_forward (same schedule choice, same bits);
+ * 1 <= T <= max_T.  moe_host_pipeline_wait accepts any ticket already handed out.
+ * Errors: INVALID_ARG (also a ticket never issued), ALIGN (weights), WORKSPACE, CUDA.
  */
 int moe_host_pipeline_submit(moe_plan_t *plan, const void *x_host, const moe_layer_weights_t *w,
                              int32_t T, int32_t k_l, int32_t renorm, void *y_host, int64_t *ticket);
