@@ -360,6 +360,31 @@ def test_one_launch_layer_on_extreme_shapes(d, E, I, I_s, gate, k, T):
         check_layer(plan, x, w, max(1, k // 2), False, shared_gate=gate, w_host=w_host)
 
 
+def test_one_launch_layer_repeated_calls_leave_no_state_behind():
+    """300 calls with changing T, k and weights on one plan: arrival counters, the barrier counter and
+    the partial-sum slots are reused by every call, so any leftover shows up as a result that differs
+    from the same call on a fresh pass (bit for bit) or from the kernel chain (within the format)."""
+    wl = _custom("rep", d=512, E=16, I=256, I_shared=256, shared_gate=True, bias=0.4, k_base=6)
+    ws = [B.make_weights(synth.make_layer(wl, l, torch.bfloat16, DEV)) for l in range(3)]
+    g = torch.Generator().manual_seed(7)
+    cases = [(int(torch.randint(1, 9, (1,), generator=g)), int(torch.randint(1, 7, (1,), generator=g)),
+              int(torch.randint(0, 3, (1,), generator=g))) for _ in range(150)]
+    xs = {T: synth.make_tokens(wl, T, torch.bfloat16, DEV, seed=T) for T in range(1, 9)}
+    with _plan(wl, 8, 6, torch.bfloat16) as plan:
+        first = []
+        for T, k, l in cases:
+            assert plan.schedule_for(T, k) == B.MOE_SCHED_DECODE_FUSED
+            first.append(plan.layer_forward(xs[T], ws[l], k, False).clone())
+        for (T, k, l), y0 in zip(cases, first):                      # second pass: same bits
+            assert torch.equal(plan.layer_forward(xs[T], ws[l], k, False), y0)
+        assert plan.device_status() == 0
+        plan.set_schedule(B.MOE_SCHED_DECODE)
+        for (T, k, l), y0 in list(zip(cases, first))[::5]:
+            c = plan.layer_forward(xs[T], ws[l], k, False).float()
+            rms = float(c.pow(2).mean().sqrt())
+            assert float((y0.float() - c).abs().max()) <= 4e-2 * rms
+
+
 def test_one_launch_layer_time_stamps_are_ordered():
     """Debug hook: the eight per-CTA stamps of a stamped call never run backwards, and the spread of
     the start stamps shows all CTAs of the cooperative grid running at once."""
