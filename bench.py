@@ -460,6 +460,29 @@ def run_ours(args):
         torch.cuda.empty_cache()
         stacks = run_stacks(B, [n for n in args.stacks.split(",") if n], peaks, device, 50)
 
+    # ---- tokens/s against the number of active experts, one layer of every model shape (the axis
+    #      of the paper's Fig. 2): k = 1..k_base at the shape's largest decode and prefill sizes
+    k_sweep = []
+    if args.sweep and args.stacks and world == 1:
+        for name in [n for n in args.stacks.split(",") if n]:
+            wl_k = synth.WORKLOADS[name]
+            lay_k = [synth.make_layer(wl_k, l, dtype, device) for l in range(2)]
+            ws_k = [B.make_weights(w) for w in lay_k]
+            Ts_k = [max(wl_k.T_decode), max(wl_k.T_prefill)]
+            with B.MoEPlan(wl_k.d, wl_k.E, wl_k.I, max(Ts_k), wl_k.k_base, dtype, I_shared=wl_k.I_shared,
+                           shared_gate=wl_k.shared_gate) as plan_k:
+                for Tk in Ts_k:
+                    xk = synth.make_tokens(wl_k, Tk, dtype, device, seed=5)
+                    yk = torch.empty_like(xk)
+                    row = {"workload": name, "T": Tk, "tokens_per_s": {}}
+                    for kk in range(1, wl_k.k_base + 1):
+                        ms_k, _ = run_case(B, plan_k, wl_k, ws_k, xk, yk, kk, 10, 3, False)
+                        row["tokens_per_s"][str(kk)] = Tk / (ms_k / 10 * 1e-3)
+                    k_sweep.append(row)
+                assert plan_k.device_status() == 0
+            del lay_k, ws_k
+            torch.cuda.empty_cache()
+
     if rank == 0:
         line = {
             "metric": "MoE layer tokens/s at per-layer top-k", "value": value, "unit": "tokens/s",
@@ -475,7 +498,7 @@ def run_ours(args):
                        "reasons": clocks.get("reasons", []), "samples": clocks.get("samples", 0)},
             "e2e": e2e, "gpu_launches": gpu_launches,
             "roofline": roof, "cpu_baseline": cpu_baseline,
-            "layer": main, "sweep": sweep, "stacks": stacks, "stage1": stage1, "pruning_shapes": pruning,
+            "layer": main, "sweep": sweep, "k_sweep": k_sweep, "stacks": stacks, "stage1": stage1, "pruning_shapes": pruning,
             "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
                       "bf16_tflops_burst": peaks["bf16_tflops"], "source": peaks["source"],
                       "nominal_hbm_gbs": NOMINAL_HBM_GBS, "nominal_bf16_tflops": NOMINAL_BF16_TFLOPS},
