@@ -23,11 +23,13 @@
 // dimension; a lane loads 16 bytes of two weight rows straight from global memory into the A
 // fragment (the k order inside a 32-element segment is permuted identically for A and B, which a
 // dot product does not notice), so no shared-memory staging exists for weights.  The work of a
-// stream is a flat list of (16-row block, 128-column chunk) items cut into equal contiguous
-// ranges, one per warp of the grid; a row block whose chunks span several warps is summed through
-// per-warp partial slots and an arrival counter: the warp that arrives last adds the partials in
-// warp order (so the result does not depend on timing) and finishes the block.  Nothing spins
-// except the two grid barriers, whose waits are bounded in time.
+// stream is a flat list of (16-row block, 128-column chunk) items.  CTAs take equal contiguous
+// ranges of it (whole row blocks in the gate/up streams), the warps of a CTA equal contiguous
+// pieces of their CTA's range.  A row block whose chunks fall to several warps is summed through
+// shared-memory partial slots and an arrival counter: the warp that arrives last adds the partials
+// in warp order (so the result does not depend on timing) and finishes the block; a 16-row block
+// of y that falls to several CTAs meets the same way through global slots.  Nothing spins except
+// the two grid barriers, whose waits are bounded in time.
 #include "moe_internal.h"
 #include "router_common.cuh"
 
