@@ -460,6 +460,35 @@ def run_ours(args):
         torch.cuda.empty_cache()
         stacks = run_stacks(B, [n for n in args.stacks.split(",") if n], peaks, device, 50)
 
+    # ---- the decomposed calls that expert parallelism strings together (route/pack, local experts,
+    #      combine), timed as ONE rank that owns every expert: no exchange happens, so the figure shows
+    #      what the extra regrouping copies cost beside the one-call layer.  More than one GPU is not
+    #      available to this benchmark; the exchange itself is not measured.
+    expert_parallel = None
+    if args.sweep and world == 1:
+        from paper_2509_02753_b200 import expert_parallel as ep
+        layers_ep = synth.make_layer(wl, 0, dtype, device)
+        rk = ep.ExpertParallelLayer(wl.d, wl.E, wl.I, T, wl.k_base, dtype, layers_ep, 0, 1, I_shared=wl.I_shared,
+                                    shared_gate=wl.shared_gate)
+        def ep_call():
+            rows, counts, ctx = rk.pack(x, k, wl.renorm)
+            return rk.finish(ctx, rk.compute(rows, counts))
+        for _ in range(3):
+            ep_call()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(10):
+            ep_call()
+        e1.record()
+        torch.cuda.synchronize()
+        expert_parallel = {"ranks": 1, "T": T, "k": k, "ms_decomposed_calls": e0.elapsed_time(e1) / 10,
+                           "ms_layer_call": ms_per_step,
+                           "note": "one rank holding all experts (no exchange); expert parallelism over several "
+                                   "GPUs is checked for correctness only (ranks run in turn on one GPU, exchange over gloo)"}
+        rk.close()
+        del rk, layers_ep
+        torch.cuda.empty_cache()
+
     # ---- tokens/s against the number of active experts, one layer of every model shape (the axis
     #      of the paper's Fig. 2): k = 1..k_base at the shape's largest decode and prefill sizes
     k_sweep = []
@@ -498,7 +527,7 @@ def run_ours(args):
                        "reasons": clocks.get("reasons", []), "samples": clocks.get("samples", 0)},
             "e2e": e2e, "gpu_launches": gpu_launches,
             "roofline": roof, "cpu_baseline": cpu_baseline,
-            "layer": main, "sweep": sweep, "k_sweep": k_sweep, "stacks": stacks, "stage1": stage1, "pruning_shapes": pruning,
+            "layer": main, "sweep": sweep, "k_sweep": k_sweep, "expert_parallel": expert_parallel, "stacks": stacks, "stage1": stage1, "pruning_shapes": pruning,
             "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
                       "bf16_tflops_burst": peaks["bf16_tflops"], "source": peaks["source"],
                       "nominal_hbm_gbs": NOMINAL_HBM_GBS, "nominal_bf16_tflops": NOMINAL_BF16_TFLOPS},

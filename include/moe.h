@@ -158,6 +158,43 @@ int moe_layer_forward_host(moe_plan_t *plan, const void *x_host, const moe_layer
                            void *cuda_stream);
 
 /*
+ * The steps of moe_layer_forward one by one (Section 2: router, then the experts, then the gated
+ * sum), for callers that put something of their own between them - above all the token exchange
+ * of expert parallelism (the Introduction notes that inter-GPU communication grows with the
+ * number of active experts): route here, send each (token, slot) pair's row to the GPU that holds
+ * its expert, run that GPU's experts on what arrived, send the outputs back, combine here.
+ * paper_2509_02753_b200/expert_parallel.py drives exactly that.  All pointers are device memory,
+ * all calls asynchronous on the stream; the plan's workspace is used as by moe_layer_forward.
+ *
+ * moe_route: logits, TopK + Softmax (and the shared expert's gate sigmoid(x . w_s) of a gated plan),
+ *   then the dispatch tables.  Outputs (each may be NULL): topk_idx/topk_w [T, k_l], gamma [T],
+ *   counts [E], offsets [E + 1], perm [T * k_l] (pairs t * k_l + j in expert-major, token-ascending
+ *   order), inv_perm [T * k_l] (position of each pair in perm).  Only router_W, router_bias and w_s
+ *   of w are read.
+ * moe_gather_rows: dst[r, :] = src[row_index[r], :] for r < n_rows; rows of d elements of the
+ *   plan's dtype, or of fp32 when rows_f32 != 0 (expert outputs).
+ * moe_experts_forward: o_rows[r, :] = E_e(x_rows[r, :]) in fp32, for rows grouped by expert: the
+ *   first counts[0] rows belong to expert 0 of this plan, the next counts[1] to expert 1, ...;
+ *   n_rows = sum of counts <= max_T * max_k.  Only W_gate, W_up, W_down of w are read (a shared
+ *   expert is a plan of its own with E = 1).  bf16 plans run the tcgen05 prefill kernels (CTA pairs
+ *   from 64 rows per expert), fp32 plans the CUDA-core kernels.
+ * moe_combine: y[t] = routed_scale * sum_j topk_w[t, j] * o_rows[inv_perm[t * k_l + j]]
+ *   (+ gamma[t] * o_shared[t], gamma NULL = 1, when o_shared [T, d] fp32 is given), in slot order,
+ *   rounded once to the plan's dtype.
+ * Errors: INVALID_ARG, ALIGN, SHAPE, CUDA.
+ */
+int moe_route(moe_plan_t *plan, const void *x, const moe_layer_weights_t *w, int32_t T, int32_t k_l,
+              int32_t renorm, int32_t *topk_idx, float *topk_w, float *gamma, int32_t *counts,
+              int32_t *offsets, int32_t *perm, int32_t *inv_perm, void *cuda_stream);
+int moe_gather_rows(moe_plan_t *plan, const void *src, const int32_t *row_index, int32_t n_rows,
+                    int32_t rows_f32, void *dst, void *cuda_stream);
+int moe_experts_forward(moe_plan_t *plan, const void *x_rows, const int32_t *counts,
+                        const moe_layer_weights_t *w, int32_t n_rows, float *o_rows, void *cuda_stream);
+int moe_combine(moe_plan_t *plan, const float *o_rows, const float *topk_w, const int32_t *inv_perm,
+                const float *o_shared, const float *gamma, int32_t T, int32_t k_l, void *y,
+                void *cuda_stream);
+
+/*
  * Pipelined host-buffer calls, for callers that feed one batch after another from HOST memory
  * (a serving loop): moe_host_pipeline_submit enqueues the upload of x_host, the layer and the
  * download into y_host on three streams of the plan and returns at once with a ticket; up to two

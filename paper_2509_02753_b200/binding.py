@@ -30,6 +30,7 @@ EXPORTS = (
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
     "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts",
     "moe_debug_fused_stamps", "moe_host_pipeline_submit", "moe_host_pipeline_wait",
+    "moe_route", "moe_gather_rows", "moe_experts_forward", "moe_combine",
     "moe_debug_wait_timeout", "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
@@ -87,6 +88,10 @@ def load_library() -> ctypes.CDLL:
     lib.moe_debug_fused_stamps.argtypes = [vp, i32, P(ctypes.c_uint64), i32, P(i32), vp]
     lib.moe_host_pipeline_submit.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, vp, P(ctypes.c_int64)]
     lib.moe_host_pipeline_wait.argtypes = [vp, ctypes.c_int64]
+    lib.moe_route.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.moe_gather_rows.argtypes = [vp, vp, vp, i32, i32, vp, vp]
+    lib.moe_experts_forward.argtypes = [vp, vp, vp, P(moe_layer_weights_t), i32, vp, vp]
+    lib.moe_combine.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
     lib.moe_profile_layer.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, P(ctypes.c_double),
                                       P(ctypes.c_double), vp]
     dbl_p, i32_p = P(ctypes.c_double), P(i32)
@@ -197,6 +202,53 @@ def moe_layer_forward_host(plan: int, x_host: torch.Tensor, w: moe_layer_weights
            load_library().moe_layer_forward_host(plan, x_host.data_ptr(), ctypes.byref(w),
                                                  x_host.shape[0], k_l, int(renorm),
                                                  y_host.data_ptr(), _stream(stream)))
+
+
+def moe_route(plan: int, x: torch.Tensor, w: moe_layer_weights_t, k_l: int, renorm: bool, E: int, stream=None):
+    """Router + dispatch tables of one call.  Returns a dict of device tensors: topk_idx, topk_w,
+    gamma, counts, offsets, perm, inv_perm."""
+    T = x.shape[0]
+    i32, f32 = torch.int32, torch.float32
+    out = {"topk_idx": torch.empty((T, k_l), dtype=i32, device=x.device),
+           "topk_w": torch.empty((T, k_l), dtype=f32, device=x.device),
+           "gamma": torch.ones((T,), dtype=f32, device=x.device),
+           "counts": torch.empty((E,), dtype=i32, device=x.device),
+           "offsets": torch.empty((E + 1,), dtype=i32, device=x.device),
+           "perm": torch.empty((T * k_l,), dtype=i32, device=x.device),
+           "inv_perm": torch.empty((T * k_l,), dtype=i32, device=x.device)}
+    _check("moe_route", load_library().moe_route(
+        plan, x.data_ptr(), ctypes.byref(w), T, k_l, int(renorm), out["topk_idx"].data_ptr(),
+        out["topk_w"].data_ptr(), out["gamma"].data_ptr(), out["counts"].data_ptr(), out["offsets"].data_ptr(),
+        out["perm"].data_ptr(), out["inv_perm"].data_ptr(), _stream(stream)))
+    return out
+
+
+def moe_gather_rows(plan: int, src: torch.Tensor, row_index: torch.Tensor, dst: torch.Tensor, stream=None) -> None:
+    """dst[r] = src[row_index[r]]; rows of the plan's dtype, or fp32 rows when src is float32."""
+    assert src.is_cuda and src.is_contiguous() and dst.is_contiguous() and row_index.dtype == torch.int32
+    assert dst.shape[0] == row_index.shape[0] and src.dtype == dst.dtype
+    _check("moe_gather_rows", load_library().moe_gather_rows(
+        plan, src.data_ptr(), row_index.data_ptr(), row_index.shape[0], int(src.dtype == torch.float32),
+        dst.data_ptr(), _stream(stream)))
+
+
+def moe_experts_forward(plan: int, x_rows: torch.Tensor, counts: torch.Tensor, w: moe_layer_weights_t,
+                        o_rows: torch.Tensor, stream=None) -> None:
+    """o_rows[r] = E_e(x_rows[r]) (fp32) for rows grouped by expert as counts says."""
+    assert x_rows.is_cuda and x_rows.is_contiguous() and o_rows.dtype == torch.float32 and o_rows.is_contiguous()
+    assert counts.dtype == torch.int32 and counts.is_cuda
+    _check("moe_experts_forward", load_library().moe_experts_forward(
+        plan, x_rows.data_ptr(), counts.data_ptr(), ctypes.byref(w), x_rows.shape[0], o_rows.data_ptr(),
+        _stream(stream)))
+
+
+def moe_combine(plan: int, o_rows: torch.Tensor, topk_w: torch.Tensor, inv_perm: torch.Tensor, y: torch.Tensor,
+                o_shared: Optional[torch.Tensor] = None, gamma: Optional[torch.Tensor] = None, stream=None) -> None:
+    T, k_l = topk_w.shape
+    assert o_rows.dtype == torch.float32 and inv_perm.dtype == torch.int32 and topk_w.dtype == torch.float32
+    _check("moe_combine", load_library().moe_combine(
+        plan, o_rows.data_ptr(), topk_w.data_ptr(), inv_perm.data_ptr(), _ptr(o_shared), _ptr(gamma), T, k_l,
+        y.data_ptr(), _stream(stream)))
 
 
 def moe_host_pipeline_submit(plan: int, x_host: torch.Tensor, w: moe_layer_weights_t, k_l: int,

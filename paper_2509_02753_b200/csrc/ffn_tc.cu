@@ -777,7 +777,7 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
     bool ok = true;
     const void *dummy = a.x;   // maps of an absent shared expert are never dereferenced
     if (sc.direct) ok = ok && encode_map(st, &m1[0], a.x, a.d, a.T, 1, a_rows);   // every group reads x itself
-    else ok = ok && encode_map(st, &m1[0], a.x_perm, a.d, pairs_alloc + 128, 1, a_rows);
+    else ok = ok && encode_map(st, &m1[0], a.x_perm, a.d, a.x_perm_rows ? a.x_perm_rows : pairs_alloc + 128, 1, a_rows);
     ok = ok && encode_map(st, &m1[1], a.x, a.d, a.T, 1, a_rows);
     ok = ok && encode_map(st, &m1[2], a.W_gate, a.d, a.I, a.E, bn1 / 2);
     ok = ok && encode_map(st, &m1[3], a.W_up, a.d, a.I, a.E, bn1 / 2);

@@ -130,6 +130,7 @@ struct FfnArgs {
     bool chained;            // launch the GEMM kernels as programmatic dependents of their predecessors
     cudaEvent_t begin_event; // recorded right before the first GEMM phase when not null
     cudaEvent_t mid_event;   // recorded between the two GEMM phases when not null
+    size_t x_perm_rows = 0;  // rows that exist behind x_perm (0: the plan's own buffer, pairs + 128)
 };
 cudaError_t launch_ffn_simt(const FfnArgs &a, cudaStream_t s, uint64_t *launches);
 

@@ -228,6 +228,32 @@ int check_call(const moe_plan *p, const void *x, const moe_layer_weights_t *w, i
     return check_weights(p, w);
 }
 
+// offsets[e] = sum of counts[0..e), offsets[E] = total: one warp, 4 experts per lane
+__global__ void offsets_from_counts_kernel(const int32_t *counts, int32_t *offsets, int E) {
+    const int lane = threadIdx.x;
+    int c[kExpertsPerLane], sum = 0;
+#pragma unroll
+    for (int j = 0; j < kExpertsPerLane; ++j) {
+        const int e = lane * kExpertsPerLane + j;
+        c[j] = e < E ? counts[e] : 0;
+        sum += c[j];
+    }
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    int run = incl - sum;
+#pragma unroll
+    for (int j = 0; j < kExpertsPerLane; ++j) {
+        const int e = lane * kExpertsPerLane + j;
+        if (e < E) offsets[e] = run;
+        run += c[j];
+    }
+    if (lane == 31) offsets[E] = incl;
+}
+
 }  // namespace
 
 extern "C" {
@@ -498,6 +524,99 @@ int moe_layer_forward_host(moe_plan_t *p, const void *x_host, const moe_layer_we
     ok = ok && cudaEventRecord(p->ev_out, p->copy_out) == cudaSuccess &&
          cudaStreamWaitEvent(s, p->ev_out, 0) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    return MOE_OK;
+}
+
+int moe_route(moe_plan_t *p, const void *x, const moe_layer_weights_t *w, int32_t T, int32_t k_l, int32_t renorm,
+              int32_t *topk_idx, float *topk_w, float *gamma, int32_t *counts, int32_t *offsets, int32_t *perm,
+              int32_t *inv_perm, void *cuda_stream) {
+    if (!p || !x || !w || !w->router_W) return MOE_ERR_INVALID_ARG;
+    if (T < 0 || T > p->cfg.max_T || k_l < 1 || k_l > p->cfg.max_k) return MOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w->router_W)) return MOE_ERR_ALIGN;
+    if (T == 0) return MOE_OK;
+    const moe_config_t &c = p->cfg;
+    Workspace &ws = p->ws;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const bool gated = c.I_shared > 0 && c.shared_gate;
+    if (gated && !w->w_s) return MOE_ERR_INVALID_ARG;
+    RouterArgs ra{x, w->router_W, w->router_bias, gated ? w->w_s : nullptr, T, c.d, c.E, k_l, renorm ? 1 : 0, c.dtype,
+                  ws.logits, ws.topk_idx, ws.topk_w, ws.gamma, ws.status, false};
+    cudaError_t err;
+    if (T > 512 && p->use_tc_router && tc_router_supported(&p->tc, ra))
+        err = launch_router_tc(&p->tc, ra, p->sm_count, s, &p->launches);
+    else
+        err = launch_router(ra, s, &p->launches);
+    if (err != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    DispatchArgs da{ws.topk_idx, T, k_l, c.E, ws.counts, ws.offsets, ws.perm, ws.inv_perm, ws.part_hist, ws.status};
+    if (launch_dispatch(da, s, &p->launches) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    p->last_T = T;
+    p->last_k = k_l;
+    const size_t pairs = (size_t)T * k_l;
+    cudaError_t e = cudaSuccess;
+    if (inv_perm) e = cudaMemcpyAsync(inv_perm, ws.inv_perm, pairs * 4, cudaMemcpyDeviceToDevice, s);
+    if (e == cudaSuccess && gamma && gated) e = cudaMemcpyAsync(gamma, ws.gamma, (size_t)T * 4, cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    return moe_last_routing(p, topk_idx, topk_w, counts, offsets, perm, nullptr, cuda_stream);
+}
+
+int moe_gather_rows(moe_plan_t *p, const void *src, const int32_t *row_index, int32_t n_rows, int32_t rows_f32,
+                    void *dst, void *cuda_stream) {
+    if (!p || !src || !row_index || !dst || n_rows < 0) return MOE_ERR_INVALID_ARG;
+    if (!aligned16(src) || !aligned16(dst)) return MOE_ERR_ALIGN;
+    if (launch_gather(src, row_index, n_rows, 1, p->cfg.d, rows_f32 ? MOE_F32 : p->cfg.dtype, dst,
+                      (cudaStream_t)cuda_stream, &p->launches) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    return MOE_OK;
+}
+
+int moe_experts_forward(moe_plan_t *p, const void *x_rows, const int32_t *counts, const moe_layer_weights_t *w,
+                        int32_t n_rows, float *o_rows, void *cuda_stream) {
+    if (!p || !x_rows || !counts || !o_rows || !w || !w->W_gate || !w->W_up || !w->W_down) return MOE_ERR_INVALID_ARG;
+    const moe_config_t &c = p->cfg;
+    if (n_rows < 0 || (int64_t)n_rows > (int64_t)c.max_T * c.max_k) return MOE_ERR_INVALID_ARG;
+    if (!aligned16(x_rows) || !aligned16(o_rows) || !aligned16(w->W_gate) || !aligned16(w->W_up) || !aligned16(w->W_down))
+        return MOE_ERR_ALIGN;
+    if (n_rows == 0) return MOE_OK;
+    Workspace &ws = p->ws;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(ws.counts, counts, (size_t)c.E * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    offsets_from_counts_kernel<<<1, 32, 0, s>>>(ws.counts, ws.offsets, c.E);
+    ++p->launches;
+    // the rows are the (token, slot) pairs of a layer call that has T = n_rows tokens and one slot
+    FfnArgs fa{c.dtype, n_rows, 1, c.d, c.E, c.I, 0, ws.counts, ws.offsets, x_rows, x_rows,
+               w->W_gate, w->W_up, w->W_down, nullptr, nullptr, nullptr,
+               ws.h, ws.h_s, o_rows, ws.o_s, false, nullptr, nullptr};
+    fa.x_perm_rows = (size_t)n_rows;
+    if (c.dtype != MOE_BF16 || !tc_shape_ok(c) || p->forced_schedule == MOE_SCHED_SIMT) {
+        if (launch_ffn_simt(fa, s, &p->launches) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+        return MOE_OK;
+    }
+    // tensor-core kernels without split-K slabs, so that the outputs land in the caller's buffer
+    TcSchedule sc{};
+    tc_make_schedule(c, ws, fa, p->forced_schedule == MOE_SCHED_PREFILL_1CTA ? MOE_SCHED_PREFILL_1CTA : MOE_SCHED_PREFILL,
+                     false, p->sm_count, &sc);
+    TcOutputLayout lay{};
+    return tc_ffn_forward(&p->tc, c, ws, fa, sc, p->sm_count, s, &p->launches, &lay);
+}
+
+int moe_combine(moe_plan_t *p, const float *o_rows, const float *topk_w, const int32_t *inv_perm,
+                const float *o_shared, const float *gamma, int32_t T, int32_t k_l, void *y, void *cuda_stream) {
+    if (!p || !o_rows || !topk_w || !inv_perm || !y) return MOE_ERR_INVALID_ARG;
+    if (T < 0 || T > p->cfg.max_T || k_l < 1 || k_l > p->cfg.max_k) return MOE_ERR_INVALID_ARG;
+    if (!aligned16(o_rows) || !aligned16(y) || (o_shared && !aligned16(o_shared))) return MOE_ERR_ALIGN;
+    if (T == 0) return MOE_OK;
+    CombineArgs ca{};
+    ca.dtype = p->cfg.dtype; ca.T = T; ca.k = k_l; ca.d = p->cfg.d;
+    ca.topk_w = topk_w; ca.inv_perm = inv_perm; ca.gamma = o_shared ? gamma : nullptr;
+    ca.o = o_rows; ca.o_is_f32 = 1; ca.o_slabs = 1; ca.o_slab_stride = 0;
+    ca.o_s = o_shared; ca.os_slabs = 1; ca.os_slab_stride = 0;
+    ca.routed_scale = p->cfg.routed_scale; ca.y = y; ca.h_run = nullptr; ca.mode = 0; ca.chained = false;
+    if (launch_combine(ca, (cudaStream_t)cuda_stream, &p->launches) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
     return MOE_OK;
 }
 

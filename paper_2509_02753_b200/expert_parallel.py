@@ -1,0 +1,177 @@
+"""Expert parallelism: the experts of a layer spread over R GPUs, tokens exchanged all-to-all.
+
+The paper serves its models on several GPUs and notes (Introduction) that inter-GPU communication
+grows with the number of active experts; with the experts sharded, the rows that cross the links
+are the T * k_l (token, slot) pairs of a call, so a layer's own k_l cuts the exchange as it cuts
+the expert work.  Rank r holds the experts [r * E / R, (r + 1) * E / R) and the replicated router
+(and shared expert); one layer call on every rank is
+
+    pack     route the rank's own tokens (moe_route), gather their rows into expert order
+             (moe_gather_rows): the rows for rank 0 come first, then those for rank 1, ...
+    exchange pairs-per-(destination, expert) counts, then the rows, all-to-all
+    compute  regroup what arrived from source-major to expert-major order, run the local experts
+             (moe_experts_forward), put the outputs back into arrival order
+    exchange the fp32 outputs back, all-to-all
+    finish   gated sum over each token's slots plus the shared expert (moe_combine)
+
+Every arithmetic step is a kernel of the C library; this module holds the integer bookkeeping
+(which rows go where: `exchange_plan`, `regroup_index`) and the calls of torch.distributed.
+`pack` / `compute` / `finish` are separate methods so that a test can run R ranks in one process
+and move the rows by hand.
+
+Not run on more than one GPU here: the kernels between the exchanges are the single-GPU ones and
+are checked against the one-GPU layer by running the ranks one after the other on one device;
+the exchange itself is checked with CPU tensors over gloo.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Tuple
+
+import torch
+
+
+# ----------------------------------------------------------------------------- integer bookkeeping
+
+def exchange_plan(counts: torch.Tensor, world: int) -> Tuple[torch.Tensor, List[int]]:
+    """From this rank's pairs per GLOBAL expert (counts [E], expert-major order of the packed rows)
+    to what it sends: the matrix send_counts [world, E / world] (row r: pairs per local expert of
+    rank r) and the number of rows for each destination."""
+    E = counts.numel()
+    assert E % world == 0, "experts must divide evenly over the ranks"
+    send_counts = counts.reshape(world, E // world)
+    return send_counts, [int(v) for v in send_counts.sum(dim=1).tolist()]
+
+
+def regroup_index(recv_counts: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """recv_counts [world, E_loc]: rows that arrived from each source rank per local expert.  The
+    arrival buffer is source-major (all rows of source 0, then source 1, ...; inside a source the
+    experts ascend).  Returns (to_expert_major [n]: arrival index of the row that sits at each
+    position of the expert-major order, with the sources of an expert in rank order; its inverse
+    [n]; rows per local expert [E_loc])."""
+    world, e_loc = recv_counts.shape
+    c = recv_counts.to(torch.int64)
+    flat = c.reshape(-1)                                       # (source, expert) blocks in arrival order
+    start = torch.cumsum(flat, 0) - flat                       # arrival offset of each block
+    order = torch.arange(world * e_loc, device=c.device).reshape(world, e_loc).t().reshape(-1)   # (expert, source)
+    blk_len = flat[order]
+    blk_start = start[order]
+    n = int(flat.sum())
+    if n == 0:
+        z = torch.zeros((0,), dtype=torch.int32, device=c.device)
+        return z, z.clone(), c.sum(dim=0).to(torch.int32)
+    out_start = torch.cumsum(blk_len, 0) - blk_len              # position of each block in expert-major order
+    which = torch.repeat_interleave(torch.arange(order.numel(), device=c.device), blk_len)
+    pos = torch.arange(n, device=c.device)
+    to_expert_major = (blk_start[which] + (pos - out_start[which])).to(torch.int32)
+    inverse = torch.empty_like(to_expert_major)
+    inverse[to_expert_major.long()] = pos.to(torch.int32)
+    return to_expert_major, inverse, c.sum(dim=0).to(torch.int32)
+
+
+def exchange_rows(rows: torch.Tensor, send_splits: List[int], recv_splits: List[int], group=None) -> torch.Tensor:
+    """All-to-all of row blocks: block r of `rows` (send_splits[r] rows) goes to rank r; returns the
+    blocks received, in source order.  Works on whatever device the process group serves."""
+    import torch.distributed as dist
+    out = rows.new_empty((sum(recv_splits),) + tuple(rows.shape[1:]))
+    dist.all_to_all_single(out, rows.contiguous(), recv_splits, send_splits, group=group)
+    return out
+
+
+def exchange_counts(send_counts: torch.Tensor, group=None) -> torch.Tensor:
+    """send_counts [world, E_loc] -> recv_counts [world, E_loc] (row s: what source s sends here)."""
+    import torch.distributed as dist
+    out = torch.empty_like(send_counts)
+    dist.all_to_all_single(out, send_counts.contiguous(), group=group)
+    return out
+
+
+# ----------------------------------------------------------------------------- one rank's layer
+
+class ExpertParallelLayer:
+    """One rank of an expert-parallel MoE layer (see the module text).  ``weights`` is the dict of
+    the FULL layer's tensors on this rank's device (as `synth.make_layer` returns it); the rank
+    keeps views of its own experts' slices, the router and the shared expert."""
+
+    def __init__(self, d: int, E: int, I: int, max_T: int, max_k: int, dtype: torch.dtype,
+                 weights: Dict[str, Optional[torch.Tensor]], rank: int, world: int, *,
+                 I_shared: int = 0, shared_gate: bool = False, routed_scale: float = 1.0):
+        from . import binding as B
+        assert E % world == 0
+        self.B, self.d, self.E, self.I, self.dtype = B, d, E, I, dtype
+        self.rank, self.world, self.e_loc = rank, world, E // world
+        self.I_shared, self.shared_gate = I_shared, shared_gate
+        lo, hi = rank * self.e_loc, (rank + 1) * self.e_loc
+        # router and combine: a plan over all E experts (only its router, tables and combine are used)
+        self.router_plan = B.MoEPlan(d, E, I, max_T, max_k, dtype, I_shared=I_shared, shared_gate=shared_gate,
+                                     routed_scale=routed_scale)
+        # the local experts may receive every pair of every rank
+        self.local_plan = B.MoEPlan(d, self.e_loc, I, max_T * world, max_k, dtype)
+        self.shared_plan = B.MoEPlan(d, 1, I_shared, max_T, 1, dtype) if I_shared > 0 else None
+        self.w_router = B.make_weights({"router_W": weights["router_W"], "router_bias": weights.get("router_bias"),
+                                        "w_s": weights.get("w_s"),
+                                        # unused by moe_route, but a layer struct wants expert pointers
+                                        "W_gate": weights["W_gate"], "W_up": weights["W_up"], "W_down": weights["W_down"],
+                                        "Ws_gate": weights.get("Ws_gate"), "Ws_up": weights.get("Ws_up"),
+                                        "Ws_down": weights.get("Ws_down")})
+        self.w_local = B.make_weights({"router_W": weights["router_W"][lo:hi], "W_gate": weights["W_gate"][lo:hi],
+                                       "W_up": weights["W_up"][lo:hi], "W_down": weights["W_down"][lo:hi]})
+        self.w_shared = None
+        if I_shared > 0:
+            self.w_shared = B.make_weights({"router_W": weights["router_W"][:1],
+                                            "W_gate": weights["Ws_gate"].unsqueeze(0), "W_up": weights["Ws_up"].unsqueeze(0),
+                                            "W_down": weights["Ws_down"].unsqueeze(0)})
+
+    def close(self):
+        for p in (self.router_plan, self.local_plan, self.shared_plan):
+            if p is not None:
+                p.close()
+
+    # -- step 1: route the rank's tokens and lay their rows out by destination
+    def pack(self, x: torch.Tensor, k_l: int, renorm: bool):
+        B = self.B
+        r = B.moe_route(self.router_plan.handle, x, self.w_router, k_l, renorm, self.E)
+        row_index = torch.div(r["perm"], k_l, rounding_mode="floor").to(torch.int32)
+        send_rows = torch.empty((x.shape[0] * k_l, self.d), dtype=x.dtype, device=x.device)
+        B.moe_gather_rows(self.router_plan.handle, x, row_index, send_rows)
+        send_counts, send_splits = exchange_plan(r["counts"], self.world)
+        ctx = {"x": x, "route": r, "k": k_l, "send_splits": send_splits}
+        return send_rows, send_counts, ctx
+
+    # -- step 2: the local experts on what arrived (rows source-major), outputs in arrival order
+    def compute(self, recv_rows: torch.Tensor, recv_counts: torch.Tensor) -> torch.Tensor:
+        B = self.B
+        to_em, inverse, per_expert = regroup_index(recv_counts)
+        n = recv_rows.shape[0]
+        grouped = torch.empty_like(recv_rows)
+        out_em = torch.empty((n, self.d), dtype=torch.float32, device=recv_rows.device)
+        back = torch.empty_like(out_em)
+        if n > 0:
+            B.moe_gather_rows(self.local_plan.handle, recv_rows, to_em, grouped)
+            B.moe_experts_forward(self.local_plan.handle, grouped, per_expert.contiguous(), self.w_local, out_em)
+            B.moe_gather_rows(self.local_plan.handle, out_em, inverse, back)
+        return back
+
+    # -- step 3: gated sum of the returned outputs (rows in the order they were sent), shared expert
+    def finish(self, ctx, returned: torch.Tensor) -> torch.Tensor:
+        B = self.B
+        x, r = ctx["x"], ctx["route"]
+        T = x.shape[0]
+        y = torch.empty_like(x)
+        o_shared = None
+        if self.shared_plan is not None:
+            o_shared = torch.empty((T, self.d), dtype=torch.float32, device=x.device)
+            one = torch.tensor([T], dtype=torch.int32, device=x.device)
+            B.moe_experts_forward(self.shared_plan.handle, x, one, self.w_shared, o_shared)
+        B.moe_combine(self.router_plan.handle, returned, r["topk_w"], r["inv_perm"], y, o_shared,
+                      r["gamma"] if self.shared_gate else None)
+        return y
+
+    # -- the whole call over torch.distributed (one process per GPU, NCCL)
+    def forward(self, x: torch.Tensor, k_l: int, renorm: bool, group=None) -> torch.Tensor:
+        send_rows, send_counts, ctx = self.pack(x, k_l, renorm)
+        recv_counts = exchange_counts(send_counts, group)
+        recv_splits = [int(v) for v in recv_counts.sum(dim=1).tolist()]
+        recv_rows = exchange_rows(send_rows, ctx["send_splits"], recv_splits, group)
+        back = self.compute(recv_rows, recv_counts)
+        returned = exchange_rows(back, recv_splits, ctx["send_splits"], group)
+        return self.finish(ctx, returned)

@@ -1,0 +1,164 @@
+"""Expert parallelism: the integer bookkeeping against brute force (CPU), the all-to-all exchange
+over gloo with two processes (CPU), and the whole path with the ranks run one after the other on
+one GPU against the CPU oracle and the one-GPU layer."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2509_02753_b200 import expert_parallel as ep
+
+
+def _brute_regroup(recv_counts):
+    world, e_loc = recv_counts.shape
+    arrival = []                                   # (source, expert, i) in arrival order
+    for s in range(world):
+        for e in range(e_loc):
+            arrival += [(s, e, i) for i in range(int(recv_counts[s, e]))]
+    want = sorted(range(len(arrival)), key=lambda a: (arrival[a][1], arrival[a][0], arrival[a][2]))
+    return want
+
+
+def test_regroup_index_is_the_expert_major_order_and_its_inverse():
+    g = torch.Generator().manual_seed(3)
+    for world, e_loc in [(1, 4), (2, 3), (4, 16), (8, 1), (3, 5)]:
+        for trial in range(4):
+            rc = torch.randint(0, 6 if trial else 1, (world, e_loc), generator=g, dtype=torch.int32)
+            to_em, inv, per = ep.regroup_index(rc)
+            want = _brute_regroup(rc.numpy())
+            assert to_em.tolist() == want
+            assert per.tolist() == rc.sum(dim=0).tolist()
+            n = len(want)
+            assert sorted(to_em.tolist()) == list(range(n))
+            assert all(inv[to_em[p]].item() == p for p in range(n))
+
+
+def test_exchange_plan_splits_by_owner_rank():
+    counts = torch.tensor([3, 0, 2, 5, 1, 1, 0, 4], dtype=torch.int32)
+    sc, splits = ep.exchange_plan(counts, 4)
+    assert sc.tolist() == [[3, 0], [2, 5], [1, 1], [0, 4]] and splits == [3, 7, 2, 4]
+    with pytest.raises(AssertionError):
+        ep.exchange_plan(counts, 3)
+
+
+def _worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        E, e_loc = 6, 3
+        g = torch.Generator().manual_seed(100 + rank)
+        counts = torch.randint(0, 5, (E,), generator=g, dtype=torch.int32)
+        # a row is tagged (source rank, global expert, running number); rows are packed expert-major
+        rows = torch.tensor([[rank, e, i] for e in range(E) for i in range(int(counts[e]))], dtype=torch.float32).reshape(-1, 3)
+        send_counts, send_splits = ep.exchange_plan(counts, world)
+        recv_counts = ep.exchange_counts(send_counts)
+        recv_splits = [int(v) for v in recv_counts.sum(dim=1).tolist()]
+        recv = ep.exchange_rows(rows, send_splits, recv_splits)
+        to_em, inv, per = ep.regroup_index(recv_counts)
+        grouped = recv[to_em.long()]
+        # what arrived belongs to this rank's experts, expert-major, sources in rank order
+        keys = [(int(r[1]), int(r[0]), int(r[2])) for r in grouped]
+        ok = keys == sorted(keys) and all(rank * e_loc <= k[0] < (rank + 1) * e_loc for k in keys)
+        ok = ok and per.tolist() == [sum(1 for k in keys if k[0] == rank * e_loc + j) for j in range(e_loc)]
+        # the way back: outputs in arrival order return to the sender in the order it sent them
+        back = grouped[inv.long()] * 2.0
+        returned = ep.exchange_rows(back, recv_splits, send_splits)
+        ok = ok and torch.equal(returned, rows * 2.0)
+        out.put((rank, bool(ok), int(recv.shape[0])))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_exchange_rows_and_get_them_back_in_order():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    results = sorted(out.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert all(ok for _, ok, _ in results)
+
+
+# --------------------------------------------------------------------------- on one GPU
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("shape,world,dtype", [("small", 2, torch.bfloat16), ("small", 4, torch.bfloat16),
+                                               ("small", 4, torch.float32), ("qwen15", 4, torch.bfloat16)])
+def test_ranks_run_in_turn_on_one_gpu_match_the_oracle_and_the_one_gpu_layer(shape, world, dtype):
+    """R ranks, each with its own tokens, all on one device; the all-to-all is done by slicing.
+    The Qwen1.5-MoE-shaped case (15 experts per rank, 2048 tokens on one rank) reaches the tcgen05
+    CTA-pair kernels inside moe_experts_forward."""
+    from oracle import moe_oracle as orc
+    from paper_2509_02753_b200 import binding as B
+    from paper_2509_02753_b200 import synth
+    from parity import TOL, assert_out_close, oracle_weights, rel_err
+
+    if shape == "small":
+        wl = synth.Workload("ep", d=256, E=16, I=256, k_base=4, L=1, I_shared=128, shared_gate=True,
+                            router_bias_std=0.4, w_std=0.02)
+        k, renorm, scale = 3, False, 1.25
+        Ts = [37, 300, 5, 129][:world]
+    else:
+        wl = synth.WORKLOADS[shape]
+        k, renorm, scale = 4, False, 1.0
+        Ts = [2048, 64, 700, 8][:world]
+    max_T = max(Ts)
+    w = synth.make_layer(wl, 0, dtype, "cuda")
+    ow = oracle_weights(synth.to_host(w))
+    xs = [synth.make_tokens(wl, T, dtype, "cuda", seed=10 + r) for r, T in enumerate(Ts)]
+    ranks = [ep.ExpertParallelLayer(wl.d, wl.E, wl.I, max_T, 4, dtype, w, r, world, I_shared=wl.I_shared,
+                                    shared_gate=True, routed_scale=scale) for r in range(world)]
+    try:
+        packed = [rk.pack(x, k, renorm) for rk, x in zip(ranks, xs)]
+        # all-to-all by hand: rank s sends block r of its rows (and row r of its counts) to rank r
+        recv_rows, recv_counts = [], []
+        for r in range(world):
+            blocks, cnts = [], []
+            for s in range(world):
+                rows_s, counts_s, ctx_s = packed[s]
+                off = sum(ctx_s["send_splits"][:r])
+                blocks.append(rows_s[off:off + ctx_s["send_splits"][r]])
+                cnts.append(counts_s[r])
+            recv_rows.append(torch.cat(blocks))
+            recv_counts.append(torch.stack(cnts))
+        backs = [rk.compute(rr, rc) for rk, rr, rc in zip(ranks, recv_rows, recv_counts)]
+        ys = []
+        for s in range(world):
+            parts = []
+            for r in range(world):
+                splits_r = [int(v) for v in recv_counts[r].sum(dim=1).tolist()]
+                off = sum(splits_r[:s])
+                parts.append(backs[r][off:off + splits_r[s]])
+            ys.append(ranks[s].finish(packed[s][2], torch.cat(parts)))
+        torch.cuda.synchronize()
+        with B.MoEPlan(wl.d, wl.E, wl.I, max_T, 4, dtype, I_shared=wl.I_shared, shared_gate=True,
+                       routed_scale=scale) as plan:
+            ws = B.make_weights(w)
+            for x, y in zip(xs, ys):
+                T = x.shape[0]
+                toks = np.arange(T) if T <= 64 else np.random.default_rng(T).choice(T, 40, replace=False)
+                ref = orc.moe_layer(x.cpu(), ow, k, renorm, shared_gate=True, routed_scale=scale, tokens=toks)
+                safe = ref.margin[ref.tokens] > 1e-3
+                assert safe.any()
+                assert_out_close(y.float().cpu().numpy()[ref.tokens][safe], ref.y[safe], dtype, "expert-parallel ranks")
+                one = plan.layer_forward(x, ws, k, renorm)
+                tol = 4e-2 if dtype == torch.bfloat16 else 1e-4
+                assert rel_err(y.float().cpu().numpy(), one.double().cpu().numpy()) <= tol
+            assert plan.device_status() == 0
+        for rk in ranks:
+            assert rk.router_plan.device_status() == 0 and rk.local_plan.device_status() == 0
+    finally:
+        for rk in ranks:
+            rk.close()
