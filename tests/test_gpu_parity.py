@@ -498,3 +498,17 @@ def test_olmoe_shaped_stack_with_seeded_k_vector():
         h8 = x.clone()
         plan.stack_forward(h8, structs, [wl.k_base] * wl.L, wl.renorm)
         assert not torch.equal(h8, h)
+    # the prefill size the benchmark times (T = 4096, same k vector), on sampled tokens
+    Tp = 4096
+    xp = synth.make_tokens(wl, Tp, torch.bfloat16, DEV)
+    toks = np.random.default_rng(5).choice(Tp, 32, replace=False)
+    hp_ref, _, mp = orc.moe_stack(xp.cpu(), ows, k_vec, wl.renorm, tokens=toks)
+    with _plan(wl, Tp, wl.k_base, torch.bfloat16) as plan:
+        hp = xp.clone()
+        plan.stack_forward(hp, structs, k_vec, wl.renorm)
+        assert plan.device_status() == 0
+        hp32 = plan.last_residual_f32(Tp).cpu().numpy()[toks]
+        safe = np.all(mp > 8e-3, axis=0)
+        assert safe.sum() >= 3, safe.sum()
+        assert rel_err(hp32[safe], hp_ref[safe]) <= TOL[torch.bfloat16]
+        assert_out_close(hp.float().cpu().numpy()[toks][safe], hp_ref[safe], torch.bfloat16, "OLMoE-shaped stack, T=4096")
