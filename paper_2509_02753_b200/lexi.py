@@ -40,3 +40,32 @@ def perturbation_profile(plan: B.MoEPlan, weights: B.moe_layer_weights_t, k_base
         n += 1
     assert n > 0, "no samples"
     return {k + 1: total[k] / n for k in range(k_base)}
+
+
+def allocate(plan: B.MoEPlan, layers, k_base: int, budget: int, renorm: bool, *, k_min: int = 1,
+             samples=None, batch: int = 16, seq_len: int = 128, n_iter: int = 8, seed: int = 0):
+    """LExI end to end on one stack (paper, Section 4): Stage 1 profiles every layer's MoE module on
+    its own (Algorithm 1; the same Monte-Carlo samples for every layer), which gives the table
+    D[j, k-1] = mean Delta of layer j at top-k = k; Stage 2 then picks the per-layer allocation
+    k* = (k_1..k_L) with sum k_j = budget and k_min <= k_j <= k_base that minimises sum_j D_j(k_j)
+    (the exact optimum of the objective Algorithm 2 searches).
+
+    ``layers``: sequence of ``moe_layer_weights_t``; ``samples``: optional list of [T, H] CUDA
+    tensors used for every layer (otherwise drawn once from N(0,1) with ``seed``).
+    Returns (k_vec, phi, D) with D a list of L rows of k_base means.
+    """
+    if samples is None:
+        g = torch.Generator(device="cuda")
+        g.manual_seed(seed)
+        samples = []
+        for _ in range(n_iter):
+            x = torch.empty((batch * seq_len, plan.d), dtype=torch.float32, device="cuda")
+            x.normal_(0.0, 1.0, generator=g)
+            samples.append(x.to(plan.dtype))
+    samples = list(samples)
+    D = []
+    for w in layers:
+        prof = perturbation_profile(plan, w, k_base, renorm, samples=samples)
+        D.append([prof[k] for k in range(1, k_base + 1)])
+    k_vec, phi = B.moe_lexi_allocate_exact(D, k_min, budget)
+    return k_vec, phi, D

@@ -68,3 +68,29 @@ def test_stage1_driver_averages_samples():
     mean1 = float(np.mean([r[1] for r in refs]))
     assert got[2] == 0.0 and abs(got[1] - mean1) <= 2e-2 * mean1
     assert drawn[2] == 0.0 and drawn[1] > 0
+
+
+def test_lexi_end_to_end_profile_then_allocate():
+    """Stage 1 on every layer of a 4-layer stack, then Stage 2: the table matches the oracle's literal
+    Algorithm 1 within the Stage-1 tolerance, and the allocation is the brute-force optimum of the
+    library's own table (and feasible)."""
+    from oracle import lexi_stage2 as ref2
+    wl = synth.Workload("e2e", d=256, E=16, I=256, k_base=4, L=4, router_bias_std=0.3)
+    hosts = [synth.make_layer(wl, l, torch.bfloat16, "cpu") for l in range(wl.L)]
+    devs = [{k: (None if v is None else v.cuda()) for k, v in h.items()} for h in hosts]
+    structs = [B.make_weights(w) for w in devs]
+    xs = [synth.make_tokens(wl, 96, torch.bfloat16, "cpu", seed=s) for s in (1, 2)]
+    with B.MoEPlan(wl.d, wl.E, wl.I, 96, 4, torch.bfloat16) as plan:
+        k_vec, phi, D = lexi.allocate(plan, structs, 4, 10, False, samples=[x.cuda() for x in xs])
+        assert plan.device_status() == 0
+    D = np.asarray(D)
+    for l in range(wl.L):
+        refs = [orc.perturbation_profile(x, oracle_weights(hosts[l]), 4, [1, 2, 3, 4], False) for x in xs]
+        base = [float(np.sqrt((orc.moe_layer(x, oracle_weights(hosts[l]), 4, False).y ** 2).sum())) for x in xs]
+        for k in range(1, 5):
+            want = float(np.mean([r[k] for r in refs]))
+            assert abs(D[l, k - 1] - want) <= 1e-2 * float(np.mean(base)), (l, k, D[l, k - 1], want)
+        assert D[l, 3] == 0.0
+    kb, vb = ref2.brute_force(D, 1, 10)
+    assert sum(k_vec) == 10 and all(1 <= v <= 4 for v in k_vec)
+    assert phi == pytest.approx(vb) and phi == pytest.approx(ref2.phi(D, k_vec))
