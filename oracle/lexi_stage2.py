@@ -12,6 +12,11 @@ uint32 numbers in order:
   mutation: if chance(eta): a = below(L); b = below(L-1), stepping over a; child_a += 1; child_b -= 1
   projection: clip; then move single units where that costs least / gains most, lowest index on ties
 The library's implementation is separate code; the two share nothing but this description.
+
+``evolutionary`` can record what it did (``trace``): the initial members and, per generation, the
+two parents' positions in the population and the child after crossover, after mutation and after
+projection.  The pins in the tests read that record against generations worked out by hand, so
+that the steps themselves - not only the final allocation - are held to Algorithm 2.
 """
 from __future__ import annotations
 
@@ -72,7 +77,7 @@ def _project(D, k, k_min, k_max, budget):
 
 
 def evolutionary(D: np.ndarray, k_min: int, budget: int, rnd, *, n_pop: int = 32, g_max: int = 2000,
-                 eta_mut: float = 0.3, tournament: int = 3) -> Tuple[List[int], float]:
+                 eta_mut: float = 0.3, tournament: int = 3, trace: list = None) -> Tuple[List[int], float]:
     D = np.asarray(D, dtype=np.float64)
     L, k_max = D.shape
     r = _Stream(rnd)
@@ -84,6 +89,8 @@ def evolutionary(D: np.ndarray, k_min: int, budget: int, rnd, *, n_pop: int = 32
             k[open_layers[r.below(len(open_layers))]] += 1
         pop.append(k)
         fit.append(phi(D, k))
+    if trace is not None:
+        trace.append({"init": [list(k) for k in pop]})
     for _g in range(g_max):
         parents = []
         for _q in range(2):
@@ -95,6 +102,7 @@ def evolutionary(D: np.ndarray, k_min: int, budget: int, rnd, *, n_pop: int = 32
             parents.append(best)
         p1, p2 = pop[parents[0]], pop[parents[1]]
         child = [p1[j] if r.coin() else p2[j] for j in range(L)]
+        crossed = list(child)
         if L >= 2 and r.chance(eta_mut):
             a = r.below(L)
             b = r.below(L - 1)
@@ -102,7 +110,11 @@ def evolutionary(D: np.ndarray, k_min: int, budget: int, rnd, *, n_pop: int = 32
                 b += 1
             child[a] += 1
             child[b] -= 1
+        mutated = list(child)
         child = _project(D, child, k_min, k_max, budget)
+        if trace is not None:
+            trace.append({"parents": tuple(parents), "crossed": crossed, "mutated": mutated,
+                          "projected": list(child)})
         pop.append(child)
         fit.append(phi(D, child))
     best = min(range(len(pop)), key=lambda m: (fit[m], m))
