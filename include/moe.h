@@ -288,14 +288,19 @@ int moe_route_from_logits(moe_plan_t *plan, const float *logits, int32_t T, int3
  * synchronisation cudaMalloc/cudaFree imply, or a component that is given buffers and a stream
  * but owns no allocator and therefore cannot create a plan.
  *
- *   topk_idx [T, k_l] int32 device (entries outside 0..E-1 are skipped);
+ *   topk_idx [T, k_l] int32 device;
  *   counts [E], offsets [E+1], perm [T*k_l] int32 device, written.
+ *   An entry of topk_idx outside 0..E-1 is skipped and nothing else reports it: the counts then sum
+ *   to fewer than T * k_l, offsets[E] is the number of pairs placed and perm[offsets[E]..] is left
+ *   untouched, so a caller that cannot rule such entries out compares offsets[E] with T * k_l.
  *   Limits: T * k_l <= 65536 and E <= 128; beyond them the call fails with MOE_ERR_SHAPE.
  *
  * The scratch of the three dispatch passes is a fixed 393,472-byte array in the library's
  * device image: every GPU that loads the library holds it until the process exits.  The first
- * call on a device looks up the array's device address (that device must be current); make that
- * first call before starting any stream capture.  All calls on a device share the array, which
+ * call on a device looks up the array's device address (that device must be current; the look-up is
+ * safe against two host threads making their first call at once, and is not repeated, so the
+ * library must not be used across a cudaDeviceReset); make that first call before starting any
+ * stream capture.  All calls on a device share the array, which
  * keeps the previous call's contents (the call clears the one word that must start at zero), so
  * two calls whose kernels overlap on the GPU race: keep them on one stream or order them.
  * Calls no cudaMalloc/cudaFree.  Asynchronous on the stream.

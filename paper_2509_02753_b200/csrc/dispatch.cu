@@ -7,6 +7,8 @@
 //
 // Everything is deterministic: ranks come from warp ballots over pairs taken in order, never
 // from the arrival order of atomics.
+#include <atomic>
+
 #include "moe_internal.h"
 #include "tile_build.cuh"
 
@@ -310,17 +312,18 @@ static __device__ __align__(256) int32_t g_dispatch_scratch[kStaticScratchInts];
 // The array's name is only a host-side handle; the device address has to be asked for, once per
 // device, with that device current.
 constexpr int kMaxDevices = 64;
-int32_t *g_scratch_addr[kMaxDevices] = {};
+std::atomic<int32_t *> g_scratch_addr[kMaxDevices];
 
 int32_t *static_scratch_for_current_device() {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return nullptr; }
-    if (!g_scratch_addr[dev]) {
-        int32_t *ptr = nullptr;
+    int32_t *ptr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
+        // two host threads may both get here on their first call; both are told the same address
         if (cudaGetSymbolAddress((void **)&ptr, g_dispatch_scratch) != cudaSuccess) { cudaGetLastError(); return nullptr; }
-        g_scratch_addr[dev] = ptr;
+        g_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    return g_scratch_addr[dev];
+    return ptr;
 }
 
 }  // namespace

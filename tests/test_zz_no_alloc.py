@@ -4,27 +4,38 @@
 the tables (a decoding loop that must not hit cudaMalloc's device-wide synchronisation, or a
 component with buffers and a stream but no allocator, which therefore cannot own a plan).  Its
 scratch is one fixed array inside the library that all calls share and that keeps the previous
-call's contents, so the test makes two calls in a row, the second one smaller than the first,
-and compares both with `moe_route_from_logits`.  Integer tables: the comparison is bit-exact,
+call's contents, so the test makes several calls in a row, smaller ones after larger ones.
+What is expected comes from the CPU oracle's dispatch (the integer definition written out as
+two loops), applied to indices the oracle selected; the plan-based entry point
+`moe_route_from_logits` must give the same tables.  Integer tables: the comparison is bit-exact,
 as in the other routing tests.  Collected last (file name) so an earlier failure cannot hide it.
 """
 import ctypes
 
+import numpy as np
 import pytest
 import torch
 
+from oracle import moe_oracle as orc
 from paper_2509_02753_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
 
 
 def _tables_from_plan(T, E, k, seed):
+    """(idx on the device, counts, offsets, perm): expected tables from the oracle; the plan-based
+    entry point is checked against them on the way."""
     g = torch.Generator().manual_seed(seed)
-    logits = torch.randn((T, E), generator=g, dtype=torch.float32).cuda()
+    logits = torch.randn((T, E), generator=g, dtype=torch.float32)
+    idx_o, _, _ = orc.topk_gates(logits.numpy(), k, False, select_f32=True)
+    counts_o, offsets_o, perm_o, _ = orc.dispatch(idx_o, E)
     with B.MoEPlan(64, E, 64, T, k, torch.float32) as plan:
-        idx, _, counts, offsets, perm = plan.route_from_logits(logits, k, False)
+        idx, _, counts, offsets, perm = plan.route_from_logits(logits.cuda(), k, False)
         assert plan.device_status() == 0
-    return idx, counts, offsets, perm
+    assert np.array_equal(idx.cpu().numpy(), idx_o)
+    assert np.array_equal(counts.cpu().numpy(), counts_o) and np.array_equal(perm.cpu().numpy(), perm_o)
+    dev = lambda a: torch.from_numpy(a).cuda()
+    return dev(idx_o), dev(counts_o), dev(offsets_o), dev(perm_o)
 
 
 def test_static_scratch_dispatch_matches_plan_dispatch_twice_in_a_row():
@@ -50,6 +61,36 @@ def test_static_scratch_dispatch_matches_plan_dispatch_twice_in_a_row():
     with torch.cuda.stream(s):
         B.moe_dispatch_tables_static(idx, E, c, o, p, stream=s)
     s.synchronize()
+    assert torch.equal(c, counts) and torch.equal(o, offsets) and torch.equal(p, perm)
+
+
+def test_static_scratch_dispatch_skips_entries_outside_the_expert_range_visibly():
+    """An index outside 0..E-1 is left out of the tables: the counts then sum to fewer than T * k_l
+    pairs, offsets[E] says how many were placed, and perm beyond that many entries is not written -
+    which is how a caller notices.  The placed pairs are those of the oracle's dispatch with the bad
+    pair removed."""
+    T, E, k = 300, 16, 2
+    g = torch.Generator().manual_seed(3)
+    idx = torch.stack([torch.randperm(E, generator=g)[:k] for _ in range(T)]).to(torch.int32)
+    idx[17, 1] = E                                   # one pair names an expert that does not exist
+    keep = np.ones(T * k, dtype=bool)
+    keep[17 * k + 1] = False
+    flat = idx.numpy().reshape(-1)
+    order = [p for e in range(E) for p in range(T * k) if keep[p] and flat[p] == e]   # the definition
+    counts_e = np.bincount(flat[keep], minlength=E).astype(np.int32)
+    c = torch.full((E,), -7, dtype=torch.int32, device="cuda")
+    o = torch.full((E + 1,), -7, dtype=torch.int32, device="cuda")
+    p = torch.full((T * k,), -7, dtype=torch.int32, device="cuda")
+    B.moe_dispatch_tables_static(idx.cuda(), E, c, o, p)
+    torch.cuda.synchronize()
+    assert np.array_equal(c.cpu().numpy(), counts_e)
+    assert int(o[E]) == T * k - 1
+    assert p.cpu().numpy()[:T * k - 1].tolist() == order
+    assert int(p[T * k - 1]) == -7                   # the tail is left as the caller had it
+    # the next call with valid indices is not affected by what the bad one left in the shared array
+    idx_ok, counts, offsets, perm = _tables_from_plan(300, 16, 2, 5)
+    B.moe_dispatch_tables_static(idx_ok, E, c, o, p)
+    torch.cuda.synchronize()
     assert torch.equal(c, counts) and torch.equal(o, offsets) and torch.equal(p, perm)
 
 
