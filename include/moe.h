@@ -62,11 +62,13 @@ typedef enum {
                                environment selects the 128x256 one-CTA kernel instead),
                                double-buffered TMEM accumulators                            */
     MOE_SCHED_PREFILL_1CTA = 4, /* prefill on the one-CTA 128x256 kernel; never chosen by AUTO */
-    MOE_SCHED_DECODE_FUSED = 5  /* bf16, at most 8 tokens: the whole layer (router to combine) in one
-                               cooperative launch that streams the touched experts' weights
+    MOE_SCHED_DECODE_FUSED = 5  /* bf16, at most 8 tokens: the whole layer (router to combine) - and in
+                               moe_stack_forward the whole stack of layers, up to 44 per launch -
+                               in one cooperative launch that streams the touched experts' weights
                                through mma.sync with the tokens in the N dimension; a call
                                with more tokens falls back to MOE_SCHED_DECODE.  Needs d, I and
-                               I_shared to be multiples of 32 (else set_schedule -> SHAPE).
+                               I_shared to be multiples of 32 and d <= 64 x the SM count (else
+                               set_schedule -> SHAPE).
                                The launch needs every SM of the device to itself while it runs. */
 } moe_schedule_t;
 
@@ -225,6 +227,10 @@ int moe_host_pipeline_wait(moe_plan_t *plan, int64_t ticket);
  *   k_vec: HOST array of n_layers values, each in 1..max_k.
  * For bf16 the running h is kept in fp32 inside the plan (each layer reads it rounded to
  * bf16; the final h is rounded once), so rounding does not accumulate over the layers.
+ * Calls of at most 8 tokens on a plan whose shape allows MOE_SCHED_DECODE_FUSED run the whole stack
+ * in one launch per 44 layers: the grid stays resident from layer to layer, the fp32 residual
+ * stream stays on chip, and the routing of layer l+1 is prepared while layer l's down projection
+ * finishes.  After the call moe_last_routing describes the last layer.
  * Errors: as moe_layer_forward.
  */
 int moe_stack_forward(moe_plan_t *plan, void *h, const moe_layer_weights_t *layers,
@@ -326,11 +332,13 @@ int moe_last_routing(moe_plan_t *plan, int32_t *topk_idx, float *topk_w, int32_t
 int moe_last_residual_f32(moe_plan_t *plan, float *h_f32, int32_t T, void *cuda_stream);
 
 /*
- * Debug hook of MOE_SCHED_DECODE_FUSED (the paper has no counterpart): with enable != 0 every
- * later one-launch layer call records, per CTA, eight %globaltimer values in ns (start, logits
- * sent, shared gate/up stream done, logits complete, routed, gate/up stream done, h' complete,
- * end).  out_host (host memory, may be NULL) receives up to `capacity` values, [CTA][8], of the
- * last stamped call after synchronising the stream; *n_ctas (may be NULL) the number of CTAs.
+ * Debug hook of MOE_SCHED_DECODE_FUSED (the paper has no counterpart): with enable = 1 + l every
+ * later one-launch call records, per CTA, eight %globaltimer values in ns for its layer l (the last
+ * layer if the call has fewer): layer start, h staged in shared memory, shared-expert gate/up
+ * stream done, routing known, gate/up stream done, all of h' written (grid barrier passed), down
+ * stream done, layer end (grid barrier passed).  enable = 0 switches the stamps off.  out_host
+ * (host memory, may be NULL) receives up to `capacity` values, [CTA][8], of the last stamped call
+ * after synchronising the stream; *n_ctas (may be NULL) the number of CTAs.
  * Errors: INVALID_ARG (also when the plan's shape has no one-launch layer), CUDA.
  */
 int moe_debug_fused_stamps(moe_plan_t *plan, int32_t enable, uint64_t *out_host, int32_t capacity,
@@ -344,6 +352,17 @@ int moe_debug_fused_stamps(moe_plan_t *plan, int32_t enable, uint64_t *out_host,
  * MOE_ERR_TIMEOUT; the context stays usable.  Errors: INVALID_ARG, CUDA.
  */
 int moe_debug_wait_timeout(moe_plan_t *plan, int32_t limit_us, void *cuda_stream);
+
+/*
+ * moe_debug_barrier_timeout (test hook for the failure path of MOE_SCHED_DECODE_FUSED): launches a
+ * one-thread kernel that runs the one-launch kernel's grid-barrier wait on a target the plan's
+ * barrier counter never reaches, with a limit of limit_us microseconds (1 .. 1,000,000).  The wait
+ * gives up and sets the time-out bit of the device status word.  While that bit is set every
+ * one-launch call returns at once without computing; moe_device_status reports MOE_ERR_TIMEOUT,
+ * clears the bit and puts the barrier counter and the logit accumulators back to zero, after which
+ * one-launch calls work again.  Errors: INVALID_ARG (also when the plan has no one-launch layer), CUDA.
+ */
+int moe_debug_barrier_timeout(moe_plan_t *plan, int32_t limit_us, void *cuda_stream);
 
 /*
  * moe_device_status: synchronises the stream, reads and clears the device status word.

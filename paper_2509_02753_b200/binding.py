@@ -31,7 +31,7 @@ EXPORTS = (
     "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts",
     "moe_debug_fused_stamps", "moe_host_pipeline_submit", "moe_host_pipeline_wait",
     "moe_route", "moe_gather_rows", "moe_experts_forward", "moe_combine",
-    "moe_debug_wait_timeout", "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
+    "moe_debug_wait_timeout", "moe_debug_barrier_timeout", "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
 
@@ -83,6 +83,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_last_routing.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.moe_device_status.argtypes = [vp, vp]
     lib.moe_debug_wait_timeout.argtypes = [vp, i32, vp]
+    lib.moe_debug_barrier_timeout.argtypes = [vp, i32, vp]
     lib.moe_last_residual_f32.argtypes = [vp, vp, i32, vp]
     lib.moe_plan_touched_experts.argtypes = [vp, P(ctypes.c_int64), vp]
     lib.moe_debug_fused_stamps.argtypes = [vp, i32, P(ctypes.c_uint64), i32, P(i32), vp]
@@ -381,9 +382,10 @@ def moe_plan_touched_experts(plan: int, stream=None) -> int:
     return int(n.value)
 
 
-def moe_debug_fused_stamps(plan: int, enable: bool, read: bool = False, stream=None):
-    """Switches the time stamps of the one-launch layer on or off; with read=True returns the last
-    stamped call's values as a list of per-CTA lists of eight ns values."""
+def moe_debug_fused_stamps(plan: int, enable: int, read: bool = False, stream=None):
+    """Switches the time stamps of the one-launch kernel on (enable = 1 + index of the layer to stamp;
+    True stamps layer 0) or off (0); with read=True returns the last stamped call's values as a list
+    of per-CTA lists of eight ns values."""
     lib = load_library()
     n = ctypes.c_int32()
     _check("moe_debug_fused_stamps", lib.moe_debug_fused_stamps(plan, int(enable), None, 0, ctypes.byref(n), _stream(stream)))
@@ -418,6 +420,12 @@ def moe_debug_wait_timeout(plan: int, limit_us: int, stream=None) -> None:
     """Runs the bounded device-side wait on a barrier nobody signals; see moe_device_status."""
     _check("moe_debug_wait_timeout",
            load_library().moe_debug_wait_timeout(plan, limit_us, _stream(stream)))
+
+
+def moe_debug_barrier_timeout(plan: int, limit_us: int, stream=None) -> None:
+    """Runs the one-launch kernel's grid-barrier wait on a target nothing reaches; see moe_device_status."""
+    _check("moe_debug_barrier_timeout",
+           load_library().moe_debug_barrier_timeout(plan, limit_us, _stream(stream)))
 
 
 def moe_device_status(plan: int, stream=None) -> int:

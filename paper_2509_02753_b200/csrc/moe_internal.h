@@ -59,11 +59,9 @@ struct Workspace {
     double  *prof_sums = nullptr;     // [max_k + 1]
     int32_t *stats = nullptr;      // [4] counters read by moe_plan_touched_experts
     int32_t *pos = nullptr;        // [E, 128] direct mode: output row of (expert, token) or -1
-    // one-launch layer for calls of at most kFusedMaxTokens tokens (decode_fused.cu)
-    float   *f_part0 = nullptr;    // router logit partials, 128 floats per (16 rows, 128 columns) chunk
-    float   *f_parts = nullptr;    // [SMs][2] per-CTA partial sums of down-stream blocks split between CTAs
-    int32_t *f_tickets = nullptr;  // [d / 16] arrival counters of the down-stream blocks (zero between calls)
-    uint32_t *f_bar = nullptr;     // grid-barrier counter (only grows; reset by the host from time to time)
+    // one-launch stack for calls of at most kFusedMaxTokens tokens (decode_stack.cu)
+    long long *f_zacc = nullptr;   // [2][8][kMaxExperts] fixed-point logit accumulators (zero between launches)
+    uint32_t *f_bar = nullptr;     // grid-barrier counter (only grows; the plan tracks its value)
     __nv_bfloat16 *f_hbuf = nullptr;  // [8, I_s + U_cap * I] gate-weighted hidden activations
     unsigned long long *f_stamps = nullptr;   // [SMs, 8] %globaltimer stamps of the last stamped call
 };
@@ -152,7 +150,7 @@ cudaError_t launch_combine(const CombineArgs &a, cudaStream_t s, uint64_t *launc
 cudaError_t launch_profile(const CombineArgs &a, int renorm, float *partial, double *sums, cudaStream_t s,
                            uint64_t *launches);
 
-// ---- one-launch layer for tiny decode calls (decode_fused.cu) ----------------------------
+// ---- one launch for a whole stack of layers at tiny decode sizes (decode_stack.cu) ------------
 constexpr int kFusedMaxTokens = 8;
 #ifndef LEXI_FUSED_WARPS
 #define LEXI_FUSED_WARPS 12
@@ -161,22 +159,35 @@ constexpr int kFusedMaxTokens = 8;
 // flight per warp without spills; 16 warps (128 registers, spills) measured 5-10 % slower.
 constexpr int kFusedWarps = LEXI_FUSED_WARPS;
 constexpr int kFusedThreads = kFusedWarps * 32;
-constexpr int kFusedMaxCtaBlocks = 512;   // row blocks of one stream that may fall to one CTA
-struct FusedArgs {
-    const void *x; __nv_bfloat16 *y; float *h_run; int mode;   // mode 0: y = MoE(x); 1: h_run += MoE(x), y = round(h_run)
+constexpr int kFusedMaxCtaBlocks = 512;   // gate/up row blocks of one stream that may fall to one CTA
+constexpr int kFusedMaxCtaRows = 64;      // rows of the residual stream one CTA may own (d <= 64 x SMs)
+constexpr int kStackMaxLayers = 44;       // layers per launch (their pointers travel as kernel parameters)
+struct LayerDesc {
     const void *router_W; const float *router_bias; const void *w_s;   // w_s NULL: shared gate = 1
     const void *W_gate, *W_up, *W_down, *Ws_gate, *Ws_up, *Ws_down;
-    int T, d, E, I, I_s, k, renorm;
-    float routed_scale;
-    float *logits; int32_t *topk_idx; float *topk_w; float *gamma;
-    int32_t *counts, *offsets, *perm, *inv_perm, *stats, *status;
-    float *part0, *parts; int32_t *tickets;   // logit partials; per-CTA partials and arrival counters of the down stream
-    uint32_t *bar; __nv_bfloat16 *hbuf; int hs;                       // hs: row pitch of hbuf
-    unsigned long long *stamps;                                       // NULL, or [grid, 8] time stamps (debug)
+    int32_t k, pad;
 };
+struct StackArgs {
+    const void *x; __nv_bfloat16 *y; float *h_run;
+    int mode;      // 0: y = MoE(x) (L = 1).  1: h <- h + MoE_l(h; k_l) for L layers, fp32 residual on chip, y = round(h)
+                   //    after every layer (y may be x), h_run = the fp32 h after the last one
+    int resume;    // mode 1: the residual stream starts from h_run (a stack continued from an earlier launch), not from x
+    int L, T, d, E, I, I_s, renorm;
+    float routed_scale;
+    float *logits; int32_t *topk_idx; float *topk_w; float *gamma;      // routing of the last layer, as moe_last_routing reports it
+    int32_t *counts, *offsets, *perm, *inv_perm, *stats, *status;
+    long long *zacc;                    // [2][8][kMaxExperts] logit accumulators (2^-40 units), zero between launches
+    uint32_t *bar; uint32_t bar_base;   // grid-barrier counter and its value when this launch starts
+    __nv_bfloat16 *hbuf; int hs;        // gate-weighted hidden activations h', row pitch hs
+    unsigned long long *stamps; int stamp_layer;   // NULL, or [grid, 8] time stamps of one layer (debug)
+    unsigned long long limit_ns;        // bound of every wait
+    LayerDesc layers[kStackMaxLayers];
+};
+static_assert(sizeof(StackArgs) <= 4000, "the stack's arguments travel as kernel parameters");
 size_t fused_smem_bytes(int d);
-cudaError_t fused_prepare(int d);    // opts the kernel in to its shared-memory size (once per plan)
-cudaError_t launch_decode_fused(const FusedArgs &a, int sm_count, cudaStream_t s, uint64_t *launches);
+cudaError_t fused_prepare(int d);    // opts the kernel in to its shared-memory size (per device, only grows)
+cudaError_t launch_decode_stack(const StackArgs &a, int sm_count, cudaStream_t s, uint64_t *launches);
+cudaError_t launch_barrier_probe(const uint32_t *bar, int32_t *status, unsigned long long limit_ns, cudaStream_t s);
 
 cudaError_t launch_widen(const void *src, float *dst, size_t n, int dtype, cudaStream_t s,
                          uint64_t *launches);

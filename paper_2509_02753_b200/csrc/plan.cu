@@ -38,9 +38,9 @@ struct moe_plan {
     bool use_pdl = true;         // programmatic dependent launch along the decode chain
     bool fused_ok = false;       // the one-launch layer for <= kFusedMaxTokens tokens is available for this shape
     bool use_fused = true;       // ... and chosen by MOE_SCHED_AUTO (LEXI_DECODE_FUSED=0 turns that off)
-    int fused_tk_total = 0, fused_hs = 0;
-    uint64_t fused_calls = 0;
-    bool fused_stamps = false;   // debug: later one-launch calls record time stamps
+    int fused_hs = 0;
+    uint32_t fused_bar_base = 0; // value of the grid-barrier counter when the next one-launch call starts
+    int fused_stamp_layer = -1;  // debug: later one-launch calls record time stamps of this layer (-1: none)
     TcState tc{};
     // stage timing: kMaxTimedCalls sets of MOE_N_STAGES + 1 events
     bool timing = false;
@@ -91,37 +91,43 @@ int pick_schedule(const moe_plan *p, int T, int k) {
     return (fused_fits && p->use_fused) ? MOE_SCHED_DECODE_FUSED : MOE_SCHED_DECODE;
 }
 
-// Whole layer in one cooperative launch (decode_fused.cu).
-int fused_layer(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, int k, int renorm, void *y,
-                int mode, cudaStream_t s) {
+// Up to kStackMaxLayers layers in one cooperative launch (decode_stack.cu); a single layer call is a
+// stack of one.  mode 0: y = MoE(x).  mode 1: h <- h + MoE_l(h; k_l), x = y = h; resume: the fp32
+// residual stream continues from ws.h_run (the stack is longer than one launch holds).
+int fused_stack(moe_plan *p, const void *x, const moe_layer_weights_t *layers, const int32_t *k_vec, int n_layers,
+                int T, int renorm, void *y, int mode, int resume, cudaStream_t s) {
     const moe_config_t &c = p->cfg;
     Workspace &ws = p->ws;
-    // the barrier counter only grows; long before it could wrap it is put back to zero in stream order
-    if ((++p->fused_calls & 0xfffffu) == 0 && cudaMemsetAsync(ws.f_bar, 0, sizeof(uint32_t), s) != cudaSuccess) {
-        cudaGetLastError();
-        return MOE_ERR_CUDA;
-    }
-    FusedArgs fa{};
-    fa.x = x; fa.y = (__nv_bfloat16 *)y; fa.h_run = ws.h_run; fa.mode = mode;
-    fa.router_W = w->router_W; fa.router_bias = w->router_bias;
-    fa.w_s = (c.I_shared > 0 && c.shared_gate) ? w->w_s : nullptr;
-    fa.W_gate = w->W_gate; fa.W_up = w->W_up; fa.W_down = w->W_down;
-    fa.Ws_gate = w->Ws_gate; fa.Ws_up = w->Ws_up; fa.Ws_down = w->Ws_down;
-    fa.T = T; fa.d = c.d; fa.E = c.E; fa.I = c.I; fa.I_s = c.I_shared; fa.k = k; fa.renorm = renorm;
+    StackArgs fa{};
+    fa.x = x; fa.y = (__nv_bfloat16 *)y; fa.h_run = ws.h_run; fa.mode = mode; fa.resume = resume;
+    fa.L = n_layers; fa.T = T; fa.d = c.d; fa.E = c.E; fa.I = c.I; fa.I_s = c.I_shared; fa.renorm = renorm;
     fa.routed_scale = c.routed_scale;
     fa.logits = ws.logits; fa.topk_idx = ws.topk_idx; fa.topk_w = ws.topk_w; fa.gamma = ws.gamma;
     fa.counts = ws.counts; fa.offsets = ws.offsets; fa.perm = ws.perm; fa.inv_perm = ws.inv_perm;
     fa.stats = ws.stats; fa.status = ws.status;
-    fa.part0 = ws.f_part0; fa.parts = ws.f_parts; fa.tickets = ws.f_tickets;
-    fa.bar = ws.f_bar; fa.hbuf = ws.f_hbuf; fa.hs = p->fused_hs;
-    fa.stamps = p->fused_stamps ? ws.f_stamps : nullptr;
-    if (launch_decode_fused(fa, p->sm_count, s, &p->launches) != cudaSuccess) {
+    fa.zacc = ws.f_zacc; fa.bar = ws.f_bar; fa.bar_base = p->fused_bar_base;
+    fa.hbuf = ws.f_hbuf; fa.hs = p->fused_hs;
+    fa.stamps = p->fused_stamp_layer >= 0 ? ws.f_stamps : nullptr;
+    fa.stamp_layer = p->fused_stamp_layer < n_layers ? p->fused_stamp_layer : n_layers - 1;
+    fa.limit_ns = 1000000000ull;
+    for (int l = 0; l < n_layers; ++l) {
+        const moe_layer_weights_t &w = layers[l];
+        LayerDesc &d = fa.layers[l];
+        d.router_W = w.router_W; d.router_bias = w.router_bias;
+        d.w_s = (c.I_shared > 0 && c.shared_gate) ? w.w_s : nullptr;
+        d.W_gate = w.W_gate; d.W_up = w.W_up; d.W_down = w.W_down;
+        d.Ws_gate = w.Ws_gate; d.Ws_up = w.Ws_up; d.Ws_down = w.Ws_down;
+        d.k = k_vec[l];
+    }
+    if (launch_decode_stack(fa, p->sm_count, s, &p->launches) != cudaSuccess) {
         // the grid did not fit the device at once (SMs taken away from this context, say): the
         // kernel chain serves this and all later calls of the plan
         cudaGetLastError();
         p->fused_ok = false;
         return MOE_ERR_NOT_IMPLEMENTED;
     }
+    // a launch passes one barrier after its pre-pass and two per layer except behind the last
+    p->fused_bar_base += (uint32_t)(2 * n_layers) * (uint32_t)p->sm_count;
     return MOE_OK;
 }
 
@@ -150,7 +156,9 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
     int sched = pick_schedule(p, T, k);
     if (sched == MOE_SCHED_DECODE_FUSED && (mode == 0 || mode == 1)) {
         mark(1); mark(2);                 // the whole call is booked under the first GEMM stage
-        const int rc = fused_layer(p, x, w, T, k, renorm, y, mode, s);
+        // a layer of a stack that is walked one call at a time (mode 1) continues the fp32 stream in ws.h_run
+        const int32_t k1 = k;
+        const int rc = fused_stack(p, x, w, &k1, 1, T, renorm, y, mode, mode == 1 ? 1 : 0, s);
         if (rc == MOE_OK) {
             mark(3); mark(4); mark(5);
             p->last_T = T;
@@ -348,27 +356,30 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
     }
     const int rc = tc_state_init(&p->tc, c);
     if (rc != MOE_OK) { moe_plan_destroy(p); return rc; }
-    // one-launch layer for tiny decode calls: scratch for its partial sums, arrival counters and h'
-    if (c.dtype == MOE_BF16 && tc_shape_ok(c) && c.d % 32 == 0 && c.I % 32 == 0 && c.I_shared % 32 == 0 &&
-        fused_smem_bytes(c.d) <= 160 * 1024 &&
-        ((c.E < kFusedMaxTokens * c.max_k ? c.E : kFusedMaxTokens * c.max_k) * (c.I / 8)) / sms + 2 <= kFusedMaxCtaBlocks &&
-        (c.I_shared / 8) / sms + 2 <= kFusedMaxCtaBlocks) {
+    // one-launch stack for tiny decode calls: logit accumulators, barrier counter, h'
+    {
         const int ucap = c.E < kFusedMaxTokens * c.max_k ? c.E : kFusedMaxTokens * c.max_k;
-        p->fused_tk_total = c.d / 16;
-        p->fused_hs = c.I_shared + ucap * c.I;
-        bool fok = ws_alloc(p, &ws.f_part0, (size_t)((c.E + 15) / 16) * ((c.d + 127) / 128) * 128) &&
-                   ws_alloc(p, &ws.f_parts, (size_t)sms * 2 * 128) &&
-                   ws_alloc(p, &ws.f_tickets, (size_t)p->fused_tk_total) &&
-                   ws_alloc(p, &ws.f_bar, (size_t)4) &&
-                   ws_alloc(p, &ws.f_hbuf, (size_t)kFusedMaxTokens * p->fused_hs) &&
-                   ws_alloc(p, &ws.f_stamps, (size_t)sms * 8);
-        fok = fok && cudaMemset(ws.f_tickets, 0, sizeof(int32_t) * p->fused_tk_total) == cudaSuccess &&
-              cudaMemset(ws.f_bar, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess &&
-              fused_prepare(c.d) == cudaSuccess;
-        if (!fok) { cudaGetLastError(); moe_plan_destroy(p); return MOE_ERR_WORKSPACE; }
-        p->fused_ok = true;
-        const char *env = getenv("LEXI_DECODE_FUSED");
-        p->use_fused = !(env && env[0] == '0');
+        // gate/up row blocks that can fall to one CTA: its features in blocks of 8, plus one ragged
+        // block per expert boundary inside its range
+        const long long feat_cta = ((long long)ucap * c.I + sms - 1) / sms + 1;
+        const long long blocks_cta = feat_cta / 8 + feat_cta / c.I + 4;
+        const long long blocks_cta_s = ((long long)c.I_shared / sms + 1) / 8 + 2;
+        if (c.dtype == MOE_BF16 && tc_shape_ok(c) && c.d % 32 == 0 && c.I % 32 == 0 && c.I_shared % 32 == 0 &&
+            fused_smem_bytes(c.d) <= 200 * 1024 && (c.d + sms - 1) / sms <= kFusedMaxCtaRows &&
+            blocks_cta <= kFusedMaxCtaBlocks && blocks_cta_s <= kFusedMaxCtaBlocks) {
+            p->fused_hs = c.I_shared + ucap * c.I;
+            bool fok = ws_alloc(p, &ws.f_zacc, (size_t)2 * kFusedMaxTokens * kMaxExperts) &&
+                       ws_alloc(p, &ws.f_bar, (size_t)4) &&
+                       ws_alloc(p, &ws.f_hbuf, (size_t)kFusedMaxTokens * p->fused_hs) &&
+                       ws_alloc(p, &ws.f_stamps, (size_t)sms * 8);
+            fok = fok && cudaMemset(ws.f_zacc, 0, sizeof(long long) * 2 * kFusedMaxTokens * kMaxExperts) == cudaSuccess &&
+                  cudaMemset(ws.f_bar, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess &&
+                  fused_prepare(c.d) == cudaSuccess;
+            if (!fok) { cudaGetLastError(); moe_plan_destroy(p); return MOE_ERR_WORKSPACE; }
+            p->fused_ok = true;
+            const char *env = getenv("LEXI_DECODE_FUSED");
+            p->use_fused = !(env && env[0] == '0');
+        }
     }
     *out = p;
     return MOE_OK;
@@ -703,6 +714,24 @@ int moe_stack_forward(moe_plan_t *p, void *h, const moe_layer_weights_t *layers,
     if (T == 0 || n_layers == 0) return MOE_OK;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     const bool bf16 = p->cfg.dtype == MOE_BF16;
+    // at most 8 tokens: the whole stack runs in one launch per kStackMaxLayers layers, the residual
+    // stream in fp32 on chip (the schedule does not depend on k_l at this size)
+    if (bf16 && pick_schedule(p, T, k_vec[0]) == MOE_SCHED_DECODE_FUSED && !p->timing) {
+        int done = 0;
+        while (done < n_layers) {
+            const int n = n_layers - done < kStackMaxLayers ? n_layers - done : kStackMaxLayers;
+            const int rc = fused_stack(p, h, layers + done, k_vec + done, n, T, renorm ? 1 : 0, h, 1, done > 0 ? 1 : 0, s);
+            if (rc == MOE_ERR_NOT_IMPLEMENTED) break;      // no cooperative grid: the per-layer path below takes over
+            if (rc != MOE_OK) return rc;
+            done += n;
+        }
+        if (done == n_layers) {
+            p->last_T = T;
+            p->last_k = k_vec[n_layers - 1];
+            return MOE_OK;
+        }
+        if (done > 0) return MOE_ERR_CUDA;     // cannot happen: the first launch decides whether the grid fits
+    }
     if (bf16 && launch_widen(h, p->ws.h_run, (size_t)T * p->cfg.d, MOE_BF16, s, &p->launches) != cudaSuccess)
         return MOE_ERR_CUDA;
     for (int l = 0; l < n_layers; ++l) {
@@ -789,8 +818,8 @@ int moe_debug_wait_timeout(moe_plan_t *p, int32_t limit_us, void *cuda_stream) {
 
 int moe_debug_fused_stamps(moe_plan_t *p, int32_t enable, uint64_t *out_host, int32_t capacity, int32_t *n_ctas,
                            void *cuda_stream) {
-    if (!p || !p->fused_ok || capacity < 0) return MOE_ERR_INVALID_ARG;
-    p->fused_stamps = enable != 0;
+    if (!p || !p->fused_ok || capacity < 0 || enable < 0) return MOE_ERR_INVALID_ARG;
+    p->fused_stamp_layer = enable - 1;
     if (n_ctas) *n_ctas = p->sm_count;
     if (out_host && capacity > 0) {
         const size_t n = (size_t)capacity < (size_t)p->sm_count * 8 ? (size_t)capacity : (size_t)p->sm_count * 8;
@@ -801,6 +830,17 @@ int moe_debug_fused_stamps(moe_plan_t *p, int32_t enable, uint64_t *out_host, in
             return MOE_ERR_CUDA;
         }
     }
+    return MOE_OK;
+}
+
+int moe_debug_barrier_timeout(moe_plan_t *p, int32_t limit_us, void *cuda_stream) {
+    if (!p || !p->fused_ok || limit_us < 1 || limit_us > 1000000) return MOE_ERR_INVALID_ARG;
+    if (launch_barrier_probe(p->ws.f_bar, p->ws.status, (unsigned long long)limit_us * 1000ull,
+                             (cudaStream_t)cuda_stream) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    ++p->launches;
     return MOE_OK;
 }
 
@@ -815,10 +855,12 @@ int moe_device_status(moe_plan_t *p, void *cuda_stream) {
     }
     const int32_t v = *p->status_host;
     if ((v & kStatusTimeout) && p->fused_ok) {
-        // a one-launch layer that gave up may have left arrival counters behind
-        cudaMemsetAsync(p->ws.f_tickets, 0, sizeof(int32_t) * p->fused_tk_total, s);
+        // a one-launch call that gave up has left the barrier counter and the logit accumulators
+        // half way: both start again from zero
+        cudaMemsetAsync(p->ws.f_zacc, 0, sizeof(long long) * 2 * kFusedMaxTokens * kMaxExperts, s);
         cudaMemsetAsync(p->ws.f_bar, 0, sizeof(uint32_t), s);
         cudaStreamSynchronize(s);
+        p->fused_bar_base = 0;
     }
     if (v & kStatusTimeout) return MOE_ERR_TIMEOUT;
     if (v & kStatusBadIndex) return MOE_ERR_DEVICE_CHECK;
