@@ -16,7 +16,8 @@
 //   router logits    z = W_g h is linear in h, so the CTA that finishes rows [r0, r1) of h_{l+1}
 //                    multiplies them at once with the columns [r0, r1) of the NEXT layer's W_g
 //                    (staged in shared memory while the down stream runs) and adds the partial
-//                    logits to a 64-bit fixed-point accumulator (2^-40 units) in global memory.
+//                    logits to 64-bit fixed-point accumulators (2^-40 units) in global memory, one
+//                    of 16 copies per CTA so that atomics on one cache line do not queue up.
 //                    Integer addition is associative, so the sum does not depend on arrival order
 //                    and every call gives the same bits.  The logits of the first layer come from
 //                    a pre-pass over x of the same form.
@@ -51,11 +52,14 @@ constexpr int kMaxPairsF = kFT * kMaxExperts;
 constexpr int kMaxCtaRows = kFusedMaxCtaRows;       // rows of h one CTA may own
 constexpr int kMaxSub = kMaxCtaRows / 16;           // ... in blocks of at most 16
 constexpr int kWgWords = kMaxCtaRows / 2 + 1;       // 32-bit words of one staged W_g row (even start)
-constexpr uint32_t kPrefetchChunks = 4;             // chunks of its next stream a warp asks L2 for ahead of a barrier
+constexpr uint32_t kPrefetchChunks = 6;             // chunks of its NEXT stream a warp asks L2 for when it starts a stream
 constexpr double kFixScale = 1099511627776.0;       // 2^40: logit partials are accumulated in units of 2^-40
 constexpr double kFixInv = 1.0 / 1099511627776.0;
+constexpr int kZCopies = kFusedZCopies;             // accumulator copies (CTA i adds to copy i % 16): same-line atomics serialise
+constexpr int kZCopyStride = kFT * kMaxExperts;     // one copy: [token][expert]
+constexpr int kZBufStride = kZCopies * kZCopyStride;
 
-static_assert(kFusedThreads >= kMaxExperts, "one thread per expert stages the router bias");
+static_assert(kFusedThreads >= kMaxExperts, "one thread per expert clears the per-layer tables");
 static_assert(kFusedWarps >= kFT, "one routing warp per token");
 static_assert(kFusedWarps >= kMaxSub, "one warp per row block in the pre-pass");
 
@@ -69,17 +73,15 @@ struct BlockTab {                         // gate/up row blocks of this CTA
 
 struct StackSmem {
     float logit[kFT][kMaxExperts];
-    float gtab[kMaxExperts][kFT];         // [touched-expert slot][token] gate weight (0 = not routed)
+    float gtab[kMaxExperts][kFT];         // [expert][token] gate weight times the routed scale (0 = not routed)
     float gamma[kFT];
     int32_t idx[kMaxPairsF];
     float w[kMaxPairsF];
     int32_t ulist[kMaxExperts];           // touched experts, ascending
-    int32_t uof[kMaxExperts];             // expert -> slot in ulist
     int32_t tokmask[kMaxExperts];
     int32_t cursor[kMaxExperts + 1];
     float4 wpart[2 * kFusedWarps][32];    // per-warp partial sums of row blocks split inside the CTA
     int32_t wticket[kFusedMaxCtaBlocks];  // arrival counters of this CTA's row blocks (zero between streams)
-    float bias[kMaxExperts];
     BlockTab tab_s, tab_r;                // shared expert (same every layer), touched experts (per layer)
     int32_t sub_row[kMaxSub], sub_n[kMaxSub];   // this CTA's rows of h in blocks of at most 16
     float hres[kFT][kMaxCtaRows];         // fp32 residual stream, this CTA's rows
@@ -130,6 +132,10 @@ __device__ __forceinline__ long long ldcg_s64(const long long *p) {
     asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
 }
+// adds to a 64-bit integer in global memory without waiting for (or asking for) the old value
+__device__ __forceinline__ void red_add_s64(long long *p, long long v) {
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
 // asks for one 128-byte line to be brought into L2 (no register, no wait)
 __device__ __forceinline__ void prefetch_l2(const void *p) {
     asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(p));
@@ -173,15 +179,15 @@ __device__ __forceinline__ void bar_arrive(uint32_t *bar) {
     __threadfence();
     atomicAdd(bar, 1u);
 }
-__device__ __forceinline__ bool bar_wait(const uint32_t *bar, uint32_t target, int32_t *status, unsigned long long limit_ns) {
+__device__ __forceinline__ bool bar_wait(const uint32_t *bar, uint32_t target, int32_t *status, unsigned long long limit_ns,
+                                         int which = 0) {
     const unsigned long long t0 = global_ns();
     uint32_t spins = 0;
     while ((int32_t)(ld_acquire(bar) - target) < 0) {
         if ((++spins & 63u) == 0 && global_ns() - t0 > limit_ns) {
-            atomicOr(status, kStatusTimeout);
+            atomicOr(status, kStatusTimeout | (0x100 << which));
             return false;
         }
-        __nanosleep(32);
     }
     __threadfence();
     return true;
@@ -362,7 +368,7 @@ __device__ __forceinline__ void logit_partial(const Ctx &x, int sub, long long *
             const int t = 2 * x.c + (i & 1);
             if (e < a.E && t < a.T) {
                 const long long v = __double2ll_rn((double)acc[i] * kFixScale);
-                atomicAdd(reinterpret_cast<unsigned long long *>(zacc + t * kMaxExperts + e), (unsigned long long)v);
+                red_add_s64(zacc + (blockIdx.x % kZCopies) * kZCopyStride + t * kMaxExperts + e, v);
             }
         }
     }
@@ -398,7 +404,7 @@ __device__ __forceinline__ void finish_block(const Ctx &x, uint32_t j, const flo
         }
         if (!x.last) {
             __syncwarp();
-            logit_partial(x, (int)j, a.zacc + (size_t)((x.layer + 1) & 1) * kFT * kMaxExperts);
+            logit_partial(x, (int)j, a.zacc + (size_t)((x.layer + 1) & 1) * kZBufStride);
         }
     } else {
         // row g = gate feature, row g + 8 = up feature of the same index
@@ -414,7 +420,7 @@ __device__ __forceinline__ void finish_block(const Ctx &x, uint32_t j, const flo
             uint32_t spins = 0;
             while (ld_volatile_shared(&x.sm.gamma_epoch) < want && ld_volatile_shared(&x.sm.abort) == 0) {
                 if ((++spins & 255u) == 0 && global_ns() - t0 > a.limit_ns) {
-                    atomicOr(a.status, kStatusTimeout);
+                    atomicOr(a.status, kStatusTimeout | 0x1000);
                     x.sm.abort = 1;
                     break;
                 }
@@ -425,7 +431,7 @@ __device__ __forceinline__ void finish_block(const Ctx &x, uint32_t j, const flo
         for (int i = 0; i < 2; ++i) {
             const int t = 2 * x.c + i;
             if (t < a.T) {
-                const float wgt = (PH == kPhShared1) ? x.sm.gamma[t] : x.sm.gtab[u][t];
+                const float wgt = (PH == kPhShared1) ? x.sm.gamma[t] : x.sm.gtab[x.sm.ulist[u]][t];
                 const float hv = wgt != 0.f ? wgt * silu_mul(v[i], v[2 + i]) : 0.f;
                 a.hbuf[(size_t)t * a.hs + hoff + feat] = __float2bfloat16_rn(hv);
             }
@@ -622,7 +628,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
         __syncwarp();
         logit_partial(ctx, warp, a.zacc);
     }
-    __threadfence();
     __syncthreads();
     bar_target += G;
     if (tid == 0) bar_arrive(a.bar);
@@ -633,16 +638,30 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
         const int k = ld.k;
         const int last = l == a.L - 1;
         ctx.layer = l; ctx.last = last; ctx.gated = (a.I_s > 0 && ld.w_s != nullptr) ? 1 : 0;
-        long long *zacc_cur = a.zacc + (size_t)(l & 1) * kFT * kMaxExperts;
+        long long *zacc_cur = a.zacc + (size_t)(l & 1) * kZBufStride;
+        // logit of (token t, expert e): the sum of the accumulator copies, exact, plus the router bias
+        auto logit_of = [&](int t, int e) -> float {
+            long long v[kZCopies];
+#pragma unroll
+            for (int cpy = 0; cpy < kZCopies; ++cpy) v[cpy] = ldcg_s64(zacc_cur + cpy * kZCopyStride + t * kMaxExperts + e);
+            long long sum = 0;
+#pragma unroll
+            for (int cpy = 0; cpy < kZCopies; ++cpy) sum += v[cpy];
+            return (float)((double)sum * kFixInv) + (ld.router_bias != nullptr ? __ldg(ld.router_bias + e) : 0.f);
+        };
         stamp(l, 0);
 
         // ---- h of this layer -> shared memory (layer 0: x, staged above); per-layer tables; the next
         //      layer's W_g columns are asked for now and used by the down stream's finishers
-        if (l > 0) load_xs(a.y);
-        if (tid < kMaxExperts) {
-            sm.tokmask[tid] = 0;
-            sm.bias[tid] = (ld.router_bias != nullptr && tid < E) ? ld.router_bias[tid] : 0.f;
+        if (l > 0) {
+            load_xs(a.y);
+            // behind the grid barrier the logits are complete: all threads add up the copies
+            for (int i = tid; i < T * E; i += kFusedThreads) {
+                const int t = i / E, e = i - t * E;
+                sm.logit[t][e] = logit_of(t, e);
+            }
         }
+        if (tid < kMaxExperts) sm.tokmask[tid] = 0;
         for (int i = tid; i < kMaxExperts * kFT; i += kFusedThreads) (&sm.gtab[0][0])[i] = 0.f;
         if (!last) stage_wg(a.layers[l + 1].router_W);
         __syncthreads();
@@ -685,27 +704,31 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
                 __threadfence_block();
                 atomicAdd(&sm.gamma_epoch, 1);
             }
-            // the first layer's logits are complete once every CTA has passed the pre-pass
+            // the first layer's logits are complete once every CTA has passed the pre-pass (the other
+            // warps do not wait: they stream the shared expert meanwhile)
             int ok = 1;
             if (l == 0) {
-                if (lane == 0) ok = bar_wait(a.bar, target_pre, a.status, a.limit_ns) ? 1 : 0;
+                if (lane == 0) ok = bar_wait(a.bar, target_pre, a.status, a.limit_ns, 1) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok && lane == 0) sm.abort = 1;
+                if (ok)
+                    for (int e = lane; e < E; e += 32) sm.logit[warp][e] = logit_of(warp, e);
+                __syncwarp();
             }
             if (ok) {
                 float z[kExpertsPerLane];
 #pragma unroll
                 for (int j = 0; j < kExpertsPerLane; ++j) {
                     const int e = lane + 32 * j;
-                    z[j] = 0.f;
-                    if (e < E) {
-                        z[j] = (float)((double)ldcg_s64(zacc_cur + warp * kMaxExperts + e) * kFixInv) + sm.bias[e];
-                        sm.logit[warp][e] = z[j];
-                    }
+                    z[j] = e < E ? sm.logit[warp][e] : 0.f;
                 }
                 warp_route(z, E, k, a.renorm, lane, sm.idx + warp * k, sm.w + warp * k);
                 __syncwarp();
-                for (int j = lane; j < k; j += 32) atomicOr(&sm.tokmask[sm.idx[warp * k + j]], 1 << warp);
+                for (int j = lane; j < k; j += 32) {
+                    const int e = sm.idx[warp * k + j];
+                    sm.gtab[e][warp] = a.routed_scale * sm.w[warp * k + j];
+                    atomicOr(&sm.tokmask[e], 1 << warp);
+                }
             }
         }
 
@@ -715,7 +738,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
         if (sm.abort) return;
         stamp(l, 2);
 
-        // ---- touched experts, gate weights per (slot, token), this CTA's blocks of the routed stream
+        // ---- touched experts (ascending), this CTA's blocks of the routed stream
         if (warp == 0) {
             int base = 0;
 #pragma unroll
@@ -723,11 +746,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
                 const int e = 32 * j + lane;
                 const bool has = e < E && sm.tokmask[e] != 0;
                 const unsigned m = __ballot_sync(0xffffffffu, has);
-                if (has) {
-                    const int pos = base + __popc(m & ((1u << lane) - 1u));
-                    sm.ulist[pos] = e;
-                    sm.uof[e] = pos;
-                }
+                if (has) sm.ulist[base + __popc(m & ((1u << lane) - 1u))] = e;
                 base += __popc(m);
             }
             if (lane == 0) sm.U = base;
@@ -751,8 +770,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
         __syncthreads();
         const int U = sm.U;
         const int n_pairs = T * k;
-        for (int p = tid; p < n_pairs; p += kFusedThreads) sm.gtab[sm.uof[sm.idx[p]]][p / k] = a.routed_scale * sm.w[p];
-        __syncthreads();
         stamp(l, 3);
 
         // ---- the last layer's routing is what moe_last_routing reports: warp 0 of CTA 0 publishes it
@@ -801,10 +818,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
             }
         }
 
-        // ---- gate/up stream of the touched experts
-        run_stream<kPhRouted1>(ctx, warp, (uint32_t)sm.nblk_r, NC1);
-
-        // head of this warp's share of the down stream: into L2 while the gate/up stream drains
+        // ---- gate/up stream of the touched experts.  Each stream is short (a few chunks per warp), so
+        //      its ramp and its drain would leave HBM idle for as long as a loaded round trip; the head
+        //      of this warp's share of the NEXT stream (the down projection, known now that the routing
+        //      is) is therefore asked for first: it arrives in L2 while this stream runs and drains.
         ctx.geo.NC2 = (uint32_t)U * ctx.geo.ncI + ctx.geo.ncIs;
         ctx.geo.nseg2 = (uint32_t)U + (ctx.geo.ncIs > 0 ? 1u : 0u);
         const uint32_t L2n = (uint32_t)nsub * ctx.geo.NC2;
@@ -816,32 +833,29 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
                     prefetch_chunk<kPh2>(ctx, q, (const __nv_bfloat16 *)ld.W_down, (const __nv_bfloat16 *)ld.Ws_down);
             }
         }
+        run_stream<kPhRouted1>(ctx, warp, (uint32_t)sm.nblk_r, NC1);
         cp_async_wait_all();                   // the next layer's W_g columns have landed
 
-        // ---- all of h' written
-        __threadfence();
+        // ---- all of h' written (thread 0's fence in bar_arrive, behind the CTA barrier, covers every
+        //      thread's stores: fences are cumulative)
         __syncthreads();
         stamp(l, 4);
         bar_target += G;
         if (tid == 0) {
             bar_arrive(a.bar);
-            if (!bar_wait(a.bar, bar_target, a.status, a.limit_ns)) sm.abort = 1;
+            if (!bar_wait(a.bar, bar_target, a.status, a.limit_ns, 2)) sm.abort = 1;
         }
         __syncthreads();
         if (sm.abort) return;
         stamp(l, 5);
         // every CTA has routed this layer: its logit accumulator is put back to zero for layer l + 2
         // (nothing adds to it before the next grid barrier)
-        if (cta == 0)
-            for (int i = tid; i < T * kMaxExperts; i += kFusedThreads) zacc_cur[i] = 0;
+        if (cta < (uint32_t)kZCopies)
+            for (int i = tid; i < T * kMaxExperts; i += kFusedThreads) zacc_cur[cta * kZCopyStride + i] = 0;
 
-        // ---- down stream over the concatenated reduction range [shared | touched experts], this CTA's rows
-        run_stream<kPh2>(ctx, warp, (uint32_t)nsub, ctx.geo.NC2);
-        stamp(l, 6);
-        if (last) break;
-
-        // head of this warp's share of the next layer's shared gate/up stream: into L2 across the barrier
-        if (a.I_s > 0) {
+        // ---- down stream over the concatenated reduction range [shared | touched experts], this CTA's rows;
+        //      first the head of this warp's share of the next layer's shared gate/up stream, into L2
+        if (!last && a.I_s > 0) {
             const uint32_t Ls = (uint32_t)sm.nblk_s * NC1;
             if (Ls > 0) {
                 const uint32_t Wls = Ls < (uint32_t)kFusedWarps ? Ls : (uint32_t)kFusedWarps;
@@ -853,13 +867,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
                 }
             }
         }
+        run_stream<kPh2>(ctx, warp, (uint32_t)nsub, ctx.geo.NC2);
+        stamp(l, 6);
+        if (last) break;
+
         // ---- h and the next layer's logits complete
-        __threadfence();
         __syncthreads();
         bar_target += G;
         if (tid == 0) {
             bar_arrive(a.bar);
-            if (!bar_wait(a.bar, bar_target, a.status, a.limit_ns)) sm.abort = 1;
+            if (!bar_wait(a.bar, bar_target, a.status, a.limit_ns, 3)) sm.abort = 1;
         }
         __syncthreads();
         if (sm.abort) return;

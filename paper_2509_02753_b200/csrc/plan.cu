@@ -368,11 +368,11 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
             fused_smem_bytes(c.d) <= 200 * 1024 && (c.d + sms - 1) / sms <= kFusedMaxCtaRows &&
             blocks_cta <= kFusedMaxCtaBlocks && blocks_cta_s <= kFusedMaxCtaBlocks) {
             p->fused_hs = c.I_shared + ucap * c.I;
-            bool fok = ws_alloc(p, &ws.f_zacc, (size_t)2 * kFusedMaxTokens * kMaxExperts) &&
+            bool fok = ws_alloc(p, &ws.f_zacc, (size_t)2 * kFusedZCopies * kFusedMaxTokens * kMaxExperts) &&
                        ws_alloc(p, &ws.f_bar, (size_t)4) &&
                        ws_alloc(p, &ws.f_hbuf, (size_t)kFusedMaxTokens * p->fused_hs) &&
                        ws_alloc(p, &ws.f_stamps, (size_t)sms * 8);
-            fok = fok && cudaMemset(ws.f_zacc, 0, sizeof(long long) * 2 * kFusedMaxTokens * kMaxExperts) == cudaSuccess &&
+            fok = fok && cudaMemset(ws.f_zacc, 0, sizeof(long long) * 2 * kFusedZCopies * kFusedMaxTokens * kMaxExperts) == cudaSuccess &&
                   cudaMemset(ws.f_bar, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess &&
                   fused_prepare(c.d) == cudaSuccess;
             if (!fok) { cudaGetLastError(); moe_plan_destroy(p); return MOE_ERR_WORKSPACE; }
@@ -854,10 +854,11 @@ int moe_device_status(moe_plan_t *p, void *cuda_stream) {
         return MOE_ERR_CUDA;
     }
     const int32_t v = *p->status_host;
+    if (v && getenv("LEXI_DEBUG_STATUS")) fprintf(stderr, "device status word 0x%x\n", v);
     if ((v & kStatusTimeout) && p->fused_ok) {
         // a one-launch call that gave up has left the barrier counter and the logit accumulators
         // half way: both start again from zero
-        cudaMemsetAsync(p->ws.f_zacc, 0, sizeof(long long) * 2 * kFusedMaxTokens * kMaxExperts, s);
+        cudaMemsetAsync(p->ws.f_zacc, 0, sizeof(long long) * 2 * kFusedZCopies * kFusedMaxTokens * kMaxExperts, s);
         cudaMemsetAsync(p->ws.f_bar, 0, sizeof(uint32_t), s);
         cudaStreamSynchronize(s);
         p->fused_bar_base = 0;
