@@ -65,8 +65,10 @@ def recorded_traffic(key):
             f = line.split()
             if len(f) == 4 and f[0] == "traffic_key" and f[1] == key:
                 src, sha = f[3].split(":")
-                cur = hashlib.sha256(open(os.path.join(ROOT, "paper_2509_02753_b200", "csrc", src),
-                                          "rb").read()).hexdigest()[:16]
+                path_src = os.path.join(ROOT, "paper_2509_02753_b200", "csrc", src)
+                if not os.path.exists(path_src):
+                    return None
+                cur = hashlib.sha256(open(path_src, "rb").read()).hexdigest()[:16]
                 return int(f[2]) if cur == sha else None
     return None
 
@@ -349,7 +351,7 @@ def run_ours(args):
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = recorded_traffic(f"{wl.name}_T{T}_k{k}_{'fused' if fused else 'ffn1'}")
     pairs = main["schedule"] == "prefill" and os.environ.get("LEXI_PREFILL_2CTA", "1") != "0"
-    roof["kernel"] = ("decode_fused_kernel (whole layer, one cooperative launch)" if fused
+    roof["kernel"] = ("decode_stack_kernel (whole layer, one cooperative launch)" if fused
                       else "ffn_tc_pair_kernel<phase 1> (gate/up GEMM + SwiGLU, CTA pairs)" if pairs
                       else "ffn_tc_kernel<phase 1> (gate/up GEMM + SwiGLU)")
     roof["launch_ms"] = stages.get("ffn1")

@@ -359,7 +359,7 @@ int moe_debug_wait_timeout(moe_plan_t *plan, int32_t limit_us, void *cuda_stream
  * barrier counter never reaches, with a limit of limit_us microseconds (1 .. 1,000,000).  The wait
  * gives up and sets the time-out bit of the device status word.  While that bit is set every
  * one-launch call returns at once without computing; moe_device_status reports MOE_ERR_TIMEOUT,
- * clears the bit and puts the barrier counter and the logit accumulators back to zero, after which
+ * clears the bit and puts the barrier counter back to zero, after which
  * one-launch calls work again.  Errors: INVALID_ARG (also when the plan has no one-launch layer), CUDA.
  */
 int moe_debug_barrier_timeout(moe_plan_t *plan, int32_t limit_us, void *cuda_stream);

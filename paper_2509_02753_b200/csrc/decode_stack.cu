@@ -15,16 +15,16 @@
 //                    meet between CTAs), and publishes their bf16 rounding for the other CTAs.
 //   router logits    z = W_g h is linear in h, so the CTA that finishes rows [r0, r1) of h_{l+1}
 //                    multiplies them at once with the columns [r0, r1) of the NEXT layer's W_g
-//                    (staged in shared memory while the down stream runs) and adds the partial
-//                    logits to 64-bit fixed-point accumulators (2^-40 units) in global memory, one
-//                    of 16 copies per CTA so that atomics on one cache line do not queue up.
-//                    Integer addition is associative, so the sum does not depend on arrival order
-//                    and every call gives the same bits.  The logits of the first layer come from
-//                    a pre-pass over x of the same form.
+//                    (staged in shared memory while the down stream runs) and stores the partial
+//                    logits in its own slot in global memory (plain stores: atomics on shared
+//                    accumulators queued up for microseconds).  Behind the grid barrier every CTA
+//                    adds the G partials up in CTA order, so every CTA - and every call - gets the
+//                    same bits.  The logits of the first layer come from a pre-pass over x of the
+//                    same form.
 //   per layer        grid barrier (h and logits complete) -> every CTA copies h into shared memory
 //                    -> warps 0..T-1 route one token each (TopK + Softmax, same code everywhere, so
 //                    all CTAs agree) while the other warps already stream the shared expert's
-//                    gate/up rows -> gate/up stream of the touched experts, h' = g[t,e] silu(gate)
+//                    gate/up rows (the routing warps take a third of a share of that stream) -> gate/up stream of the touched experts, h' = g[t,e] silu(gate)
 //                    up in bf16 -> grid barrier -> down stream over [shared | touched experts] ->
 //                    h += y.  Two grid barriers per layer, none inside a stream.
 //
@@ -52,16 +52,11 @@ constexpr int kMaxPairsF = kFT * kMaxExperts;
 constexpr int kMaxCtaRows = kFusedMaxCtaRows;       // rows of h one CTA may own
 constexpr int kMaxSub = kMaxCtaRows / 16;           // ... in blocks of at most 16
 constexpr int kWgWords = kMaxCtaRows / 2 + 1;       // 32-bit words of one staged W_g row (even start)
-constexpr uint32_t kPrefetchChunks = 6;             // chunks of its NEXT stream a warp asks L2 for when it starts a stream
-constexpr double kFixScale = 1099511627776.0;       // 2^40: logit partials are accumulated in units of 2^-40
-constexpr double kFixInv = 1.0 / 1099511627776.0;
-constexpr int kZCopies = kFusedZCopies;             // accumulator copies (CTA i adds to copy i % 16): same-line atomics serialise
-constexpr int kZCopyStride = kFT * kMaxExperts;     // one copy: [token][expert]
-constexpr int kZBufStride = kZCopies * kZCopyStride;
+constexpr int kZSlot = kFT * kMaxExperts;           // floats of one CTA's slot of logit partials, [token][expert]
+constexpr int kStreamerWeight = 3;                  // share of the shared-expert stream of a warp that does not route (routing warps: 1)
 
 static_assert(kFusedThreads >= kMaxExperts, "one thread per expert clears the per-layer tables");
 static_assert(kFusedWarps >= kFT, "one routing warp per token");
-static_assert(kFusedWarps >= kMaxSub, "one warp per row block in the pre-pass");
 
 enum { kPhShared1 = 0, kPhRouted1 = 1, kPh2 = 2 };
 
@@ -86,7 +81,8 @@ struct StackSmem {
     int32_t sub_row[kMaxSub], sub_n[kMaxSub];   // this CTA's rows of h in blocks of at most 16
     float hres[kFT][kMaxCtaRows];         // fp32 residual stream, this CTA's rows
     uint32_t wg_raw[kMaxExperts][kWgWords];     // columns [r0 & ~1, r1) of the next layer's W_g
-    __nv_bfloat16 hb[kMaxSub][kFT][16];   // a finished block of h, [token][row], operand of the logit partials
+    __nv_bfloat16 hnew[kFT][kMaxCtaRows]; // this CTA's rows of the layer's result h (bf16), operand of the logit partials
+    float4 zsl[kFusedThreads];            // sums over a slice of the CTAs' slots, [slice][token x 4-expert column]
     int32_t nblk_s, nblk_r, nsub;
     int32_t r0, r1;                       // this CTA's rows of h
     int32_t U;
@@ -127,18 +123,10 @@ __device__ __forceinline__ uint4 ldcg_pinned(const __nv_bfloat16 *p) {
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ long long ldcg_s64(const long long *p) {
-    long long v;
-    asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+__device__ __forceinline__ float4 ldcg_f4(const float *p) {
+    float4 v;
+    asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
     return v;
-}
-// adds to a 64-bit integer in global memory without waiting for (or asking for) the old value
-__device__ __forceinline__ void red_add_s64(long long *p, long long v) {
-    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-// asks for one 128-byte line to be brought into L2 (no register, no wait)
-__device__ __forceinline__ void prefetch_l2(const void *p) {
-    asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(p));
 }
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p) {
     uint32_t v;
@@ -154,6 +142,12 @@ __device__ __forceinline__ void cp_async4(void *smem_dst, const void *gmem_src) 
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
                  : "memory");
 }
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_but_last() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
@@ -310,68 +304,107 @@ struct LoadCursor {
     }
 };
 
-// L2 prefetch of chunk q of one of this CTA's streams: 16 rows x 256 bytes = one 128-byte line per lane.
-// For the gate/up streams the rows are 8 of W_gate and the same 8 of W_up.
-template <int PH>
-__device__ __forceinline__ void prefetch_chunk(const Ctx &x, uint32_t q, const __nv_bfloat16 *Wa, const __nv_bfloat16 *Wb) {
-    const StackArgs &a = x.a;
-    const uint32_t r = (uint32_t)x.lane >> 1, half = (uint32_t)x.lane & 1u;
-    if (PH == kPhShared1) {
-        const uint32_t j = q / x.geo.NC1, kc = q - j * x.geo.NC1;
-        const uint32_t f = r & 7u;
-        const uint32_t col = kc * kChunk + half * 64;
-        if (f < x.sm.tab_s.n[j] && col < (uint32_t)a.d)
-            prefetch_l2((r < 8 ? Wa : Wb) + (size_t)(x.sm.tab_s.row[j] + f) * a.d + col);
-    } else {
-        const uint32_t j = q / x.geo.NC2;
-        const uint32_t rr = q - j * x.geo.NC2;
-        if ((int)r >= x.sm.sub_n[j]) return;
-        const uint32_t row = (uint32_t)x.sm.sub_row[j] + r;
-        const __nv_bfloat16 *p;
-        uint32_t kc, K;
-        if (rr < x.geo.ncIs) {
-            kc = rr; K = a.I_s;
-            p = Wb + (size_t)row * a.I_s;
-        } else {
-            const uint32_t r2 = rr - x.geo.ncIs;
-            const uint32_t slot = r2 / x.geo.ncI;
-            kc = r2 - slot * x.geo.ncI; K = a.I;
-            p = Wa + ((size_t)x.sm.ulist[slot] * a.d + row) * a.I;
-        }
-        const uint32_t col = kc * kChunk + half * 64;
-        if (col < K) prefetch_l2(p + col);
+// Partial logits of the next layer from this CTA's finished rows of h, all threads of the CTA behind
+// a CTA barrier that follows the down stream: thread (t, e) adds W_g[e, r0 + k] h[t, r0 + k] over the
+// CTA's rows in row order (fp32; the products of bf16 values are exact) and stores the sum in this
+// CTA's slot.  A CTA without rows stores zeros.
+__device__ __forceinline__ void store_logit_partials(const StackArgs &a, const StackSmem &sm, int tid) {
+    float *slot = a.zslot + (size_t)blockIdx.x * kZSlot;
+    const int n = sm.r1 - sm.r0, off = sm.r0 & 1;          // the staged W_g rows start at the even column r0 & ~1
+    for (int i = tid; i < a.T * a.E; i += kFusedThreads) {
+        const int t = i / a.E, e = i - t * a.E;
+        const __nv_bfloat16 *wrow = reinterpret_cast<const __nv_bfloat16 *>(sm.wg_raw[e]) + off;
+        float acc = 0.f;
+        for (int k = 0; k < n; ++k) acc = fmaf(__bfloat162float(wrow[k]), __bfloat162float(sm.hnew[t][k]), acc);
+        __stcg(slot + t * kMaxExperts + e, acc);
     }
 }
 
-// Partial logits of the next layer from a finished block of h: z[e][t] += sum_k W_g[e, row0 + k] hb[t][k],
-// in 2^-40 units on a 64-bit integer accumulator (exact, order-independent).
-__device__ __forceinline__ void logit_partial(const Ctx &x, int sub, long long *zacc) {
-    const StackArgs &a = x.a;
-    const int n = x.sm.sub_n[sub];
-    const int off = x.sm.sub_row[sub] - (x.sm.r0 & ~1);          // halfword offset inside the staged rows
-    const uint32_t b0 = *reinterpret_cast<const uint32_t *>(&x.sm.hb[sub][x.g][2 * x.c]);
-    const uint32_t b1 = *reinterpret_cast<const uint32_t *>(&x.sm.hb[sub][x.g][2 * x.c + 8]);
-    for (int m0 = 0; m0 < a.E; m0 += 16) {
-        auto ld2 = [&](int e, int k) -> uint32_t {               // W_g[e, row0 + k], W_g[e, row0 + k + 1]
-            if (e >= a.E) return 0u;
-            const unsigned short *row = reinterpret_cast<const unsigned short *>(x.sm.wg_raw[e]);
-            const uint32_t lo = k < n ? row[off + k] : 0u;
-            const uint32_t hi = k + 1 < n ? row[off + k + 1] : 0u;
-            return lo | (hi << 16);
-        };
-        const int e_lo = m0 + x.g, e_hi = e_lo + 8;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        mma16816(acc, ld2(e_lo, 2 * x.c), ld2(e_hi, 2 * x.c), ld2(e_lo, 2 * x.c + 8), ld2(e_hi, 2 * x.c + 8), b0, b1);
+// Logits of the tokens [t0, t0 + nt) from the G slots, by a group of gsize threads (the whole CTA, or
+// the one warp that routes token t0): thread (slice, column) adds the slots of its slice of the CTAs in
+// CTA order for four neighbouring experts, then the slices are added in slice order.  Every CTA
+// does the same sums in the same order.  sync() separates the two passes (CTA or warp barrier).
+template <typename Sync>
+__device__ __forceinline__ void sum_logits(const StackArgs &a, StackSmem &sm, float4 *zsl, int gtid, int gsize, int t0, int nt,
+                                           const float *bias, uint32_t G, Sync sync) {
+    const int ecol = (a.E + 3) >> 2, ncol = nt * ecol;
+    int nslice = gsize / ncol;
+    if (nslice < 1) nslice = 1;
+    if (nslice > (int)G) nslice = (int)G;
+    for (int i = gtid; i < ncol * nslice; i += gsize) {
+        const int sl = i / ncol, col = i - sl * ncol;
+        const int t = t0 + col / ecol, e4 = (col % ecol) * 4;
+        const uint32_t c0 = (uint32_t)sl * G / nslice, c1 = ((uint32_t)sl + 1) * G / nslice;
+        const float *p = a.zslot + (size_t)c0 * kZSlot + t * kMaxExperts + e4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (uint32_t cc = c0; cc < c1; cc += 16) {              // sixteen loads in flight, added in CTA order
+            float4 v[16];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int e = (i >> 1) ? e_hi : e_lo;
-            const int t = 2 * x.c + (i & 1);
-            if (e < a.E && t < a.T) {
-                const long long v = __double2ll_rn((double)acc[i] * kFixScale);
-                red_add_s64(zacc + (blockIdx.x % kZCopies) * kZCopyStride + t * kMaxExperts + e, v);
-            }
+            for (int u = 0; u < 16; ++u)
+                v[u] = cc + u < c1 ? ldcg_f4(p + (size_t)(cc - c0 + u) * kZSlot) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 16; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+        }
+        zsl[i] = acc;
+    }
+    sync();
+    for (int i = gtid; i < nt * a.E; i += gsize) {
+        const int tt = i / a.E, e = i - tt * a.E;
+        const int col = tt * ecol + (e >> 2);
+        float v = 0.f;
+        for (int sl = 0; sl < nslice; ++sl) v += reinterpret_cast<const float *>(&zsl[sl * ncol + col])[e & 3];
+        sm.logit[t0 + tt][e] = v + (bias != nullptr ? __ldg(bias + e) : 0.f);
+    }
+    sync();
+}
+
+// TopK + Softmax of one token by one warp from its row of logits in shared memory.  Every lane
+// ranks its experts against all E logits (larger first, equal -> lower index), so the rank is the
+// slot in the descending order and no pass over the row depends on the one before; the gates are
+// exp(z - max) over the sum of the selected (renorm) or of all experts.
+template <int NJ>
+__device__ __forceinline__ void route_token_n(const float *zrow, int E, int k, int renorm, int lane, int32_t *idx_out, float *w_out) {
+    float z[NJ];
+    int rank[NJ];
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+        const int e = lane + 32 * j;
+        z[j] = e < E ? zrow[e] : -CUDART_INF_F;
+        rank[j] = 0;
+    }
+    for (int e2 = 0; e2 < E; ++e2) {
+        const float o = zrow[e2];
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) {
+            const int e = lane + 32 * j;
+            rank[j] += (o > z[j] || (o == z[j] && e2 < e)) ? 1 : 0;
         }
     }
+    float m = z[0];
+#pragma unroll
+    for (int j = 1; j < NJ; ++j) m = fmaxf(m, z[j]);
+    m = warp_max(m);
+    float p[NJ], s_all = 0.f, s_sel = 0.f;
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+        const int e = lane + 32 * j;
+        p[j] = e < E ? expf(z[j] - m) : 0.f;
+        s_all += p[j];
+        if (e < E && rank[j] < k) s_sel += p[j];
+    }
+    s_all = warp_sum(s_all);
+    s_sel = warp_sum(s_sel);
+    const float inv = 1.0f / (renorm ? s_sel : s_all);
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+        const int e = lane + 32 * j;
+        if (e < E && rank[j] < k) { idx_out[rank[j]] = e; w_out[rank[j]] = p[j] * inv; }
+    }
+}
+__device__ __forceinline__ void route_token(const float *zrow, int E, int k, int renorm, int lane, int32_t *idx_out, float *w_out) {
+    if (E <= 32) route_token_n<1>(zrow, E, k, renorm, lane, idx_out, w_out);
+    else if (E <= 64) route_token_n<2>(zrow, E, k, renorm, lane, idx_out, w_out);
+    else route_token_n<kExpertsPerLane>(zrow, E, k, renorm, lane, idx_out, w_out);
 }
 
 // Finishes a row block from its complete sums v[4]: v[0], v[1] = row g, tokens 2c, 2c+1;
@@ -387,7 +420,6 @@ __device__ __forceinline__ void finish_block(const Ctx &x, uint32_t j, const flo
         for (int i = 0; i < 4; ++i) {
             const int t = 2 * x.c + (i & 1);
             const int kk = x.g + (i >> 1) * 8;
-            __nv_bfloat16 hb16 = __float2bfloat16_rn(0.f);
             if (t < a.T && kk < n) {
                 const int row = row0 + kk;
                 const size_t off = (size_t)t * a.d + row;
@@ -397,14 +429,10 @@ __device__ __forceinline__ void finish_block(const Ctx &x, uint32_t j, const flo
                     x.sm.hres[t][row - x.sm.r0] = hn;
                     if (x.last) a.h_run[off] = hn;
                 }
-                hb16 = __float2bfloat16_rn(hn);
+                const __nv_bfloat16 hb16 = __float2bfloat16_rn(hn);
                 a.y[off] = hb16;
+                x.sm.hnew[t][row - x.sm.r0] = hb16;
             }
-            x.sm.hb[j][t][kk] = hb16;
-        }
-        if (!x.last) {
-            __syncwarp();
-            logit_partial(x, (int)j, a.zacc + (size_t)((x.layer + 1) & 1) * kZBufStride);
         }
     } else {
         // row g = gate feature, row g + 8 = up feature of the same index
@@ -439,16 +467,35 @@ __device__ __forceinline__ void finish_block(const Ctx &x, uint32_t j, const flo
     }
 }
 
-// One stream inside a CTA: nblk row blocks of NC chunks each, a flat list the warps cut into equal
-// contiguous pieces.
+// Where warp w's piece of a stream of L chunks starts.  light = 0: Wl equal pieces.  light > 0: the
+// first `light` warps (the routing warps, which join the stream late) have weight 1, the others
+// kStreamerWeight.
+__device__ __forceinline__ uint32_t piece_start(uint32_t w, uint32_t Wl, uint32_t L, uint32_t light) {
+    if (light == 0) return w * L / Wl;
+    const uint32_t cw = w < light ? w : light + (w - light) * kStreamerWeight;
+    const uint32_t W = light + (Wl - light) * kStreamerWeight;
+    return (uint32_t)((unsigned long long)cw * L / W);
+}
+// The warp whose piece holds chunk q (inverse of piece_start).
+__device__ __forceinline__ uint32_t piece_owner(uint32_t q, uint32_t Wl, uint32_t L, uint32_t light) {
+    if (light == 0) return ((q + 1) * Wl - 1) / L;
+    const uint32_t W = light + (Wl - light) * kStreamerWeight;
+    const uint32_t cw = (uint32_t)((((unsigned long long)q + 1) * W - 1) / L);     // largest cumulative weight that starts at or before q
+    return cw < light ? cw : light + (cw - light) / kStreamerWeight;
+}
+
+// One stream inside a CTA: nblk row blocks of NC chunks each, a flat list the warps cut into
+// contiguous pieces (equal, or weighted as piece_start says).
 template <int PH>
-__device__ __forceinline__ void run_stream(const Ctx &x, int warp, uint32_t nblk, uint32_t NC) {
+__device__ __forceinline__ void run_stream(const Ctx &x, int warp, uint32_t nblk, uint32_t NC, uint32_t light = 0) {
     const uint32_t L = nblk * NC;
     if (L == 0) return;
     const uint32_t Wl = L < (uint32_t)kFusedWarps ? L : (uint32_t)kFusedWarps;
+    if (light >= Wl || L < 4u * Wl) light = 0;
     if ((uint32_t)warp >= Wl) return;
-    const uint32_t qa = (uint32_t)warp * L / Wl;
-    const uint32_t qb = ((uint32_t)warp + 1) * L / Wl;
+    const uint32_t qa = piece_start((uint32_t)warp, Wl, L, light);
+    const uint32_t qb = piece_start((uint32_t)warp + 1, Wl, L, light);
+    if (qa == qb) return;
     Frag f[2];
     FragB fb[2];
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -479,9 +526,8 @@ __device__ __forceinline__ void run_stream(const Ctx &x, int warp, uint32_t nblk
             }
             if (q + 1 == blk_end || q + 1 == qb) {
                 // the warps that share block rb
-                const uint32_t lo = rb * NC, hi = (rb + 1) * NC;
-                const uint32_t first = ((lo + 1) * Wl - 1) / L;
-                const uint32_t last = (hi * Wl - 1) / L;
+                const uint32_t first = piece_owner(rb * NC, Wl, L, light);
+                const uint32_t last = piece_owner((rb + 1) * NC - 1, Wl, L, light);
                 if (first == last) {
                     finish_block<PH>(x, rb, acc);
                 } else {
@@ -495,7 +541,7 @@ __device__ __forceinline__ void run_stream(const Ctx &x, int warp, uint32_t nblk
                     if (is_last) {
                         __threadfence_block();
                         float v[4] = {0.f, 0.f, 0.f, 0.f};
-                        const uint32_t qa_first = first * L / Wl;
+                        const uint32_t qa_first = piece_start(first, Wl, L, light);
                         for (uint32_t w2 = first; w2 <= last; ++w2) {
                             // a warp after the first starts inside this block: it used its head slot
                             const uint32_t slot2 = 2 * w2 + ((w2 == first && rb != qa_first / NC) ? 1u : 0u);
@@ -568,27 +614,24 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
             cp_async4(&sm.wg_raw[e][w], W + (size_t)e * a.d + rbase + 2 * w);
         }
     };
-    auto load_xs = [&](const __nv_bfloat16 *src) {      // h (or x) -> shared memory; rows >= T and the padding are zero
-        const int vec_per_row = xstride / 8;
-        for (int i0 = tid; i0 < kFT * vec_per_row; i0 += 4 * kFusedThreads) {   // four loads in flight per thread
-            uint4 v[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i = i0 + u * kFusedThreads;
-                const int row = i / vec_per_row, col = (i - row * vec_per_row) * 8;
-                v[u] = make_uint4(0u, 0u, 0u, 0u);
-                if (row < T && col < a.d) v[u] = __ldcg(reinterpret_cast<const uint4 *>(src + (size_t)row * a.d + col));
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i = i0 + u * kFusedThreads;
-                const int row = i / vec_per_row, col = (i - row * vec_per_row) * 8;
-                if (i < kFT * vec_per_row) *reinterpret_cast<uint4 *>(xs + row * xstride + col) = v[u];
-            }
+    // h (or x) -> shared memory, asynchronously (cp.async: no registers, other loads can be in flight
+    // meanwhile).  Rows >= T and the padding are zeroed once; only the rows < T change per layer.
+    const int dvec = a.d / 8;
+    auto xs_copy = [&](const __nv_bfloat16 *src) {
+        for (int i = tid; i < T * dvec; i += kFusedThreads) {
+            const int row = i / dvec, col = (i - row * dvec) * 8;
+            cp_async16(xs + row * xstride + col, src + (size_t)row * a.d + col);
         }
     };
+    {
+        const int vec_per_row = xstride / 8;
+        for (int i = tid; i < kFT * vec_per_row; i += kFusedThreads) {
+            const int row = i / vec_per_row, col = (i - row * vec_per_row) * 8;
+            if (row >= T || col >= a.d) *reinterpret_cast<uint4 *>(xs + row * xstride + col) = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
     stage_wg(a.layers[0].router_W);
-    load_xs((const __nv_bfloat16 *)a.x);
+    xs_copy((const __nv_bfloat16 *)a.x);
     if (tid == 0) {
         sm.abort = 0; sm.gamma_epoch = 0;
         sm.r0 = r0; sm.r1 = r1; sm.nsub = nsub;
@@ -612,22 +655,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
     __syncthreads();
 
     // ---- pre-pass: this CTA's rows of x start the residual stream and give the first layer's logit partials
-    if (warp < nsub) {
-        const int n = sm.sub_n[warp], row0 = sm.sub_row[warp];
-        for (int i = lane; i < kFT * 16; i += 32) {
-            const int t = i >> 4, kk = i & 15;
-            __nv_bfloat16 v = __float2bfloat16_rn(0.f);
-            if (t < T && kk < n) {
-                const int row = row0 + kk;
-                v = xs[t * xstride + row];
-                if (a.mode == 1)
-                    sm.hres[t][row - r0] = a.resume ? a.h_run[(size_t)t * a.d + row] : __bfloat162float(v);
-            }
-            sm.hb[warp][t][kk] = v;
-        }
-        __syncwarp();
-        logit_partial(ctx, warp, a.zacc);
+    for (int i = tid; i < T * nrows; i += kFusedThreads) {
+        const int t = i / nrows, kk = i - t * nrows;
+        const __nv_bfloat16 v = xs[t * xstride + r0 + kk];
+        sm.hnew[t][kk] = v;
+        if (a.mode == 1) sm.hres[t][kk] = a.resume ? a.h_run[(size_t)t * a.d + r0 + kk] : __bfloat162float(v);
     }
+    __syncthreads();
+    store_logit_partials(a, sm, tid);
     __syncthreads();
     bar_target += G;
     if (tid == 0) bar_arrive(a.bar);
@@ -638,33 +673,26 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
         const int k = ld.k;
         const int last = l == a.L - 1;
         ctx.layer = l; ctx.last = last; ctx.gated = (a.I_s > 0 && ld.w_s != nullptr) ? 1 : 0;
-        long long *zacc_cur = a.zacc + (size_t)(l & 1) * kZBufStride;
-        // logit of (token t, expert e): the sum of the accumulator copies, exact, plus the router bias
-        auto logit_of = [&](int t, int e) -> float {
-            long long v[kZCopies];
-#pragma unroll
-            for (int cpy = 0; cpy < kZCopies; ++cpy) v[cpy] = ldcg_s64(zacc_cur + cpy * kZCopyStride + t * kMaxExperts + e);
-            long long sum = 0;
-#pragma unroll
-            for (int cpy = 0; cpy < kZCopies; ++cpy) sum += v[cpy];
-            return (float)((double)sum * kFixInv) + (ld.router_bias != nullptr ? __ldg(ld.router_bias + e) : 0.f);
-        };
         stamp(l, 0);
 
         // ---- h of this layer -> shared memory (layer 0: x, staged above); per-layer tables; the next
-        //      layer's W_g columns are asked for now and used by the down stream's finishers
-        if (l > 0) {
-            load_xs(a.y);
-            // behind the grid barrier the logits are complete: all threads add up the copies
-            for (int i = tid; i < T * E; i += kFusedThreads) {
-                const int t = i / E, e = i - t * E;
-                sm.logit[t][e] = logit_of(t, e);
-            }
-        }
+        //      layer's W_g columns are asked for now and used after the down stream.  Behind a grid
+        //      barrier the logit partials are complete and all threads add them up.
+        if (l > 0) xs_copy(a.y);
+        cp_async_commit();
         if (tid < kMaxExperts) sm.tokmask[tid] = 0;
         for (int i = tid; i < kMaxExperts * kFT; i += kFusedThreads) (&sm.gtab[0][0])[i] = 0.f;
         if (!last) stage_wg(a.layers[l + 1].router_W);
-        __syncthreads();
+        cp_async_commit();
+        if (l == 0) {          // the first layer's logit partials are complete once every CTA has passed the pre-pass
+            if (tid == 0 && !bar_wait(a.bar, target_pre, a.status, a.limit_ns, 1)) sm.abort = 1;
+            __syncthreads();
+            if (sm.abort) return;
+        }
+        sum_logits(a, sm, sm.zsl, tid, kFusedThreads, 0, T, ld.router_bias, G, [&] {
+            cp_async_wait_but_last();      // h has landed (the W_g columns may still be on their way)
+            __syncthreads();
+        });
         stamp(l, 1);
 
         // ---- warps 0..T-1: the shared expert's gate, then TopK + Softmax of one token each
@@ -704,36 +732,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
                 __threadfence_block();
                 atomicAdd(&sm.gamma_epoch, 1);
             }
-            // the first layer's logits are complete once every CTA has passed the pre-pass (the other
-            // warps do not wait: they stream the shared expert meanwhile)
-            int ok = 1;
-            if (l == 0) {
-                if (lane == 0) ok = bar_wait(a.bar, target_pre, a.status, a.limit_ns, 1) ? 1 : 0;
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok && lane == 0) sm.abort = 1;
-                if (ok)
-                    for (int e = lane; e < E; e += 32) sm.logit[warp][e] = logit_of(warp, e);
-                __syncwarp();
-            }
-            if (ok) {
-                float z[kExpertsPerLane];
-#pragma unroll
-                for (int j = 0; j < kExpertsPerLane; ++j) {
-                    const int e = lane + 32 * j;
-                    z[j] = e < E ? sm.logit[warp][e] : 0.f;
-                }
-                warp_route(z, E, k, a.renorm, lane, sm.idx + warp * k, sm.w + warp * k);
-                __syncwarp();
-                for (int j = lane; j < k; j += 32) {
-                    const int e = sm.idx[warp * k + j];
-                    sm.gtab[e][warp] = a.routed_scale * sm.w[warp * k + j];
-                    atomicOr(&sm.tokmask[e], 1 << warp);
-                }
+            route_token(sm.logit[warp], E, k, a.renorm, lane, sm.idx + warp * k, sm.w + warp * k);
+            __syncwarp();
+            for (int j = lane; j < k; j += 32) {
+                const int e = sm.idx[warp * k + j];
+                sm.gtab[e][warp] = a.routed_scale * sm.w[warp * k + j];
+                atomicOr(&sm.tokmask[e], 1 << warp);
             }
         }
 
         // ---- shared expert, gate/up stream (needs no routing)
-        if (a.I_s > 0) run_stream<kPhShared1>(ctx, warp, (uint32_t)sm.nblk_s, NC1);
+        if (a.I_s > 0) run_stream<kPhShared1>(ctx, warp, (uint32_t)sm.nblk_s, NC1, (uint32_t)T);
         __syncthreads();
         if (sm.abort) return;
         stamp(l, 2);
@@ -818,22 +827,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
             }
         }
 
-        // ---- gate/up stream of the touched experts.  Each stream is short (a few chunks per warp), so
-        //      its ramp and its drain would leave HBM idle for as long as a loaded round trip; the head
-        //      of this warp's share of the NEXT stream (the down projection, known now that the routing
-        //      is) is therefore asked for first: it arrives in L2 while this stream runs and drains.
+        // ---- gate/up stream of the touched experts
+        run_stream<kPhRouted1>(ctx, warp, (uint32_t)sm.nblk_r, NC1);
+
         ctx.geo.NC2 = (uint32_t)U * ctx.geo.ncI + ctx.geo.ncIs;
         ctx.geo.nseg2 = (uint32_t)U + (ctx.geo.ncIs > 0 ? 1u : 0u);
-        const uint32_t L2n = (uint32_t)nsub * ctx.geo.NC2;
-        if (L2n > 0) {
-            const uint32_t Wl2 = L2n < (uint32_t)kFusedWarps ? L2n : (uint32_t)kFusedWarps;
-            if ((uint32_t)warp < Wl2) {
-                const uint32_t qa2 = (uint32_t)warp * L2n / Wl2, qb2 = ((uint32_t)warp + 1) * L2n / Wl2;
-                for (uint32_t q = qa2; q < qb2 && q < qa2 + kPrefetchChunks; ++q)
-                    prefetch_chunk<kPh2>(ctx, q, (const __nv_bfloat16 *)ld.W_down, (const __nv_bfloat16 *)ld.Ws_down);
-            }
-        }
-        run_stream<kPhRouted1>(ctx, warp, (uint32_t)sm.nblk_r, NC1);
         cp_async_wait_all();                   // the next layer's W_g columns have landed
 
         // ---- all of h' written (thread 0's fence in bar_arrive, behind the CTA barrier, covers every
@@ -848,30 +846,15 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
         __syncthreads();
         if (sm.abort) return;
         stamp(l, 5);
-        // every CTA has routed this layer: its logit accumulator is put back to zero for layer l + 2
-        // (nothing adds to it before the next grid barrier)
-        if (cta < (uint32_t)kZCopies)
-            for (int i = tid; i < T * kMaxExperts; i += kFusedThreads) zacc_cur[cta * kZCopyStride + i] = 0;
 
-        // ---- down stream over the concatenated reduction range [shared | touched experts], this CTA's rows;
-        //      first the head of this warp's share of the next layer's shared gate/up stream, into L2
-        if (!last && a.I_s > 0) {
-            const uint32_t Ls = (uint32_t)sm.nblk_s * NC1;
-            if (Ls > 0) {
-                const uint32_t Wls = Ls < (uint32_t)kFusedWarps ? Ls : (uint32_t)kFusedWarps;
-                if ((uint32_t)warp < Wls) {
-                    const uint32_t qa = (uint32_t)warp * Ls / Wls, qb = ((uint32_t)warp + 1) * Ls / Wls;
-                    for (uint32_t q = qa; q < qb && q < qa + kPrefetchChunks; ++q)
-                        prefetch_chunk<kPhShared1>(ctx, q, (const __nv_bfloat16 *)a.layers[l + 1].Ws_gate,
-                                                   (const __nv_bfloat16 *)a.layers[l + 1].Ws_up);
-                }
-            }
-        }
+        // ---- down stream over the concatenated reduction range [shared | touched experts], this CTA's rows
         run_stream<kPh2>(ctx, warp, (uint32_t)nsub, ctx.geo.NC2);
         stamp(l, 6);
         if (last) break;
 
         // ---- h and the next layer's logits complete
+        __syncthreads();
+        store_logit_partials(a, sm, tid);
         __syncthreads();
         bar_target += G;
         if (tid == 0) {

@@ -60,7 +60,7 @@ struct Workspace {
     int32_t *stats = nullptr;      // [4] counters read by moe_plan_touched_experts
     int32_t *pos = nullptr;        // [E, 128] direct mode: output row of (expert, token) or -1
     // one-launch stack for calls of at most kFusedMaxTokens tokens (decode_stack.cu)
-    long long *f_zacc = nullptr;   // [2][kFusedZCopies][8][kMaxExperts] fixed-point logit accumulators (zero between launches)
+    float *f_zslot = nullptr;      // [SMs][8][kMaxExperts] per-CTA partial router logits
     uint32_t *f_bar = nullptr;     // grid-barrier counter (only grows; the plan tracks its value)
     __nv_bfloat16 *f_hbuf = nullptr;  // [8, I_s + U_cap * I] gate-weighted hidden activations
     unsigned long long *f_stamps = nullptr;   // [SMs, 8] %globaltimer stamps of the last stamped call
@@ -161,7 +161,6 @@ constexpr int kFusedWarps = LEXI_FUSED_WARPS;
 constexpr int kFusedThreads = kFusedWarps * 32;
 constexpr int kFusedMaxCtaBlocks = 512;   // gate/up row blocks of one stream that may fall to one CTA
 constexpr int kFusedMaxCtaRows = 64;      // rows of the residual stream one CTA may own (d <= 64 x SMs)
-constexpr int kFusedZCopies = 16;         // copies of the fixed-point logit accumulators
 constexpr int kStackMaxLayers = 44;       // layers per launch (their pointers travel as kernel parameters)
 struct LayerDesc {
     const void *router_W; const float *router_bias; const void *w_s;   // w_s NULL: shared gate = 1
@@ -177,7 +176,7 @@ struct StackArgs {
     float routed_scale;
     float *logits; int32_t *topk_idx; float *topk_w; float *gamma;      // routing of the last layer, as moe_last_routing reports it
     int32_t *counts, *offsets, *perm, *inv_perm, *stats, *status;
-    long long *zacc;                    // [2][kFusedZCopies][8][kMaxExperts] logit accumulators (2^-40 units), zero between launches
+    float *zslot;                       // [grid][8][kMaxExperts] every CTA's partial router logits of the coming layer
     uint32_t *bar; uint32_t bar_base;   // grid-barrier counter and its value when this launch starts
     __nv_bfloat16 *hbuf; int hs;        // gate-weighted hidden activations h', row pitch hs
     unsigned long long *stamps; int stamp_layer;   // NULL, or [grid, 8] time stamps of one layer (debug)

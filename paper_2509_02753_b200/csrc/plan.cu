@@ -105,7 +105,7 @@ int fused_stack(moe_plan *p, const void *x, const moe_layer_weights_t *layers, c
     fa.logits = ws.logits; fa.topk_idx = ws.topk_idx; fa.topk_w = ws.topk_w; fa.gamma = ws.gamma;
     fa.counts = ws.counts; fa.offsets = ws.offsets; fa.perm = ws.perm; fa.inv_perm = ws.inv_perm;
     fa.stats = ws.stats; fa.status = ws.status;
-    fa.zacc = ws.f_zacc; fa.bar = ws.f_bar; fa.bar_base = p->fused_bar_base;
+    fa.zslot = ws.f_zslot; fa.bar = ws.f_bar; fa.bar_base = p->fused_bar_base;
     fa.hbuf = ws.f_hbuf; fa.hs = p->fused_hs;
     fa.stamps = p->fused_stamp_layer >= 0 ? ws.f_stamps : nullptr;
     fa.stamp_layer = p->fused_stamp_layer < n_layers ? p->fused_stamp_layer : n_layers - 1;
@@ -356,7 +356,7 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
     }
     const int rc = tc_state_init(&p->tc, c);
     if (rc != MOE_OK) { moe_plan_destroy(p); return rc; }
-    // one-launch stack for tiny decode calls: logit accumulators, barrier counter, h'
+    // one-launch stack for tiny decode calls: per-CTA logit slots, barrier counter, h'
     {
         const int ucap = c.E < kFusedMaxTokens * c.max_k ? c.E : kFusedMaxTokens * c.max_k;
         // gate/up row blocks that can fall to one CTA: its features in blocks of 8, plus one ragged
@@ -368,12 +368,11 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
             fused_smem_bytes(c.d) <= 200 * 1024 && (c.d + sms - 1) / sms <= kFusedMaxCtaRows &&
             blocks_cta <= kFusedMaxCtaBlocks && blocks_cta_s <= kFusedMaxCtaBlocks) {
             p->fused_hs = c.I_shared + ucap * c.I;
-            bool fok = ws_alloc(p, &ws.f_zacc, (size_t)2 * kFusedZCopies * kFusedMaxTokens * kMaxExperts) &&
+            bool fok = ws_alloc(p, &ws.f_zslot, (size_t)sms * kFusedMaxTokens * kMaxExperts) &&
                        ws_alloc(p, &ws.f_bar, (size_t)4) &&
                        ws_alloc(p, &ws.f_hbuf, (size_t)kFusedMaxTokens * p->fused_hs) &&
                        ws_alloc(p, &ws.f_stamps, (size_t)sms * 8);
-            fok = fok && cudaMemset(ws.f_zacc, 0, sizeof(long long) * 2 * kFusedZCopies * kFusedMaxTokens * kMaxExperts) == cudaSuccess &&
-                  cudaMemset(ws.f_bar, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess &&
+            fok = fok && cudaMemset(ws.f_bar, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess &&
                   fused_prepare(c.d) == cudaSuccess;
             if (!fok) { cudaGetLastError(); moe_plan_destroy(p); return MOE_ERR_WORKSPACE; }
             p->fused_ok = true;
@@ -854,11 +853,8 @@ int moe_device_status(moe_plan_t *p, void *cuda_stream) {
         return MOE_ERR_CUDA;
     }
     const int32_t v = *p->status_host;
-    if (v && getenv("LEXI_DEBUG_STATUS")) fprintf(stderr, "device status word 0x%x\n", v);
     if ((v & kStatusTimeout) && p->fused_ok) {
-        // a one-launch call that gave up has left the barrier counter and the logit accumulators
-        // half way: both start again from zero
-        cudaMemsetAsync(p->ws.f_zacc, 0, sizeof(long long) * 2 * kFusedZCopies * kFusedMaxTokens * kMaxExperts, s);
+        // a one-launch call that gave up has left the barrier counter half way: it starts again from zero
         cudaMemsetAsync(p->ws.f_bar, 0, sizeof(uint32_t), s);
         cudaStreamSynchronize(s);
         p->fused_bar_base = 0;
