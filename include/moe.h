@@ -106,6 +106,10 @@ typedef struct moe_plan moe_plan_t;   /* opaque; owns the workspace and the sche
  * top-k indices and gates, dispatch tables, the expert-ordered copy of x, the intermediate
  * h, the per-pair expert outputs, the fp32 residual stream of the stack.
  * Synchronises.  *out receives the plan (NULL on failure).
+ * With LEXI_DEBUG_GUARD=1 in the environment the plan gets a debug workspace (the library's stand-in
+ * for a memory checker): every sub-buffer lies between two 256-byte guard bands, the buffers a call
+ * must write before it reads them are filled with 0xFF bytes (NaN, -1) before every layer or stack
+ * call, and moe_device_status also returns MOE_ERR_DEVICE_CHECK if a band was written to.
  * Errors: INVALID_ARG, SHAPE, CUDA (no sm_100 device), WORKSPACE.
  */
 int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out);
@@ -173,11 +177,21 @@ int moe_layer_forward_host(moe_plan_t *plan, const void *x_host, const moe_layer
  *   counts [E], offsets [E + 1], perm [T * k_l] (pairs t * k_l + j in expert-major, token-ascending
  *   order), inv_perm [T * k_l] (position of each pair in perm).  Only router_W, router_bias and w_s
  *   of w are read.
- * moe_gather_rows: dst[r, :] = src[row_index[r], :] for r < n_rows; rows of d elements of the
- *   plan's dtype, or of fp32 when rows_f32 != 0 (expert outputs).
+ * moe_gather_rows: dst[r, :] = src[row_index[r] / index_div, :] for r < n_rows (index_div >= 1; with
+ *   row_index = perm and index_div = k_l the rows of x land in expert order); rows of d elements of
+ *   the plan's dtype, or of fp32 when rows_f32 != 0 (expert outputs).
+ * moe_regroup_index: the receiving side's bookkeeping on the device.  recv_counts [world, E] int32
+ *   (E = this plan's experts, the local ones): rows that arrived from each source rank per local
+ *   expert, the arrival buffer being source-major (inside a source the experts ascend).  Writes
+ *   to_expert_major [n_rows] (arrival index of the row at each position of the expert-major order,
+ *   sources of an expert in rank order), inverse [n_rows] and per_expert [E] (the counts
+ *   moe_experts_forward takes).  world * E <= 1024.  Counts that do not add up to n_rows write
+ *   nothing but per_expert = 0 and raise MOE_ERR_DEVICE_CHECK at the next moe_device_status.
  * moe_experts_forward: o_rows[r, :] = E_e(x_rows[r, :]) in fp32, for rows grouped by expert: the
  *   first counts[0] rows belong to expert 0 of this plan, the next counts[1] to expert 1, ...;
- *   n_rows = sum of counts <= max_T * max_k.  Only W_gate, W_up, W_down of w are read (a shared
+ *   n_rows = sum of counts <= max_T * max_k; counts (device memory) that are negative or do not add
+ *   up to n_rows are caught on the device: nothing is computed or written and the next
+ *   moe_device_status returns MOE_ERR_DEVICE_CHECK.  Only W_gate, W_up, W_down of w are read (a shared
  *   expert is a plan of its own with E = 1).  bf16 plans run the tcgen05 prefill kernels (CTA pairs
  *   from 64 rows per expert), fp32 plans the CUDA-core kernels.
  * moe_combine: y[t] = routed_scale * sum_j topk_w[t, j] * o_rows[inv_perm[t * k_l + j]]
@@ -188,8 +202,10 @@ int moe_layer_forward_host(moe_plan_t *plan, const void *x_host, const moe_layer
 int moe_route(moe_plan_t *plan, const void *x, const moe_layer_weights_t *w, int32_t T, int32_t k_l,
               int32_t renorm, int32_t *topk_idx, float *topk_w, float *gamma, int32_t *counts,
               int32_t *offsets, int32_t *perm, int32_t *inv_perm, void *cuda_stream);
-int moe_gather_rows(moe_plan_t *plan, const void *src, const int32_t *row_index, int32_t n_rows,
-                    int32_t rows_f32, void *dst, void *cuda_stream);
+int moe_gather_rows(moe_plan_t *plan, const void *src, const int32_t *row_index, int32_t index_div,
+                    int32_t n_rows, int32_t rows_f32, void *dst, void *cuda_stream);
+int moe_regroup_index(moe_plan_t *plan, const int32_t *recv_counts, int32_t world, int32_t n_rows,
+                      int32_t *to_expert_major, int32_t *inverse, int32_t *per_expert, void *cuda_stream);
 int moe_experts_forward(moe_plan_t *plan, const void *x_rows, const int32_t *counts,
                         const moe_layer_weights_t *w, int32_t n_rows, float *o_rows, void *cuda_stream);
 int moe_combine(moe_plan_t *plan, const float *o_rows, const float *topk_w, const int32_t *inv_perm,

@@ -30,7 +30,7 @@ EXPORTS = (
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
     "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts",
     "moe_debug_fused_stamps", "moe_host_pipeline_submit", "moe_host_pipeline_wait",
-    "moe_route", "moe_gather_rows", "moe_experts_forward", "moe_combine",
+    "moe_route", "moe_gather_rows", "moe_regroup_index", "moe_experts_forward", "moe_combine",
     "moe_debug_wait_timeout", "moe_debug_barrier_timeout", "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
@@ -90,7 +90,8 @@ def load_library() -> ctypes.CDLL:
     lib.moe_host_pipeline_submit.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, vp, P(ctypes.c_int64)]
     lib.moe_host_pipeline_wait.argtypes = [vp, ctypes.c_int64]
     lib.moe_route.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
-    lib.moe_gather_rows.argtypes = [vp, vp, vp, i32, i32, vp, vp]
+    lib.moe_gather_rows.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
+    lib.moe_regroup_index.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
     lib.moe_experts_forward.argtypes = [vp, vp, vp, P(moe_layer_weights_t), i32, vp, vp]
     lib.moe_combine.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
     lib.moe_profile_layer.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, P(ctypes.c_double),
@@ -224,13 +225,28 @@ def moe_route(plan: int, x: torch.Tensor, w: moe_layer_weights_t, k_l: int, reno
     return out
 
 
-def moe_gather_rows(plan: int, src: torch.Tensor, row_index: torch.Tensor, dst: torch.Tensor, stream=None) -> None:
-    """dst[r] = src[row_index[r]]; rows of the plan's dtype, or fp32 rows when src is float32."""
+def moe_gather_rows(plan: int, src: torch.Tensor, row_index: torch.Tensor, dst: torch.Tensor, index_div: int = 1,
+                    stream=None) -> None:
+    """dst[r] = src[row_index[r] // index_div]; rows of the plan's dtype, or fp32 rows when src is float32."""
     assert src.is_cuda and src.is_contiguous() and dst.is_contiguous() and row_index.dtype == torch.int32
     assert dst.shape[0] == row_index.shape[0] and src.dtype == dst.dtype
     _check("moe_gather_rows", load_library().moe_gather_rows(
-        plan, src.data_ptr(), row_index.data_ptr(), row_index.shape[0], int(src.dtype == torch.float32),
+        plan, src.data_ptr(), row_index.data_ptr(), index_div, row_index.shape[0], int(src.dtype == torch.float32),
         dst.data_ptr(), _stream(stream)))
+
+
+def moe_regroup_index(plan: int, recv_counts: torch.Tensor, n_rows: int, stream=None):
+    """Receiving side of expert parallelism: (to_expert_major [n_rows], inverse [n_rows], per_expert [E_loc])
+    int32 device tensors from recv_counts [world, E_loc] (rows per source rank and local expert)."""
+    assert recv_counts.is_cuda and recv_counts.dtype == torch.int32 and recv_counts.is_contiguous()
+    world, e_loc = recv_counts.shape
+    dev = recv_counts.device
+    to_em = torch.empty((max(n_rows, 1),), dtype=torch.int32, device=dev)     # never empty: the call wants real pointers
+    inv = torch.empty((max(n_rows, 1),), dtype=torch.int32, device=dev)
+    per = torch.empty((e_loc,), dtype=torch.int32, device=dev)
+    _check("moe_regroup_index", load_library().moe_regroup_index(
+        plan, recv_counts.data_ptr(), world, n_rows, to_em.data_ptr(), inv.data_ptr(), per.data_ptr(), _stream(stream)))
+    return to_em[:n_rows], inv[:n_rows], per
 
 
 def moe_experts_forward(plan: int, x_rows: torch.Tensor, counts: torch.Tensor, w: moe_layer_weights_t,

@@ -286,6 +286,57 @@ cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k,
     return e;
 }
 
+// Expert parallelism, receiving side: rows arrive source-major (all rows of source rank 0, then
+// rank 1, ...; inside a source the local experts ascend) and the grouped GEMMs want them
+// expert-major (inside an expert the sources in rank order).  recv_counts [world, E] = rows per
+// (source, local expert).  to_em[p] = arrival index of the row at expert-major position p, inv its
+// inverse, per_expert[e] = rows of local expert e.  Every CTA redoes the two small scans over the
+// world x E blocks in shared memory and then copies index ranges of its share of the blocks.
+constexpr int kMaxRegroupBlocks = 1024;
+__global__ void __launch_bounds__(256) regroup_index_kernel(const int32_t *__restrict__ recv_counts, int world, int E,
+                                                            int n_rows, int32_t *to_em, int32_t *inv,
+                                                            int32_t *per_expert, int32_t *status) {
+    __shared__ int32_t len[kMaxRegroupBlocks], arr_start[kMaxRegroupBlocks], out_start[kMaxRegroupBlocks];
+    __shared__ int32_t total;
+    const int nb = world * E;
+    for (int b = threadIdx.x; b < nb; b += blockDim.x) len[b] = max(recv_counts[b], 0);      // b = source * E + expert
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int b = 0; b < nb; ++b) { arr_start[b] = run; run += len[b]; }                 // arrival order
+        total = run;
+        run = 0;
+        for (int e = 0; e < E; ++e)
+            for (int sr = 0; sr < world; ++sr) { out_start[sr * E + e] = run; run += len[sr * E + e]; }   // expert-major order
+    }
+    __syncthreads();
+    const bool bad = total != n_rows;
+    if (blockIdx.x == 0) {
+        if (bad && threadIdx.x == 0) atomicOr(status, kStatusBadIndex);
+        for (int e = threadIdx.x; e < E; e += blockDim.x) {
+            int c = 0;
+            for (int sr = 0; sr < world; ++sr) c += len[sr * E + e];
+            per_expert[e] = bad ? 0 : c;
+        }
+    }
+    if (bad) return;
+    for (int b = blockIdx.x; b < nb; b += gridDim.x) {
+        const int a0 = arr_start[b], o0 = out_start[b];
+        for (int i = threadIdx.x; i < len[b]; i += blockDim.x) {
+            to_em[o0 + i] = a0 + i;
+            inv[a0 + i] = o0 + i;
+        }
+    }
+}
+
+cudaError_t launch_regroup_index(const int32_t *recv_counts, int world, int E, int n_rows, int32_t *to_em, int32_t *inv,
+                                 int32_t *per_expert, int32_t *status, cudaStream_t s, uint64_t *launches) {
+    const int nb = world * E;
+    regroup_index_kernel<<<nb < 296 ? nb : 296, 256, 0, s>>>(recv_counts, world, E, n_rows, to_em, inv, per_expert, status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
 }  // namespace lexi
 
 // ---------------------------------------------------------------------------------------

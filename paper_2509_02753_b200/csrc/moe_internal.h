@@ -119,6 +119,9 @@ cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k,
                           void *x_perm, cudaStream_t s, uint64_t *launches, bool chained = false,
                           const TileBuildArgs *tiles = nullptr);   // tiles: also build the tile lists
 
+cudaError_t launch_regroup_index(const int32_t *recv_counts, int world, int E, int n_rows, int32_t *to_em, int32_t *inv,
+                                 int32_t *per_expert, int32_t *status, cudaStream_t s, uint64_t *launches);
+
 struct FfnArgs {
     int dtype, T, k, d, E, I, I_s;
     const int32_t *counts, *offsets;

@@ -17,6 +17,13 @@ struct moe_plan {
     Workspace ws{};
     std::vector<void *> allocs;
     uint64_t bytes = 0;
+    // debug build of the workspace (LEXI_DEBUG_GUARD=1 when the plan is made): every sub-buffer sits
+    // between two 256-byte guard bands of a known pattern, buffers that a call fully rewrites before it
+    // reads them are filled with 0xFF bytes (NaN / -1) before every layer or stack call, and
+    // moe_device_status also compares the bands
+    bool guard = false;
+    struct Buf { unsigned char *base; size_t bytes; bool scratch; };
+    std::vector<Buf> bufs;
     uint64_t launches = 0;
     int32_t forced_schedule = MOE_SCHED_AUTO;
     int32_t last_T = 0, last_k = 0;
@@ -56,16 +63,56 @@ size_t elem_size(int dtype) { return dtype == MOE_BF16 ? 2 : 4; }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+constexpr size_t kGuardBytes = 256;
+constexpr int kGuardByte = 0xA5;
+
+// scratch: the buffer holds nothing across calls (every call writes what it later reads), so the
+// debug workspace may poison it before a call
 template <typename T>
-bool ws_alloc(moe_plan *p, T **out, size_t count, size_t elem = sizeof(T)) {
+bool ws_alloc(moe_plan *p, T **out, size_t count, size_t elem = sizeof(T), bool scratch = false) {
     size_t bytes = count * elem;
     bytes = (bytes + 255) & ~size_t(255);
     if (bytes == 0) bytes = 256;
+    const size_t pad = p->guard ? kGuardBytes : 0;
     void *ptr = nullptr;
-    if (cudaMalloc(&ptr, bytes) != cudaSuccess) { cudaGetLastError(); return false; }
+    if (cudaMalloc(&ptr, bytes + 2 * pad) != cudaSuccess) { cudaGetLastError(); return false; }
     p->allocs.push_back(ptr);
-    p->bytes += bytes;
-    *out = reinterpret_cast<T *>(ptr);
+    p->bytes += bytes + 2 * pad;
+    unsigned char *base = reinterpret_cast<unsigned char *>(ptr) + pad;
+    if (p->guard) {
+        if (cudaMemset(ptr, kGuardByte, pad) != cudaSuccess || cudaMemset(base + bytes, kGuardByte, pad) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        p->bufs.push_back({base, bytes, scratch});
+    }
+    *out = reinterpret_cast<T *>(base);
+    return true;
+}
+template <typename T>
+bool ws_scratch(moe_plan *p, T **out, size_t count, size_t elem = sizeof(T)) { return ws_alloc(p, out, count, elem, true); }
+
+// debug workspace: poison what the coming call must write before it reads
+void guard_poison(moe_plan *p, cudaStream_t s) {
+    if (!p->guard) return;
+    for (const moe_plan::Buf &b : p->bufs)
+        if (b.scratch) cudaMemsetAsync(b.base, 0xFF, b.bytes, s);
+}
+
+// debug workspace: true if every guard band still holds its pattern (synchronises the stream)
+bool guard_intact(moe_plan *p, cudaStream_t s) {
+    if (!p->guard) return true;
+    std::vector<unsigned char> host(2 * kGuardBytes);
+    for (const moe_plan::Buf &b : p->bufs) {
+        if (cudaMemcpyAsync(host.data(), b.base - kGuardBytes, kGuardBytes, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaMemcpyAsync(host.data() + kGuardBytes, b.base + b.bytes, kGuardBytes, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        for (unsigned char v : host)
+            if (v != kGuardByte) return false;
+    }
     return true;
 }
 
@@ -98,6 +145,7 @@ int fused_stack(moe_plan *p, const void *x, const moe_layer_weights_t *layers, c
                 int T, int renorm, void *y, int mode, int resume, cudaStream_t s) {
     const moe_config_t &c = p->cfg;
     Workspace &ws = p->ws;
+    guard_poison(p, s);
     StackArgs fa{};
     fa.x = x; fa.y = (__nv_bfloat16 *)y; fa.h_run = ws.h_run; fa.mode = mode; fa.resume = resume;
     fa.L = n_layers; fa.T = T; fa.d = c.d; fa.E = c.E; fa.I = c.I; fa.I_s = c.I_shared; fa.renorm = renorm;
@@ -142,6 +190,7 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
     if (p->timing && p->timed_calls < kMaxTimedCalls)
         ev = &p->events[(size_t)p->timed_calls++ * (MOE_N_STAGES + 1)];
     auto mark = [&](int i) { if (ev) cudaEventRecord(ev[i], s); };
+    guard_poison(p, s);
     mark(0);
 
     RouterArgs ra{x, w->router_W, w->router_bias, (c.I_shared > 0 && c.shared_gate) ? w->w_s : nullptr,
@@ -236,8 +285,11 @@ int check_call(const moe_plan *p, const void *x, const moe_layer_weights_t *w, i
     return check_weights(p, w);
 }
 
-// offsets[e] = sum of counts[0..e), offsets[E] = total: one warp, 4 experts per lane
-__global__ void offsets_from_counts_kernel(const int32_t *counts, int32_t *offsets, int E) {
+// offsets[e] = sum of counts[0..e), offsets[E] = total: one warp, 4 experts per lane.  The caller says
+// how many rows exist behind its buffers; counts that do not add up to that (they may have crossed a
+// network) would make the GEMMs write beyond them, so then the status word is set and every count
+// becomes zero (no tile is built, nothing is written).
+__global__ void offsets_from_counts_kernel(int32_t *counts, int32_t *offsets, int E, int n_rows, int32_t *status) {
     const int lane = threadIdx.x;
     int c[kExpertsPerLane], sum = 0;
 #pragma unroll
@@ -252,14 +304,23 @@ __global__ void offsets_from_counts_kernel(const int32_t *counts, int32_t *offse
         const int v = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += v;
     }
+    const int total = __shfl_sync(0xffffffffu, incl, 31);
+    bool neg = false;
+#pragma unroll
+    for (int j = 0; j < kExpertsPerLane; ++j) neg = neg || c[j] < 0;
+    const bool bad = total != n_rows || __any_sync(0xffffffffu, neg);
+    if (bad && lane == 0) atomicOr(status, kStatusBadIndex);
     int run = incl - sum;
 #pragma unroll
     for (int j = 0; j < kExpertsPerLane; ++j) {
         const int e = lane * kExpertsPerLane + j;
-        if (e < E) offsets[e] = run;
+        if (e < E) {
+            offsets[e] = bad ? 0 : run;
+            if (bad) counts[e] = 0;
+        }
         run += c[j];
     }
-    if (lane == 31) offsets[E] = incl;
+    if (lane == 31) offsets[E] = bad ? 0 : incl;
 }
 
 }  // namespace
@@ -307,6 +368,7 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
     if (!p) return MOE_ERR_WORKSPACE;
     p->cfg = *cfg;
     p->sm_count = sms;
+    { const char *g = getenv("LEXI_DEBUG_GUARD"); p->guard = g && g[0] == '1'; }
     const moe_config_t &c = p->cfg;
     Workspace &ws = p->ws;
     const size_t es = elem_size(c.dtype);
@@ -315,34 +377,34 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
     const int slabs = tc_max_slabs(c);
     const int slabs_s = tc_max_shared_slabs(c);
     bool ok = true;
-    ok = ok && ws_alloc(p, &ws.logits, (size_t)c.max_T * c.E);
-    ok = ok && ws_alloc(p, &ws.topk_idx, pairs);
-    ok = ok && ws_alloc(p, &ws.topk_w, pairs);
-    ok = ok && ws_alloc(p, &ws.counts, (size_t)c.E);
-    ok = ok && ws_alloc(p, &ws.offsets, (size_t)c.E + 1);
-    ok = ok && ws_alloc(p, &ws.perm, pairs);
-    ok = ok && ws_alloc(p, &ws.inv_perm, pairs);
-    ok = ok && ws_alloc(p, &ws.part_hist, n_parts * c.E);
-    ok = ok && ws_alloc(p, &ws.gamma, (size_t)c.max_T);
-    ok = ok && ws_alloc(p, &ws.x_perm, pairs * c.d + 128 * (size_t)c.d, es);
-    ok = ok && ws_alloc(p, &ws.h, pairs * c.I + 128 * (size_t)c.I, es);
-    ok = ok && ws_alloc(p, &ws.h_s, (size_t)c.max_T * c.I_shared + 128 * (size_t)c.I_shared, es);
+    ok = ok && ws_scratch(p, &ws.logits, (size_t)c.max_T * c.E);
+    ok = ok && ws_scratch(p, &ws.topk_idx, pairs);
+    ok = ok && ws_scratch(p, &ws.topk_w, pairs);
+    ok = ok && ws_scratch(p, &ws.counts, (size_t)c.E);
+    ok = ok && ws_scratch(p, &ws.offsets, (size_t)c.E + 1);
+    ok = ok && ws_scratch(p, &ws.perm, pairs);
+    ok = ok && ws_scratch(p, &ws.inv_perm, pairs);
+    ok = ok && ws_scratch(p, &ws.part_hist, n_parts * c.E);
+    ok = ok && ws_scratch(p, &ws.gamma, (size_t)c.max_T);
+    ok = ok && ws_scratch(p, &ws.x_perm, pairs * c.d + 128 * (size_t)c.d, es);
+    ok = ok && ws_scratch(p, &ws.h, pairs * c.I + 128 * (size_t)c.I, es);
+    ok = ok && ws_scratch(p, &ws.h_s, (size_t)c.max_T * c.I_shared + 128 * (size_t)c.I_shared, es);
     // expert outputs: fp32 partial-sum slabs when the decode schedule splits K, else one slab
     const size_t o_elems = tc_o_elems(c, slabs);
     const size_t os_elems = tc_os_elems(c, slabs_s);
-    ok = ok && ws_alloc(p, &ws.o, o_elems, 4);
-    ok = ok && ws_alloc(p, &ws.o_s, c.I_shared > 0 ? os_elems : 0, 4);
+    ok = ok && ws_scratch(p, &ws.o, o_elems, 4);
+    ok = ok && ws_scratch(p, &ws.o_s, c.I_shared > 0 ? os_elems : 0, 4);
     ok = ok && ws_alloc(p, &ws.h_run, (size_t)c.max_T * c.d);
     ok = ok && ws_alloc(p, &ws.x_stage, (size_t)c.max_T * c.d, es);
     ok = ok && ws_alloc(p, &ws.y_stage, (size_t)c.max_T * c.d, es);
     ok = ok && ws_alloc(p, &ws.status, (size_t)4);
-    ok = ok && ws_alloc(p, &ws.tiles1, tc_max_tiles(c, 1));
-    ok = ok && ws_alloc(p, &ws.tiles2, tc_max_tiles(c, 2));
+    ok = ok && ws_scratch(p, &ws.tiles1, tc_max_tiles(c, 1));
+    ok = ok && ws_scratch(p, &ws.tiles2, tc_max_tiles(c, 2));
     ok = ok && ws_alloc(p, &ws.n_tiles, (size_t)4);
     ok = ok && ws_alloc(p, &ws.ticket, (size_t)4 + kFrontMaxTokens);
-    ok = ok && ws_alloc(p, &ws.pos, (size_t)c.E * kFrontMaxTokens);
+    ok = ok && ws_scratch(p, &ws.pos, (size_t)c.E * kFrontMaxTokens);
     ok = ok && ws_alloc(p, &ws.stats, (size_t)4);
-    ok = ok && ws_alloc(p, &ws.prof_partial, (((size_t)c.max_T * c.d / 4 + 255) / 256) * (c.max_k + 1));
+    ok = ok && ws_scratch(p, &ws.prof_partial, (((size_t)c.max_T * c.d / 4 + 255) / 256) * (c.max_k + 1));
     ok = ok && ws_alloc(p, &ws.prof_sums, (size_t)c.max_k + 1);
     if (ok && cudaMallocHost(&p->status_host, sizeof(int32_t)) != cudaSuccess) { cudaGetLastError(); ok = false; }
     if (ok) {
@@ -368,9 +430,9 @@ int moe_plan_create(const moe_config_t *cfg, moe_plan_t **out) {
             fused_smem_bytes(c.d) <= 200 * 1024 && (c.d + sms - 1) / sms <= kFusedMaxCtaRows &&
             blocks_cta <= kFusedMaxCtaBlocks && blocks_cta_s <= kFusedMaxCtaBlocks) {
             p->fused_hs = c.I_shared + ucap * c.I;
-            bool fok = ws_alloc(p, &ws.f_zslot, (size_t)sms * kFusedMaxTokens * kMaxExperts) &&
+            bool fok = ws_scratch(p, &ws.f_zslot, (size_t)sms * kFusedMaxTokens * kMaxExperts) &&
                        ws_alloc(p, &ws.f_bar, (size_t)4) &&
-                       ws_alloc(p, &ws.f_hbuf, (size_t)kFusedMaxTokens * p->fused_hs) &&
+                       ws_scratch(p, &ws.f_hbuf, (size_t)kFusedMaxTokens * p->fused_hs) &&
                        ws_alloc(p, &ws.f_stamps, (size_t)sms * 8);
             fok = fok && cudaMemset(ws.f_bar, 0, 16) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess &&
                   fused_prepare(c.d) == cudaSuccess;
@@ -569,12 +631,24 @@ int moe_route(moe_plan_t *p, const void *x, const moe_layer_weights_t *w, int32_
     return moe_last_routing(p, topk_idx, topk_w, counts, offsets, perm, nullptr, cuda_stream);
 }
 
-int moe_gather_rows(moe_plan_t *p, const void *src, const int32_t *row_index, int32_t n_rows, int32_t rows_f32,
-                    void *dst, void *cuda_stream) {
-    if (!p || !src || !row_index || !dst || n_rows < 0) return MOE_ERR_INVALID_ARG;
+int moe_gather_rows(moe_plan_t *p, const void *src, const int32_t *row_index, int32_t index_div, int32_t n_rows,
+                    int32_t rows_f32, void *dst, void *cuda_stream) {
+    if (!p || !src || !row_index || !dst || n_rows < 0 || index_div < 1) return MOE_ERR_INVALID_ARG;
     if (!aligned16(src) || !aligned16(dst)) return MOE_ERR_ALIGN;
-    if (launch_gather(src, row_index, n_rows, 1, p->cfg.d, rows_f32 ? MOE_F32 : p->cfg.dtype, dst,
+    if (launch_gather(src, row_index, n_rows, index_div, p->cfg.d, rows_f32 ? MOE_F32 : p->cfg.dtype, dst,
                       (cudaStream_t)cuda_stream, &p->launches) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    return MOE_OK;
+}
+
+int moe_regroup_index(moe_plan_t *p, const int32_t *recv_counts, int32_t world, int32_t n_rows, int32_t *to_expert_major,
+                      int32_t *inverse, int32_t *per_expert, void *cuda_stream) {
+    if (!p || !recv_counts || !to_expert_major || !inverse || !per_expert) return MOE_ERR_INVALID_ARG;
+    if (world < 1 || n_rows < 0 || (int64_t)world * p->cfg.E > 1024) return MOE_ERR_INVALID_ARG;
+    if (launch_regroup_index(recv_counts, world, p->cfg.E, n_rows, to_expert_major, inverse, per_expert, p->ws.status,
+                             (cudaStream_t)cuda_stream, &p->launches) != cudaSuccess) {
         cudaGetLastError();
         return MOE_ERR_CUDA;
     }
@@ -595,7 +669,7 @@ int moe_experts_forward(moe_plan_t *p, const void *x_rows, const int32_t *counts
         cudaGetLastError();
         return MOE_ERR_CUDA;
     }
-    offsets_from_counts_kernel<<<1, 32, 0, s>>>(ws.counts, ws.offsets, c.E);
+    offsets_from_counts_kernel<<<1, 32, 0, s>>>(ws.counts, ws.offsets, c.E, n_rows, ws.status);
     ++p->launches;
     // the rows are the (token, slot) pairs of a layer call that has T = n_rows tokens and one slot
     FfnArgs fa{c.dtype, n_rows, 1, c.d, c.E, c.I, 0, ws.counts, ws.offsets, x_rows, x_rows,
@@ -861,6 +935,7 @@ int moe_device_status(moe_plan_t *p, void *cuda_stream) {
     }
     if (v & kStatusTimeout) return MOE_ERR_TIMEOUT;
     if (v & kStatusBadIndex) return MOE_ERR_DEVICE_CHECK;
+    if (!guard_intact(p, s)) return MOE_ERR_DEVICE_CHECK;
     return MOE_OK;
 }
 

@@ -14,14 +14,18 @@ the expert work.  Rank r holds the experts [r * E / R, (r + 1) * E / R) and the 
     exchange the fp32 outputs back, all-to-all
     finish   gated sum over each token's slots plus the shared expert (moe_combine)
 
-Every arithmetic step is a kernel of the C library; this module holds the integer bookkeeping
-(which rows go where: `exchange_plan`, `regroup_index`) and the calls of torch.distributed.
-`pack` / `compute` / `finish` are separate methods so that a test can run R ranks in one process
-and move the rows by hand.
+Every arithmetic step and the receiving side's index tables are kernels of the C library
+(moe_route, moe_gather_rows, moe_regroup_index, moe_experts_forward, moe_combine); this module
+holds the calls of torch.distributed and the one thing they need on the host: how many rows go
+to and come from each rank.  `forward` learns both from ONE all-gather of the per-expert counts
+(a single device-to-host read per call); `regroup_index` below is the same bookkeeping in torch,
+kept as the reference the tests compare the kernel with.  `pack` / `compute` / `finish` are
+separate methods so that a test can run R ranks in one process and move the rows by hand.
 
 Not run on more than one GPU here: the kernels between the exchanges are the single-GPU ones and
 are checked against the one-GPU layer by running the ranks one after the other on one device;
-the exchange itself is checked with CPU tensors over gloo.
+`forward` itself is run end to end by two processes that share one GPU and exchange through host
+memory over gloo (`host_staging=True`), and the exchange alone with CPU tensors over gloo.
 """
 from __future__ import annotations
 
@@ -68,10 +72,18 @@ def regroup_index(recv_counts: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor
     return to_expert_major, inverse, c.sum(dim=0).to(torch.int32)
 
 
-def exchange_rows(rows: torch.Tensor, send_splits: List[int], recv_splits: List[int], group=None) -> torch.Tensor:
+def exchange_rows(rows: torch.Tensor, send_splits: List[int], recv_splits: List[int], group=None,
+                  host_staging: bool = False) -> torch.Tensor:
     """All-to-all of row blocks: block r of `rows` (send_splits[r] rows) goes to rank r; returns the
-    blocks received, in source order.  Works on whatever device the process group serves."""
+    blocks received, in source order.  Works on whatever device the process group serves; with
+    host_staging the rows of a CUDA tensor cross through host memory (a group that only moves CPU
+    tensors, such as gloo)."""
     import torch.distributed as dist
+    if host_staging and rows.is_cuda:
+        src = rows.contiguous().cpu()
+        out = src.new_empty((sum(recv_splits),) + tuple(rows.shape[1:]))
+        dist.all_to_all_single(out, src, recv_splits, send_splits, group=group)
+        return out.to(rows.device)
     out = rows.new_empty((sum(recv_splits),) + tuple(rows.shape[1:]))
     dist.all_to_all_single(out, rows.contiguous(), recv_splits, send_splits, group=group)
     return out
@@ -127,21 +139,22 @@ class ExpertParallelLayer:
                 p.close()
 
     # -- step 1: route the rank's tokens and lay their rows out by destination
-    def pack(self, x: torch.Tensor, k_l: int, renorm: bool):
+    def pack(self, x: torch.Tensor, k_l: int, renorm: bool, splits: bool = True):
         B = self.B
         r = B.moe_route(self.router_plan.handle, x, self.w_router, k_l, renorm, self.E)
-        row_index = torch.div(r["perm"], k_l, rounding_mode="floor").to(torch.int32)
         send_rows = torch.empty((x.shape[0] * k_l, self.d), dtype=x.dtype, device=x.device)
-        B.moe_gather_rows(self.router_plan.handle, x, row_index, send_rows)
-        send_counts, send_splits = exchange_plan(r["counts"], self.world)
-        ctx = {"x": x, "route": r, "k": k_l, "send_splits": send_splits}
+        B.moe_gather_rows(self.router_plan.handle, x, r["perm"], send_rows, index_div=k_l)   # row of pair p is token p // k_l
+        send_counts = r["counts"].reshape(self.world, self.e_loc)
+        ctx = {"x": x, "route": r, "k": k_l}
+        if splits:
+            ctx["send_splits"] = [int(v) for v in send_counts.sum(dim=1).tolist()]
         return send_rows, send_counts, ctx
 
     # -- step 2: the local experts on what arrived (rows source-major), outputs in arrival order
     def compute(self, recv_rows: torch.Tensor, recv_counts: torch.Tensor) -> torch.Tensor:
         B = self.B
-        to_em, inverse, per_expert = regroup_index(recv_counts)
         n = recv_rows.shape[0]
+        to_em, inverse, per_expert = B.moe_regroup_index(self.local_plan.handle, recv_counts.contiguous(), n)
         grouped = torch.empty_like(recv_rows)
         out_em = torch.empty((n, self.d), dtype=torch.float32, device=recv_rows.device)
         back = torch.empty_like(out_em)
@@ -166,12 +179,22 @@ class ExpertParallelLayer:
                       r["gamma"] if self.shared_gate else None)
         return y
 
-    # -- the whole call over torch.distributed (one process per GPU, NCCL)
-    def forward(self, x: torch.Tensor, k_l: int, renorm: bool, group=None) -> torch.Tensor:
-        send_rows, send_counts, ctx = self.pack(x, k_l, renorm)
-        recv_counts = exchange_counts(send_counts, group)
-        recv_splits = [int(v) for v in recv_counts.sum(dim=1).tolist()]
-        recv_rows = exchange_rows(send_rows, ctx["send_splits"], recv_splits, group)
+    # -- the whole call over torch.distributed (one process per GPU, NCCL; or host_staging over gloo)
+    def forward(self, x: torch.Tensor, k_l: int, renorm: bool, group=None, host_staging: bool = False) -> torch.Tensor:
+        import torch.distributed as dist
+        send_rows, send_counts, ctx = self.pack(x, k_l, renorm, splits=False)
+        # every rank's pairs per global expert, gathered once: row s says what rank s sends; the
+        # only device-to-host read of the call
+        mine = ctx["route"]["counts"]
+        if host_staging:
+            mine = mine.cpu()
+        parts = [torch.empty_like(mine) for _ in range(self.world)]
+        dist.all_gather(parts, mine.contiguous(), group=group)
+        host = torch.stack(parts).cpu().reshape(self.world, self.world, self.e_loc)  # [source, destination, local expert]
+        send_splits = [int(v) for v in host[self.rank].sum(dim=1)]
+        recv_splits = [int(v) for v in host[:, self.rank].sum(dim=1)]
+        recv_counts = host[:, self.rank].contiguous().to(torch.int32).to(x.device, non_blocking=True)
+        recv_rows = exchange_rows(send_rows, send_splits, recv_splits, group, host_staging)
         back = self.compute(recv_rows, recv_counts)
-        returned = exchange_rows(back, recv_splits, ctx["send_splits"], group)
+        returned = exchange_rows(back, recv_splits, send_splits, group, host_staging)
         return self.finish(ctx, returned)

@@ -13,6 +13,17 @@ import torch
 from . import binding as B
 
 
+def draw_samples(plan: B.MoEPlan, batch: int, seq_len: int, n_iter: int, seed: int):
+    """n_iter Monte-Carlo samples X ~ N(0,1)^{(batch * seq_len) x H} (Algorithm 1's input law), drawn on
+    the device one at a time from one seeded generator and rounded to the plan's dtype."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    for _ in range(n_iter):
+        x = torch.empty((batch * seq_len, plan.d), dtype=torch.float32, device="cuda")
+        x.normal_(0.0, 1.0, generator=g)
+        yield x.to(plan.dtype)
+
+
 def perturbation_profile(plan: B.MoEPlan, weights: B.moe_layer_weights_t, k_base: int, renorm: bool, *,
                          batch: int = 16, seq_len: int = 128, n_iter: int = 8, seed: int = 0,
                          samples: Optional[Iterable[torch.Tensor]] = None) -> Dict[int, float]:
@@ -23,15 +34,7 @@ def perturbation_profile(plan: B.MoEPlan, weights: B.moe_layer_weights_t, k_base
     Returns {k: mean Delta_k}; by construction the entry for k_base is exactly 0.
     """
     if samples is None:
-        g = torch.Generator(device="cuda")
-        g.manual_seed(seed)
-
-        def draw():
-            for _ in range(n_iter):
-                x = torch.empty((batch * seq_len, plan.d), dtype=torch.float32, device="cuda")
-                x.normal_(0.0, 1.0, generator=g)
-                yield x.to(plan.dtype)
-        samples = draw()
+        samples = draw_samples(plan, batch, seq_len, n_iter, seed)
     total = [0.0] * k_base
     n = 0
     for x in samples:
@@ -54,15 +57,7 @@ def allocate(plan: B.MoEPlan, layers, k_base: int, budget: int, renorm: bool, *,
     tensors used for every layer (otherwise drawn once from N(0,1) with ``seed``).
     Returns (k_vec, phi, D) with D a list of L rows of k_base means.
     """
-    if samples is None:
-        g = torch.Generator(device="cuda")
-        g.manual_seed(seed)
-        samples = []
-        for _ in range(n_iter):
-            x = torch.empty((batch * seq_len, plan.d), dtype=torch.float32, device="cuda")
-            x.normal_(0.0, 1.0, generator=g)
-            samples.append(x.to(plan.dtype))
-    samples = list(samples)
+    samples = list(draw_samples(plan, batch, seq_len, n_iter, seed) if samples is None else samples)
     D = []
     for w in layers:
         prof = perturbation_profile(plan, w, k_base, renorm, samples=samples)

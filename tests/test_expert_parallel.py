@@ -162,3 +162,119 @@ def test_ranks_run_in_turn_on_one_gpu_match_the_oracle_and_the_one_gpu_layer(sha
     finally:
         for rk in ranks:
             rk.close()
+
+
+def _forward_worker(rank, world, port, out):
+    """One rank of a two-process expert-parallel layer; both processes use GPU 0 and exchange rows
+    through host memory over gloo.  Neither process's kernels wait for the other's: the ranks meet
+    in the host-side collectives only."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    from oracle import moe_oracle as orc
+    from paper_2509_02753_b200 import synth
+    from parity import assert_out_close, oracle_weights
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        torch.cuda.set_device(0)
+        dtype = torch.bfloat16
+        wl = synth.Workload("ep2", d=256, E=16, I=256, k_base=4, L=1, I_shared=128, shared_gate=True,
+                            router_bias_std=0.4, w_std=0.02)
+        k, renorm, scale = 3, False, 1.25
+        T = [300, 41][rank]
+        w = synth.make_layer(wl, 0, dtype, "cuda")
+        x = synth.make_tokens(wl, T, dtype, "cuda", seed=20 + rank)
+        layer = ep.ExpertParallelLayer(wl.d, wl.E, wl.I, 300, 4, dtype, w, rank, world, I_shared=wl.I_shared,
+                                       shared_gate=True, routed_scale=scale)
+        try:
+            ok, worst = True, 0.0
+            for rep in range(2):                  # the second call reuses every buffer of the first
+                y = layer.forward(x, k, renorm, host_staging=True)
+                torch.cuda.synchronize()
+                ref = orc.moe_layer(x.cpu(), oracle_weights(synth.to_host(w)), k, renorm, shared_gate=True, routed_scale=scale)
+                safe = ref.margin > 1e-3
+                worst = max(worst, assert_out_close(y.float().cpu().numpy()[safe], ref.y[safe], dtype, "two-process forward"))
+                ok = ok and layer.router_plan.device_status() == 0 and layer.local_plan.device_status() == 0
+            out.put((rank, bool(ok), float(worst)))
+        finally:
+            layer.close()
+        dist.barrier()
+    except Exception as e:      # the parent must not wait for a queue entry that never comes
+        out.put((rank, False, repr(e)))
+        raise
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.gpu
+def test_forward_end_to_end_with_two_processes_sharing_one_gpu():
+    """ExpertParallelLayer.forward itself (route, pack, count all-gather, row all-to-all, device-side
+    regrouping, local experts, all-to-all back, combine) with world = 2, against the oracle."""
+    sys_path_root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    os.environ["PYTHONPATH"] = os.pathsep.join([sys_path_root, os.path.join(sys_path_root, "tests"),
+                                                os.environ.get("PYTHONPATH", "")])
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_forward_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    results = sorted(out.get(timeout=300) for _ in range(2))
+    for p in procs:
+        p.join(timeout=120)
+    assert all(ok for _, ok, _ in results), results
+    assert all(p.exitcode == 0 for p in procs)
+
+
+@pytest.mark.gpu
+def test_regroup_kernel_matches_the_reference_bookkeeping_and_bad_counts_are_caught():
+    from paper_2509_02753_b200 import binding as B
+    g = torch.Generator().manual_seed(5)
+    for world, e_loc in [(1, 4), (2, 3), (4, 16), (8, 1), (3, 5), (8, 128)]:
+        with B.MoEPlan(64, e_loc, 64, 64, 1, torch.float32) as plan:
+            for trial in range(3):
+                rc = torch.randint(0, 40 if trial else 1, (world, e_loc), generator=g, dtype=torch.int32)
+                n = int(rc.sum())
+                to_em, inv, per = B.moe_regroup_index(plan.handle, rc.cuda(), n)
+                assert plan.device_status() == 0
+                assert to_em.cpu().tolist() == _brute_regroup(rc.numpy())
+                ref_em, ref_inv, ref_per = ep.regroup_index(rc)
+                assert torch.equal(inv.cpu(), ref_inv) and torch.equal(per.cpu(), ref_per)
+            # counts that claim one row more than the buffers hold: nothing is written, the status says so
+            rc = torch.ones((world, e_loc), dtype=torch.int32)
+            n = world * e_loc - 1
+            to_em = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+            inv = to_em.clone()
+            per = torch.full((e_loc,), -7, dtype=torch.int32, device="cuda")
+            lib = B.load_library()
+            assert lib.moe_regroup_index(plan.handle, rc.cuda().data_ptr(), world, n, to_em.data_ptr(), inv.data_ptr(),
+                                         per.data_ptr(), None) == 0
+            assert plan.device_status() == -8            # MOE_ERR_DEVICE_CHECK
+            assert bool((to_em == -7).all()) and bool((inv == -7).all()) and bool((per == 0).all())
+
+
+@pytest.mark.gpu
+def test_experts_forward_refuses_counts_that_do_not_match_the_rows_given():
+    """Counts that arrive over a network may not match the buffers: the device check finds a sum that
+    differs from n_rows, computes nothing (the guard rows behind the output stay as they were) and
+    moe_device_status reports it; the next valid call works."""
+    from paper_2509_02753_b200 import binding as B
+    from paper_2509_02753_b200 import synth
+    wl = synth.Workload("chk", d=256, E=4, I=256, k_base=1, L=1)
+    w = B.make_weights(synth.make_layer(wl, 0, torch.bfloat16, "cuda"))
+    n = 200
+    x = synth.make_tokens(wl, n, torch.bfloat16, "cuda")
+    with B.MoEPlan(wl.d, wl.E, wl.I, 512, 1, torch.bfloat16) as plan:
+        good = torch.tensor([50, 70, 0, 80], dtype=torch.int32, device="cuda")
+        o_ok = torch.zeros((n, wl.d), dtype=torch.float32, device="cuda")
+        B.moe_experts_forward(plan.handle, x, good, w, o_ok)
+        assert plan.device_status() == 0 and float(o_ok.abs().sum()) > 0
+        bad = torch.tensor([50, 70, 1, 80], dtype=torch.int32, device="cuda")       # sums to n + 1
+        o = torch.full((n + 64, wl.d), 7.0, dtype=torch.float32, device="cuda")
+        B.moe_experts_forward(plan.handle, x, bad, w, o[:n])
+        assert plan.device_status() == -8
+        assert bool((o == 7.0).all())
+        o2 = torch.zeros((n, wl.d), dtype=torch.float32, device="cuda")
+        B.moe_experts_forward(plan.handle, x, good, w, o2)
+        assert plan.device_status() == 0 and torch.equal(o2, o_ok)

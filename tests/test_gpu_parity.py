@@ -242,6 +242,49 @@ def test_chunked_host_entry_point_matches_device_entry_point():
             assert plan.device_status() == 0
 
 
+def test_debug_workspace_guard_bands_stay_intact_and_no_kernel_reads_stale_scratch(monkeypatch):
+    """Plans made with LEXI_DEBUG_GUARD=1 put every workspace sub-buffer between guard bands and fill
+    the scratch buffers with 0xFF bytes (NaN, -1) before every call.  Every schedule then still agrees
+    with the oracle (nothing reads a value the call did not write: a NaN or a -1 index would show) and
+    moe_device_status, which compares the bands, stays 0 (nothing writes outside its buffer) - on ragged
+    shapes, a model-shaped decode, ridge and prefill call, the one-launch kernel and a stack."""
+    monkeypatch.setenv("LEXI_DEBUG_GUARD", "1")
+    wl = _custom("guard", d=192, E=5, I=320, I_shared=448, shared_gate=True, bias=0.5)
+    for T in (1, 37, 130, 700):
+        w, x, w_host = _small(wl, T, torch.bfloat16)
+        with _plan(wl, 700, 5, torch.bfloat16, routed_scale=1.25) as plan:
+            for sched in _schedules(plan):
+                plan.set_schedule(sched)
+                check_layer(plan, x, w, 2, False, shared_gate=True, routed_scale=1.25, w_host=w_host)
+                check_layer(plan, x, w, 5, True, shared_gate=True, routed_scale=1.25, w_host=w_host)
+    wq = synth.WORKLOADS["qwen15"]
+    w = synth.make_layer(wq, 0, torch.bfloat16, DEV)
+    w_host = synth.to_host(w)
+    for T, k in ((4, 4), (64, 4), (2048, 2), (8192, 4)):
+        x = synth.make_tokens(wq, T, torch.bfloat16, DEV)
+        toks = None if T <= 64 else np.random.default_rng(T).choice(T, 24, replace=False)
+        with _plan(wq, T, 4, torch.bfloat16) as plan:
+            check_layer(plan, x, w, k, False, shared_gate=True, tokens=toks, w_host=w_host)
+    ws = _custom("gstack", d=256, E=16, I=256, I_shared=128, shared_gate=True, bias=0.3, L=4, k_base=6)
+    layers, x = _stack_case(ws, 4, 96, torch.bfloat16)
+    structs = [B.make_weights(w_) for w_ in layers]
+    ows = [oracle_weights(synth.to_host(w_)) for w_ in layers]
+    k_vec = [6, 2, 4, 1]
+    h_ref, _, margins = orc.moe_stack(x.cpu(), ows, k_vec, False, shared_gate=True)
+    safe = np.all(margins > 1e-3, axis=0)
+    with _plan(ws, 96, 6, torch.bfloat16) as plan:
+        for T in (96, 6):
+            h = x[:T].clone()
+            plan.stack_forward(h, structs, k_vec, False)
+            assert plan.device_status() == 0
+            assert_out_close(h.float().cpu().numpy()[safe[:T]], h_ref[:T][safe[:T]], torch.bfloat16, "(stack, debug workspace)")
+    monkeypatch.delenv("LEXI_DEBUG_GUARD")
+    with _plan(ws, 96, 6, torch.bfloat16) as plain, monkeypatch.context() as m:
+        m.setenv("LEXI_DEBUG_GUARD", "1")
+        with _plan(ws, 96, 6, torch.bfloat16) as guarded:
+            assert guarded.workspace_bytes > plain.workspace_bytes       # the bands are really there
+
+
 # --------------------------------------------------------------------------- model-shaped layers
 
 @pytest.mark.parametrize("T,k", [(1, 4), (8, 4), (64, 4), (64, 1), (2048, 4), (2048, 2), (8192, 4), (8192, 1)])
