@@ -503,6 +503,32 @@ def run_ours(args):
                 del lay_p, ws_p
                 torch.cuda.empty_cache()
 
+    # ---- one hot expert (Section 3: "token-to-expert routing balance"): the router bias of expert 0
+    #      is raised until it takes a large share of the tokens; the schedule is still chosen from the
+    #      mean load T k / E while the tile lists follow the actual counts
+    skew = []
+    if args.sweep and world == 1 and wl.router_bias_std > 0:
+        hot = []
+        for w_ in layers[:2]:
+            w2 = dict(w_)
+            w2["router_bias"] = w_["router_bias"].clone()
+            w2["router_bias"][0] += 3.0
+            hot.append(w2)
+        ws_hot = [B.make_weights(w_) for w_ in hot]
+        for Ts in (64, 512):
+            if Ts > max_T:
+                continue
+            xs = synth.make_tokens(wl, Ts, dtype, device, seed=6)
+            ys = torch.empty_like(xs)
+            for label, ws_ in (("seeded bias", wsets[:2]), ("expert 0 hot", ws_hot)):
+                ms_s, _ = run_case(B, plan, wl, ws_, xs, ys, k, 20, 5, False)
+                rep = case_report(B, plan, wl, Ts, k, ms_s / 20, {}, peaks, device)
+                counts = plan.last_routing(Ts, k, device)[2]
+                skew.append({"T": Ts, "k": k, "router": label, "schedule": rep["schedule"],
+                             "largest_expert_rows": int(counts.max()), "touched_experts": rep["touched_experts"],
+                             "ms": rep["ms"], "frac_roof_measured": rep["frac_roof_measured"]})
+        del hot, ws_hot
+
     # ---- whole stacks with uniform and per-layer k (rank 0 at N = 1)
     stacks = []
     if args.stacks and world == 1:
@@ -569,6 +595,7 @@ def run_ours(args):
         detail += [{"detail": "k_sweep", **c} for c in k_sweep]
         detail += [{"detail": "stack", **c} for c in stacks]
         detail += [{"detail": "pruning_shape", **c} for c in pruning]
+        detail += [{"detail": "skewed_load", "workload": wl.name, **c} for c in skew]
         if stage1:
             detail.append({"detail": "stage1", **stage1})
         if expert_parallel:

@@ -155,13 +155,6 @@ cudaError_t launch_profile(const CombineArgs &a, int renorm, float *partial, dou
 
 // ---- one launch for a whole stack of layers at tiny decode sizes (decode_stack.cu) ------------
 constexpr int kFusedMaxTokens = 8;
-#ifndef LEXI_FUSED_WARPS
-#define LEXI_FUSED_WARPS 12
-#endif
-// warps per CTA (one CTA per SM).  12 leaves each thread 168 registers: two chunks of weights in
-// flight per warp without spills; 16 warps (128 registers, spills) measured 5-10 % slower.
-constexpr int kFusedWarps = LEXI_FUSED_WARPS;
-constexpr int kFusedThreads = kFusedWarps * 32;
 constexpr int kFusedMaxCtaBlocks = 512;   // gate/up row blocks of one stream that may fall to one CTA
 constexpr int kFusedMaxCtaRows = 64;      // rows of the residual stream one CTA may own (d <= 64 x SMs)
 constexpr int kStackMaxLayers = 44;       // layers per launch (their pointers travel as kernel parameters)
