@@ -407,6 +407,16 @@ int moe_plan_stage_times(moe_plan_t *plan, float *ms, int32_t *n_calls);
  */
 int moe_plan_touched_experts(moe_plan_t *plan, int64_t *total, void *cuda_stream);
 
+/*
+ * moe_plan_tile_stats (measurement aid): like moe_plan_touched_experts, plus how much padded work the
+ * tensor-core GEMMs executed.  out3[0] = touched routed experts, out3[1] / out3[2] = token rows the MMAs
+ * ran for the routed experts / the shared expert (each expert's rows rounded up to the tile heights
+ * the kernels use), all summed over the layer calls on the kernel-chain schedules since the last read
+ * of either function; synchronises the stream and resets the sums.  Against T * k_l and T algorithmic
+ * rows per call this gives executed over algorithmic flops.
+ */
+int moe_plan_tile_stats(moe_plan_t *plan, int64_t *out3, void *cuda_stream);
+
 /* Number of kernel launches this plan has issued since it was created. */
 uint64_t moe_plan_launch_count(const moe_plan_t *plan);
 

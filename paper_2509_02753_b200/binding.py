@@ -28,7 +28,7 @@ EXPORTS = (
     "moe_plan_get_schedule", "moe_layer_forward", "moe_layer_forward_host", "moe_stack_forward",
     "moe_route_from_logits", "moe_last_routing", "moe_device_status", "moe_plan_launch_count",
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
-    "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts",
+    "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts", "moe_plan_tile_stats",
     "moe_debug_fused_stamps", "moe_host_pipeline_submit", "moe_host_pipeline_wait",
     "moe_route", "moe_gather_rows", "moe_regroup_index", "moe_experts_forward", "moe_combine",
     "moe_debug_wait_timeout", "moe_debug_barrier_timeout", "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
@@ -86,6 +86,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_debug_barrier_timeout.argtypes = [vp, i32, vp]
     lib.moe_last_residual_f32.argtypes = [vp, vp, i32, vp]
     lib.moe_plan_touched_experts.argtypes = [vp, P(ctypes.c_int64), vp]
+    lib.moe_plan_tile_stats.argtypes = [vp, P(ctypes.c_int64), vp]
     lib.moe_debug_fused_stamps.argtypes = [vp, i32, P(ctypes.c_uint64), i32, P(i32), vp]
     lib.moe_host_pipeline_submit.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, vp, P(ctypes.c_int64)]
     lib.moe_host_pipeline_wait.argtypes = [vp, ctypes.c_int64]
@@ -396,6 +397,14 @@ def moe_plan_touched_experts(plan: int, stream=None) -> int:
     _check("moe_plan_touched_experts",
            load_library().moe_plan_touched_experts(plan, ctypes.byref(n), _stream(stream)))
     return int(n.value)
+
+
+def moe_plan_tile_stats(plan: int, stream=None):
+    """(touched experts, MMA rows executed for the routed experts, ... for the shared expert) summed over the
+    kernel-chain layer calls since the last read."""
+    out = (ctypes.c_int64 * 3)()
+    _check("moe_plan_tile_stats", load_library().moe_plan_tile_stats(plan, out, _stream(stream)))
+    return int(out[0]), int(out[1]), int(out[2])
 
 
 def moe_debug_fused_stamps(plan: int, enable: int, read: bool = False, stream=None):

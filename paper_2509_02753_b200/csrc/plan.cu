@@ -879,6 +879,19 @@ int moe_plan_touched_experts(moe_plan_t *p, int64_t *total, void *cuda_stream) {
     return MOE_OK;
 }
 
+int moe_plan_tile_stats(moe_plan_t *p, int64_t *out3, void *cuda_stream) {
+    if (!p || !out3) return MOE_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    int32_t host[3] = {0, 0, 0};
+    if (cudaMemcpyAsync(host, p->ws.stats, sizeof(host), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemsetAsync(p->ws.stats, 0, sizeof(host), s) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    for (int i = 0; i < 3; ++i) out3[i] = host[i];
+    return MOE_OK;
+}
+
 int moe_debug_wait_timeout(moe_plan_t *p, int32_t limit_us, void *cuda_stream) {
     if (!p || limit_us < 1 || limit_us > 1000000) return MOE_ERR_INVALID_ARG;
     if (launch_wait_probe(p->ws.status, (unsigned long long)limit_us * 1000ull, (cudaStream_t)cuda_stream) != cudaSuccess) {

@@ -25,7 +25,9 @@ struct TileBuildArgs {
     // reduce over a longer K than the routed ones; null tiles (rows = 0) are slipped in behind the
     // shared tiles so that every consumer ends up with the same amount of work
     int32_t rr2;
-    int32_t *stats;   // stats[0] += number of routed experts that received at least one token
+    int32_t *stats;   // stats[0] += routed experts that received at least one token; stats[1], stats[2] += token
+                      // rows the MMAs of this call execute for the routed / shared groups (valid rows rounded up to
+                      // the MMA heights the kernels use): executed = padded work, against T k_l and T algorithmic rows
 };
 
 // Shared-memory scratch of build_tiles_block.
@@ -56,6 +58,11 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
         const int g = group_of(sidx);
         const int mblk = (rows_of(g) + a.tile_rows - 1) / a.tile_rows;
         if (rank == 0 && a.stats && g != a.E && rows_of(g) > 0) atomicAdd(a.stats, 1);
+        if (rank == 0 && a.stats && !a.direct) {
+            const int r = rows_of(g), rem = r % a.tile_rows;
+            const int small = a.tile_rows / 2;          // a last block of at most half a tile runs at half height
+            atomicAdd(a.stats + (g == a.E ? 2 : 1), r / a.tile_rows * a.tile_rows + (rem == 0 ? 0 : (rem <= small ? small : a.tile_rows)));
+        }
         sm.pre1[sidx] = mblk1_of(g) * (g == a.E ? n1_shared : n1_routed);
         sm.pre2[sidx] = mblk * n2 * (g == a.E ? a.ksplit_shared : a.ksplit_routed);
     }
