@@ -389,12 +389,20 @@ __device__ __forceinline__ void route_token_n(const float *zrow, int E, int k, i
         z[j] = e < E ? zrow[e] : -CUDART_INF_F;
         rank[j] = 0;
     }
-    for (int e2 = 0; e2 < E; ++e2) {
-        const float o = zrow[e2];
+    // four logits per step (one 16-byte broadcast load, independent compares: a single warp routes a
+    // token, so the loop's latency is what counts); columns beyond E compare as -inf
+#pragma unroll 4
+    for (int e2 = 0; e2 < E; e2 += 4) {
+        const float4 o4 = *reinterpret_cast<const float4 *>(zrow + e2);
+        const float o[4] = {o4.x, o4.y, o4.z, o4.w};
 #pragma unroll
-        for (int j = 0; j < NJ; ++j) {
-            const int e = lane + 32 * j;
-            rank[j] += (o > z[j] || (o == z[j] && e2 < e)) ? 1 : 0;
+        for (int u = 0; u < 4; ++u) {
+            const float ov = e2 + u < E ? o[u] : -CUDART_INF_F;
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) {
+                const int e = lane + 32 * j;
+                rank[j] += (ov > z[j] || (ov == z[j] && e2 + u < e)) ? 1 : 0;
+            }
         }
     }
     float m = z[0];

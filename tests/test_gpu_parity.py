@@ -128,6 +128,34 @@ def test_unused_experts_and_heavy_skew():
             check_layer(plan, x, w, 1, False)
 
 
+def test_tile_statistics_count_the_rows_the_tensor_cores_run():
+    """moe_plan_tile_stats: touched experts and the token rows the GEMMs execute, from the counts the
+    call produced: every expert's rows in tiles of 256 (CTA pairs) or 128 (one CTA), a last tile of at
+    most half a tile at half height; the shared expert runs all T tokens."""
+    wl = _custom("stats", d=256, E=6, I=256, I_shared=256, bias=0.8)
+    T, k = 1500, 2
+    w, x, _ = _small(wl, T, torch.bfloat16)
+    ws = B.make_weights(w)
+    y = torch.empty_like(x)
+    with _plan(wl, T, k, torch.bfloat16) as plan:
+        for sched, tile in ((B.MOE_SCHED_PREFILL, 256), (B.MOE_SCHED_PREFILL_1CTA, 128)):
+            plan.set_schedule(sched)
+            B.moe_plan_tile_stats(plan.handle)
+            for _ in range(3):
+                plan.layer_forward(x, ws, k, False, y)
+            counts = plan.last_routing(T, k)[2]
+            touched, rows_r, rows_s = B.moe_plan_tile_stats(plan.handle)
+
+            def padded(c):
+                rem = c % tile
+                return c // tile * tile + (0 if rem == 0 else tile // 2 if rem <= tile // 2 else tile)
+            assert touched == 3 * int((counts > 0).sum())
+            assert rows_r == 3 * sum(padded(int(c)) for c in counts)
+            assert rows_s == 3 * padded(T)
+            assert B.moe_plan_tile_stats(plan.handle) == (0, 0, 0)        # reading resets
+        assert plan.device_status() == 0
+
+
 def test_zero_tokens_is_a_no_op_and_bad_arguments_are_refused():
     wl = synth.WORKLOADS["tiny"]
     w = B.make_weights(synth.make_layer(wl, 0, torch.bfloat16, DEV))
