@@ -539,7 +539,7 @@ __device__ __forceinline__ void run_stream(const Ctx &x, int warp, uint32_t nblk
     uint32_t q = qa;
     uint32_t rb = qa / NC;                    // block of chunk q and the flat index where it ends
     uint32_t blk_end = (rb + 1) * NC;
-    const __nv_bfloat16 *xrow = x.xs + x.g * x.xstride + x.c * 8;
+    const __nv_bfloat16 *xrow = x.xs + (x.g < x.a.T ? x.g : x.a.T) * x.xstride + x.c * 8;   // token slots >= T share one row of zeros
 #pragma unroll 1
     while (true) {
 #pragma unroll
@@ -659,7 +659,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) decode_stack_kernel(const __
     };
     {
         const int vec_per_row = xstride / 8;
-        for (int i = tid; i < kFT * vec_per_row; i += kFusedThreads) {
+        const int xrows = T < kFT ? T + 1 : kFT;        // the T tokens and, with fewer than 8, one row of zeros for the other MMA columns
+        for (int i = tid; i < xrows * vec_per_row; i += kFusedThreads) {
             const int row = i / vec_per_row, col = (i - row * vec_per_row) * 8;
             if (row >= T || col >= a.d) *reinterpret_cast<uint4 *>(xs + row * xstride + col) = make_uint4(0u, 0u, 0u, 0u);
         }
@@ -913,10 +914,14 @@ __global__ void barrier_probe_kernel(const uint32_t *bar, int32_t *status, unsig
 #define LEXI_CAT(a, b) LEXI_CAT2(a, b)
 #define LEXI_VARIANT(name) LEXI_CAT(name, LEXI_FUSED_WARPS)
 
-size_t LEXI_VARIANT(fused_smem_bytes_w)(int d) {
+// Shared memory for hidden size d and T tokens: the tables and T + 1 (at most 8) rows of h.  What the
+// kernel does not take stays L1, which is where the weight loads in flight are held.
+static size_t smem_bytes(int d, int T) {
     const int dpad = (d + kChunk - 1) / kChunk * kChunk;
-    return ((sizeof(StackSmem) + 15) / 16) * 16 + (size_t)kFT * (dpad + kXPad) * sizeof(__nv_bfloat16);
+    const int rows = T < kFT ? T + 1 : kFT;
+    return ((sizeof(StackSmem) + 15) / 16) * 16 + (size_t)rows * (dpad + kXPad) * sizeof(__nv_bfloat16);
 }
+size_t LEXI_VARIANT(fused_smem_bytes_w)(int d) { return smem_bytes(d, kFT); }
 
 cudaError_t LEXI_VARIANT(fused_prepare_w)(int d) {
     // the attribute belongs to the kernel on the current device, not to a plan: per device it only
@@ -936,7 +941,7 @@ cudaError_t LEXI_VARIANT(launch_decode_stack_w)(const StackArgs &a, int sm_count
     StackArgs args = a;
     void *params[] = {&args};
     const cudaError_t e = cudaLaunchCooperativeKernel((const void *)decode_stack_kernel, dim3(sm_count),
-                                                      dim3(kFusedThreads), params, LEXI_VARIANT(fused_smem_bytes_w)(a.d), s);
+                                                      dim3(kFusedThreads), params, smem_bytes(a.d, a.T), s);
     ++*launches;
     return e;
 }
