@@ -211,6 +211,54 @@ def test_two_calls_are_bit_identical():
             assert torch.equal(a, b)
 
 
+def test_plans_come_and_go_and_share_the_device_without_leaks_or_cross_talk():
+    """Thirty plans created, used on every schedule and destroyed leave the device memory where it
+    was; two plans alive at once, driven from two side streams with calls interleaved, give the bits
+    that each gives alone (a plan owns its workspace, counters and barrier; nothing is global)."""
+    wl = _custom("churn", d=256, E=16, I=384, I_shared=256, shared_gate=True)
+    w = synth.make_layer(wl, 0, torch.bfloat16, DEV)
+    ws = B.make_weights(w)
+    xs = {T: synth.make_tokens(wl, T, torch.bfloat16, DEV, seed=T) for T in (4, 40, 700)}
+    want = {}
+    with _plan(wl, 700, 4, torch.bfloat16) as plan:
+        for T, x in xs.items():
+            want[T] = plan.layer_forward(x, ws, 3, False).clone()
+        assert plan.device_status() == 0
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(30):
+        with _plan(wl, 700, 4, torch.bfloat16) as plan:
+            for T, x in xs.items():
+                assert torch.equal(plan.layer_forward(x, ws, 3, False), want[T])
+            assert plan.device_status() == 0
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free0 - free1 < 32 * 2**20, f"{(free0 - free1) / 2**20:.0f} MiB not returned after 30 plans"
+
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    with _plan(wl, 700, 4, torch.bfloat16) as pa, _plan(wl, 700, 4, torch.bfloat16) as pb:
+        outs = []
+        for rep in range(4):
+            for T in (40, 700):          # kernel chains of the two plans run side by side on the two streams
+                with torch.cuda.stream(s1):
+                    ya = pa.layer_forward(xs[T], ws, 3, False).clone()
+                with torch.cuda.stream(s2):
+                    yb = pb.layer_forward(xs[T], ws, 3, False).clone()
+                outs.append((T, ya, yb))
+            torch.cuda.synchronize()
+            with torch.cuda.stream(s1):      # the one-launch kernel from a side stream, one plan at a time
+                ya = pa.layer_forward(xs[4], ws, 3, False).clone()
+            s1.synchronize()
+            with torch.cuda.stream(s2):
+                yb = pb.layer_forward(xs[4], ws, 3, False).clone()
+            s2.synchronize()
+            outs.append((4, ya, yb))
+        torch.cuda.synchronize()
+        for T, ya, yb in outs:
+            assert torch.equal(ya, want[T]) and torch.equal(yb, want[T])
+        assert pa.device_status() == 0 and pb.device_status() == 0
+
+
 def test_host_buffer_entry_point_matches_device_entry_point():
     wl = synth.WORKLOADS["tiny"]
     w = B.make_weights(synth.make_layer(wl, 0, torch.bfloat16, DEV))
