@@ -507,36 +507,36 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
                     }
                 }
             } else {
-                float *stg = reinterpret_cast<float *>(smem_raw + (bar_base + 256u - raw)) + q * 32 * kStagePitch;
-                // this warp's 32 rows of the tile and its first output column
+                // this warp's 32 rows of the tile and its first output column; the accumulator is read
+                // in fragment layout (16 lanes x 64 columns at a time) and stored straight from the
+                // registers: four threads fill a 32-byte sector, and no shared memory is touched,
+                // which the MMA operand reads and the TMA writes already keep busy
                 const int warp_row0 = half ? 64 * (int)rank + 32 * (q & 1) : 128 * (int)rank + 32 * q;
                 const int col0 = t.n0 + (half ? 128 * (q >> 1) : 0);
                 const int cols = half ? 128 : BN;
                 OutT *wbase = obase + (size_t)(t.row0 + warp_row0) * N + col0;
                 const int rows_here = t.rows - warp_row0;
-                const int rr0 = lane >> 3, cc = 4 * (lane & 7);
+                static_assert(PHASE != 2 || sizeof(OutT) == 4, "the down projection's outputs are fp32");
+                const int fr = lane >> 2, fc = 2 * (lane & 3);
 #pragma unroll 1
-                for (int c = 0; c < cols; c += 32) {
-                    uint32_t v0[16], v1[16];
-                    tmem_ld16(taddr + c, v0);
-                    tmem_ld16(taddr + c + 16, v1);
-                    tmem_ld_wait();
-                    uint4 *wr = reinterpret_cast<uint4 *>(stg + lane * kStagePitch);
+                for (int hl = 0; hl < 2; ++hl) {
+                    const int ra = 16 * hl + fr, rb = ra + 8;
+                    OutT *pa = wbase + (size_t)ra * N + fc, *pb = wbase + (size_t)rb * N + fc;
+                    const bool oka = ra < rows_here, okb = rb < rows_here;
+#pragma unroll 1
+                    for (int c = 0; c < cols; c += 64) {
+                        uint32_t v[32];
+                        tmem_ld_16x256b_x8(taddr + ((uint32_t)(16 * hl) << 16) + c, v);
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        wr[i] = make_uint4(v0[4 * i], v0[4 * i + 1], v0[4 * i + 2], v0[4 * i + 3]);
-                        wr[4 + i] = make_uint4(v1[4 * i], v1[4 * i + 1], v1[4 * i + 2], v1[4 * i + 3]);
+                        for (int j = 0; j < 8; ++j) {
+                            const int col = c + 8 * j;
+                            if (col0 + col + fc + 2 <= N) {
+                                if (oka) *reinterpret_cast<uint2 *>(pa + col) = make_uint2(v[4 * j], v[4 * j + 1]);
+                                if (okb) *reinterpret_cast<uint2 *>(pb + col) = make_uint2(v[4 * j + 2], v[4 * j + 3]);
+                            }
+                        }
                     }
-                    __syncwarp();
-                    const bool col_ok = col0 + c + cc + 4 <= N;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int rr = 4 * j + rr0;
-                        const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * kStagePitch + cc);
-                        if (rr < rows_here && col_ok)
-                            *reinterpret_cast<uint4 *>(wbase + (size_t)rr * N + c + cc) = val;
-                    }
-                    __syncwarp();
                 }
             }
             tc_fence_before();
