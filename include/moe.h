@@ -193,7 +193,11 @@ int moe_layer_forward_host(moe_plan_t *plan, const void *x_host, const moe_layer
  *   up to n_rows are caught on the device: nothing is computed or written and the next
  *   moe_device_status returns MOE_ERR_DEVICE_CHECK.  Only W_gate, W_up, W_down of w are read (a shared
  *   expert is a plan of its own with E = 1).  bf16 plans run the tcgen05 prefill kernels (CTA pairs
- *   from 64 rows per expert), fp32 plans the CUDA-core kernels.
+ *   from 64 rows per expert), fp32 plans the CUDA-core kernels.  out_index (device, [n_rows] int32, or
+ *   NULL): row r of the result is stored at o_rows[out_index[r]] instead of o_rows[r] - with
+ *   moe_regroup_index's to_expert_major the outputs land in arrival order and no copy puts them
+ *   back; an entry outside 0..n_rows-1 drops its row and raises MOE_ERR_DEVICE_CHECK at the next
+ *   moe_device_status.
  * moe_combine: y[t] = routed_scale * sum_j topk_w[t, j] * o_rows[inv_perm[t * k_l + j]]
  *   (+ gamma[t] * o_shared[t], gamma NULL = 1, when o_shared [T, d] fp32 is given), in slot order,
  *   rounded once to the plan's dtype.
@@ -207,7 +211,8 @@ int moe_gather_rows(moe_plan_t *plan, const void *src, const int32_t *row_index,
 int moe_regroup_index(moe_plan_t *plan, const int32_t *recv_counts, int32_t world, int32_t n_rows,
                       int32_t *to_expert_major, int32_t *inverse, int32_t *per_expert, void *cuda_stream);
 int moe_experts_forward(moe_plan_t *plan, const void *x_rows, const int32_t *counts,
-                        const moe_layer_weights_t *w, int32_t n_rows, float *o_rows, void *cuda_stream);
+                        const moe_layer_weights_t *w, int32_t n_rows, float *o_rows,
+                        const int32_t *out_index, void *cuda_stream);
 int moe_combine(moe_plan_t *plan, const float *o_rows, const float *topk_w, const int32_t *inv_perm,
                 const float *o_shared, const float *gamma, int32_t T, int32_t k_l, void *y,
                 void *cuda_stream);

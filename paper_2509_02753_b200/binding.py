@@ -93,7 +93,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_route.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.moe_gather_rows.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
     lib.moe_regroup_index.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
-    lib.moe_experts_forward.argtypes = [vp, vp, vp, P(moe_layer_weights_t), i32, vp, vp]
+    lib.moe_experts_forward.argtypes = [vp, vp, vp, P(moe_layer_weights_t), i32, vp, vp, vp]
     lib.moe_combine.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
     lib.moe_profile_layer.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, P(ctypes.c_double),
                                       P(ctypes.c_double), vp]
@@ -251,13 +251,17 @@ def moe_regroup_index(plan: int, recv_counts: torch.Tensor, n_rows: int, stream=
 
 
 def moe_experts_forward(plan: int, x_rows: torch.Tensor, counts: torch.Tensor, w: moe_layer_weights_t,
-                        o_rows: torch.Tensor, stream=None) -> None:
-    """o_rows[r] = E_e(x_rows[r]) (fp32) for rows grouped by expert as counts says."""
+                        o_rows: torch.Tensor, out_index: Optional[torch.Tensor] = None, stream=None) -> None:
+    """o_rows[r] = E_e(x_rows[r]) (fp32) for rows grouped by expert as counts says; with out_index
+    (int32, one entry per row) row r is stored at o_rows[out_index[r]] instead."""
     assert x_rows.is_cuda and x_rows.is_contiguous() and o_rows.dtype == torch.float32 and o_rows.is_contiguous()
     assert counts.dtype == torch.int32 and counts.is_cuda
+    if out_index is not None:
+        assert out_index.dtype == torch.int32 and out_index.is_cuda and out_index.is_contiguous()
+        assert out_index.numel() == x_rows.shape[0]
     _check("moe_experts_forward", load_library().moe_experts_forward(
         plan, x_rows.data_ptr(), counts.data_ptr(), ctypes.byref(w), x_rows.shape[0], o_rows.data_ptr(),
-        _stream(stream)))
+        None if out_index is None else out_index.data_ptr(), _stream(stream)))
 
 
 def moe_combine(plan: int, o_rows: torch.Tensor, topk_w: torch.Tensor, inv_perm: torch.Tensor, y: torch.Tensor,

@@ -41,7 +41,8 @@ __global__ void __launch_bounds__(256) ffn_simt_kernel(
     const T *A_routed, const T *A_shared, int T_tokens, const int32_t *offsets, int E,
     const T *Bg_routed, const T *Bu_routed, const T *Bg_shared, const T *Bu_shared,
     int K, int N_routed, int N_shared, int K_shared,
-    OutT *out_routed, OutT *out_shared) {
+    OutT *out_routed, OutT *out_shared,
+    const int32_t *row_map, int row_map_n, int32_t *status) {   // row_map: routed output row r goes to row row_map[r]
     __shared__ float As[kBK][kBM + 1];
     __shared__ float Bgs[kBK][kBN + 1];
     __shared__ float Bus[GATED ? kBK : 1][kBN + 1];
@@ -96,13 +97,21 @@ __global__ void __launch_bounds__(256) ffn_simt_kernel(
         for (int i = 0; i < 4; ++i) {
             const int r = m0 + ty * 4 + i;
             if (r >= row_end) continue;
+            int r_out = r;
+            if (row_map != nullptr && !shared) {
+                r_out = row_map[r];
+                if ((unsigned)r_out >= (unsigned)row_map_n) {       // outside the buffer: flagged, dropped
+                    if (status != nullptr) atomicOr(status, kStatusBadIndex);
+                    continue;
+                }
+            }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int n = n0 + tx * 4 + j;
                 if (n >= N) continue;
                 float v = accg[i][j];
                 if (GATED) v = (v / (1.0f + expf(-v))) * accu[i][j];
-                st_from_f32(out + (size_t)r * N + n, v);
+                st_from_f32(out + (size_t)r_out * N + n, v);
             }
         }
     }
@@ -118,14 +127,14 @@ static cudaError_t run_simt(const FfnArgs &a, cudaStream_t s, uint64_t *launches
     ffn_simt_kernel<T, T, true><<<g1, 256, 0, s>>>(
         (const T *)a.x_perm, (const T *)a.x, a.T, a.offsets, a.E,
         (const T *)a.W_gate, (const T *)a.W_up, (const T *)a.Ws_gate, (const T *)a.Ws_up,
-        a.d, a.I, a.I_s, a.d, (T *)a.h, (T *)a.h_s);
+        a.d, a.I, a.I_s, a.d, (T *)a.h, (T *)a.h_s, nullptr, 0, nullptr);
     if (a.mid_event) cudaEventRecord(a.mid_event, s);
     // phase 2: K = I (I_s for the shared expert), outputs o / o_s in fp32
     dim3 g2((a.d + kBN - 1) / kBN, groups);
     ffn_simt_kernel<T, float, false><<<g2, 256, 0, s>>>(
         (const T *)a.h, (const T *)a.h_s, a.T, a.offsets, a.E,
         (const T *)a.W_down, nullptr, (const T *)a.Ws_down, nullptr,
-        a.I, a.d, a.d, a.I_s, (float *)a.o, (float *)a.o_s);
+        a.I, a.d, a.d, a.I_s, (float *)a.o, (float *)a.o_s, a.o_index, a.T * a.k, a.status);
     *launches += 2;
     return cudaGetLastError();
 }

@@ -44,7 +44,18 @@ struct TcParams {
     int32_t *status;
     const int32_t *pos;          // direct mode: pos[group * pos_stride + token] = output row or -1
     int32_t pos_stride;
+    const int32_t *row_map;      // not null: routed output row r goes to row row_map[r] (0 <= row_map[r] < row_map_n)
+    int32_t row_map_n;
 };
+
+// Where routed output row `row` is stored: itself, or its entry of the row map; an entry outside
+// the buffer raises the bad-index status and the row is dropped (-1).
+__device__ __forceinline__ int mapped_row(const TcParams &p, int row) {
+    if (p.row_map == nullptr) return row;
+    const int v = p.row_map[row];
+    if ((unsigned)v >= (unsigned)p.row_map_n) { atomicOr(p.status, kStatusBadIndex); return -1; }
+    return v;
+}
 
 // Phase-2 tiles of the prefill schedule pass their fp32 output through a per-warp staging buffer
 // (32 rows x 32 columns, row pitch 36 floats) so that global stores are row-contiguous.
@@ -222,6 +233,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
                 out_row = row_ok ? p.pos[t.group * p.pos_stride + row_in_tile] : -1;
                 row_ok = out_row >= 0;
             }
+            if (PHASE == 2 && p.row_map != nullptr && !shared && row_ok) {
+                out_row = mapped_row(p, out_row);
+                row_ok = out_row >= 0;
+            }
             const bool got = mbar_wait(tfull_bar(buf), bph, p.status);
             if (!__all_sync(0xffffffffu, got)) break;
             tc_fence_after();
@@ -258,6 +273,20 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
                               (size_t)(t.row0 + warp_row0) * N + t.n0;
                 const int rows_here = min(t.rows - warp_row0, small ? 16 : 32);   // valid rows of this warp
                 const int rr0 = lane >> 3, cc = 4 * (lane & 7);
+                long long drow[8];                 // destination of the eight rows this lane stores, relative to wbase
+                uint32_t row_mask = 0;             // bit j: row 4 j + rr0 exists and has a destination
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int rr = 4 * j + rr0;
+                    bool ok_row = rr < rows_here;
+                    drow[j] = rr;
+                    if (p.row_map != nullptr && !shared && ok_row) {
+                        const int m = mapped_row(p, t.row0 + warp_row0 + rr);
+                        ok_row = m >= 0;
+                        drow[j] = (long long)m - (t.row0 + warp_row0);
+                    }
+                    row_mask |= (ok_row ? 1u : 0u) << j;
+                }
 #pragma unroll 1
                 for (int c = 0; c < BN; c += 32) {
                     uint32_t v0[16], v1[16];
@@ -276,8 +305,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid_cons
                     for (int j = 0; j < 8; ++j) {
                         const int rr = 4 * j + rr0;
                         const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * kStagePitch + cc);
-                        if (rr < rows_here && col_ok)
-                            *reinterpret_cast<uint4 *>(wbase + (size_t)rr * N + c + cc) = val;
+                        if (((row_mask >> j) & 1u) && col_ok)
+                            *reinterpret_cast<uint4 *>(wbase + drow[j] * N + c + cc) = val;
                     }
                     __syncwarp();
                 }
@@ -521,8 +550,15 @@ ffn_tc_pair_kernel(const __grid_constant__ CUtensorMap mapA_routed, const __grid
 #pragma unroll 1
                 for (int hl = 0; hl < 2; ++hl) {
                     const int ra = 16 * hl + fr, rb = ra + 8;
-                    OutT *pa = wbase + (size_t)ra * N + fc, *pb = wbase + (size_t)rb * N + fc;
-                    const bool oka = ra < rows_here, okb = rb < rows_here;
+                    bool oka = ra < rows_here, okb = rb < rows_here;
+                    long long da = ra, db = rb;            // destination rows relative to wbase
+                    if (p.row_map != nullptr && !shared) {
+                        const int first = t.row0 + warp_row0;
+                        const int ma = oka ? mapped_row(p, first + ra) : -1, mb = okb ? mapped_row(p, first + rb) : -1;
+                        oka = ma >= 0; okb = mb >= 0;
+                        da = (long long)ma - first; db = (long long)mb - first;
+                    }
+                    OutT *pa = wbase + da * N + fc, *pb = wbase + db * N + fc;
 #pragma unroll 1
                     for (int c = 0; c < cols; c += 64) {
                         uint32_t v[32];
@@ -830,6 +866,7 @@ int tc_ffn_forward(TcState *st, const moe_config_t &c, const Workspace &ws, cons
     p2.slab_stride_shared = (unsigned long long)a.T * a.d;
     p2.status = ws.status;
     p2.pos = nullptr; p2.pos_stride = 0;
+    p2.row_map = a.o_index; p2.row_map_n = rows;
 
     cudaError_t e1, e2;
     const bool ch = a.chained && !a.mid_event;

@@ -132,6 +132,8 @@ struct FfnArgs {
     cudaEvent_t begin_event; // recorded right before the first GEMM phase when not null
     cudaEvent_t mid_event;   // recorded between the two GEMM phases when not null
     size_t x_perm_rows = 0;  // rows that exist behind x_perm (0: the plan's own buffer, pairs + 128)
+    const int32_t *o_index = nullptr;   // not null: routed output row r is stored at row o_index[r] of o (checked against T k)
+    int32_t *status = nullptr;          // device status word (where o_index is checked by the CUDA-core kernels)
 };
 cudaError_t launch_ffn_simt(const FfnArgs &a, cudaStream_t s, uint64_t *launches);
 

@@ -656,7 +656,7 @@ int moe_regroup_index(moe_plan_t *p, const int32_t *recv_counts, int32_t world, 
 }
 
 int moe_experts_forward(moe_plan_t *p, const void *x_rows, const int32_t *counts, const moe_layer_weights_t *w,
-                        int32_t n_rows, float *o_rows, void *cuda_stream) {
+                        int32_t n_rows, float *o_rows, const int32_t *out_index, void *cuda_stream) {
     if (!p || !x_rows || !counts || !o_rows || !w || !w->W_gate || !w->W_up || !w->W_down) return MOE_ERR_INVALID_ARG;
     const moe_config_t &c = p->cfg;
     if (n_rows < 0 || (int64_t)n_rows > (int64_t)c.max_T * c.max_k) return MOE_ERR_INVALID_ARG;
@@ -676,6 +676,8 @@ int moe_experts_forward(moe_plan_t *p, const void *x_rows, const int32_t *counts
                w->W_gate, w->W_up, w->W_down, nullptr, nullptr, nullptr,
                ws.h, ws.h_s, o_rows, ws.o_s, false, nullptr, nullptr};
     fa.x_perm_rows = (size_t)n_rows;
+    fa.o_index = out_index;
+    fa.status = ws.status;
     if (c.dtype != MOE_BF16 || !tc_shape_ok(c) || p->forced_schedule == MOE_SCHED_SIMT) {
         if (launch_ffn_simt(fa, s, &p->launches) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
         return MOE_OK;

@@ -10,7 +10,7 @@ the expert work.  Rank r holds the experts [r * E / R, (r + 1) * E / R) and the 
              (moe_gather_rows): the rows for rank 0 come first, then those for rank 1, ...
     exchange pairs-per-(destination, expert) counts, then the rows, all-to-all
     compute  regroup what arrived from source-major to expert-major order, run the local experts
-             (moe_experts_forward), put the outputs back into arrival order
+             (moe_experts_forward), whose down projection stores the outputs in arrival order
     exchange the fp32 outputs back, all-to-all
     finish   gated sum over each token's slots plus the shared expert (moe_combine)
 
@@ -156,12 +156,12 @@ class ExpertParallelLayer:
         n = recv_rows.shape[0]
         to_em, inverse, per_expert = B.moe_regroup_index(self.local_plan.handle, recv_counts.contiguous(), n)
         grouped = torch.empty_like(recv_rows)
-        out_em = torch.empty((n, self.d), dtype=torch.float32, device=recv_rows.device)
-        back = torch.empty_like(out_em)
+        back = torch.empty((n, self.d), dtype=torch.float32, device=recv_rows.device)
         if n > 0:
             B.moe_gather_rows(self.local_plan.handle, recv_rows, to_em, grouped)
-            B.moe_experts_forward(self.local_plan.handle, grouped, per_expert.contiguous(), self.w_local, out_em)
-            B.moe_gather_rows(self.local_plan.handle, out_em, inverse, back)
+            # the down projection stores row r of the expert-major order at its arrival index
+            B.moe_experts_forward(self.local_plan.handle, grouped, per_expert.contiguous(), self.w_local, back,
+                                  out_index=to_em.contiguous())
         return back
 
     # -- step 3: gated sum of the returned outputs (rows in the order they were sent), shared expert

@@ -278,3 +278,47 @@ def test_experts_forward_refuses_counts_that_do_not_match_the_rows_given():
         o2 = torch.zeros((n, wl.d), dtype=torch.float32, device="cuda")
         B.moe_experts_forward(plan.handle, x, good, w, o2)
         assert plan.device_status() == 0 and torch.equal(o2, o_ok)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype,n,counts,sched", [
+    (torch.bfloat16, 900, [300, 17, 0, 583], "pairs"),        # 256-row pair tiles, a half-height tile, an empty expert
+    (torch.bfloat16, 150, [40, 64, 1, 45], "one-cta"),        # one-CTA tiles, M = 64 and M = 128
+    (torch.float32, 200, [50, 70, 0, 80], "simt"),            # CUDA-core kernels
+])
+def test_experts_forward_stores_rows_where_the_index_says(dtype, n, counts, sched):
+    """With out_index the down projection stores row r at o_rows[out_index[r]]: the result is the
+    plain call's, permuted, bit for bit; an entry outside the buffer drops its row, leaves the rest
+    as it is and raises the device check."""
+    from paper_2509_02753_b200 import binding as B
+    from paper_2509_02753_b200 import synth
+    wl = synth.Workload("idx", d=256, E=4, I=256, k_base=1, L=1)
+    w = B.make_weights(synth.make_layer(wl, 0, dtype, "cuda"))
+    x = synth.make_tokens(wl, n, dtype, "cuda")
+    cnt = torch.tensor(counts, dtype=torch.int32, device="cuda")
+    g = torch.Generator().manual_seed(n)
+    perm = torch.randperm(n, generator=g).to(torch.int32).cuda()
+    with B.MoEPlan(wl.d, wl.E, wl.I, 1024, 1, dtype) as plan:
+        if sched == "one-cta":
+            plan.set_schedule(B.MOE_SCHED_PREFILL_1CTA)
+        plain = torch.zeros((n, wl.d), dtype=torch.float32, device="cuda")
+        B.moe_experts_forward(plan.handle, x, cnt, w, plain)
+        moved = torch.full((n + 8, wl.d), 7.0, dtype=torch.float32, device="cuda")
+        B.moe_experts_forward(plan.handle, x, cnt, w, moved[:n], out_index=perm)
+        assert plan.device_status() == 0
+        want = torch.empty_like(plain)
+        want[perm.long()] = plain
+        assert torch.equal(moved[:n], want) and bool((moved[n:] == 7.0).all())
+        # one entry points behind the buffer: that row is dropped and reported, the others arrive
+        bad = perm.clone()
+        victim = 123 % n
+        bad[victim] = n + 3
+        again = torch.full((n + 8, wl.d), 7.0, dtype=torch.float32, device="cuda")
+        B.moe_experts_forward(plan.handle, x, cnt, w, again[:n], out_index=bad)
+        assert plan.device_status() == -8            # MOE_ERR_DEVICE_CHECK
+        keep = torch.ones(n, dtype=torch.bool, device="cuda")
+        keep[perm[victim].long()] = False
+        assert torch.equal(again[:n][keep], want[keep])
+        assert bool((again[:n][~keep] == 7.0).all()) and bool((again[n:] == 7.0).all())
+        B.moe_experts_forward(plan.handle, x, cnt, w, moved[:n], out_index=perm)
+        assert plan.device_status() == 0 and torch.equal(moved[:n], want)
