@@ -7,12 +7,13 @@ the expert work.  Rank r holds the experts [r * E / R, (r + 1) * E / R) and the 
 (and shared expert); one layer call on every rank is
 
     pack     route the rank's own tokens (moe_route), gather their rows into expert order
-             (moe_gather_rows): the rows for rank 0 come first, then those for rank 1, ...
+             (moe_gather_rows): the rows for rank 0 come first, then those for rank 1, ...; the
+             shared expert (replicated, no routing) is queued here so that it runs during the exchange
     exchange pairs-per-(destination, expert) counts, then the rows, all-to-all
     compute  regroup what arrived from source-major to expert-major order, run the local experts
              (moe_experts_forward), whose down projection stores the outputs in arrival order
     exchange the fp32 outputs back, all-to-all
-    finish   gated sum over each token's slots plus the shared expert (moe_combine)
+    finish   gated sum over each token's slots plus the shared expert's output (moe_combine)
 
 Every arithmetic step and the receiving side's index tables are kernels of the C library
 (moe_route, moe_gather_rows, moe_regroup_index, moe_experts_forward, moe_combine); this module
@@ -145,7 +146,15 @@ class ExpertParallelLayer:
         send_rows = torch.empty((x.shape[0] * k_l, self.d), dtype=x.dtype, device=x.device)
         B.moe_gather_rows(self.router_plan.handle, x, r["perm"], send_rows, index_div=k_l)   # row of pair p is token p // k_l
         send_counts = r["counts"].reshape(self.world, self.e_loc)
-        ctx = {"x": x, "route": r, "k": k_l}
+        ctx = {"x": x, "route": r, "k": k_l, "o_shared": None}
+        if self.shared_plan is not None:
+            # the shared expert needs no routing and no exchange: queued here, it runs while the host
+            # reads the counts and the rows cross the links
+            T = x.shape[0]
+            o_shared = torch.empty((T, self.d), dtype=torch.float32, device=x.device)
+            one = torch.tensor([T], dtype=torch.int32, device=x.device)
+            B.moe_experts_forward(self.shared_plan.handle, x, one, self.w_shared, o_shared)
+            ctx["o_shared"] = o_shared
         if splits:
             ctx["send_splits"] = [int(v) for v in send_counts.sum(dim=1).tolist()]
         return send_rows, send_counts, ctx
@@ -168,13 +177,8 @@ class ExpertParallelLayer:
     def finish(self, ctx, returned: torch.Tensor) -> torch.Tensor:
         B = self.B
         x, r = ctx["x"], ctx["route"]
-        T = x.shape[0]
         y = torch.empty_like(x)
-        o_shared = None
-        if self.shared_plan is not None:
-            o_shared = torch.empty((T, self.d), dtype=torch.float32, device=x.device)
-            one = torch.tensor([T], dtype=torch.int32, device=x.device)
-            B.moe_experts_forward(self.shared_plan.handle, x, one, self.w_shared, o_shared)
+        o_shared = ctx["o_shared"]
         B.moe_combine(self.router_plan.handle, returned, r["topk_w"], r["inv_perm"], y, o_shared,
                       r["gamma"] if self.shared_gate else None)
         return y
