@@ -493,20 +493,22 @@ __device__ __forceinline__ void finish_block(const Ctx &x, uint32_t j, const flo
 }
 
 // Where warp w's piece of a stream of L chunks starts.  light = 0: Wl equal pieces.  light > 0: the
-// first `light` warps (the routing warps, which join the stream late) have weight 1, the others
-// kStreamerWeight.
-__device__ __forceinline__ uint32_t piece_start(uint32_t w, uint32_t Wl, uint32_t L, uint32_t light) {
+// first `light` warps (the routing warps, which join the stream late) have weight lw (1, or 0 in
+// a stream so short that they had better stay out of it), the others kStreamerWeight (1 where lw is 0).
+__device__ __forceinline__ uint32_t piece_start(uint32_t w, uint32_t Wl, uint32_t L, uint32_t light, uint32_t lw) {
     if (light == 0) return w * L / Wl;
-    const uint32_t cw = w < light ? w : light + (w - light) * kStreamerWeight;
-    const uint32_t W = light + (Wl - light) * kStreamerWeight;
+    const uint32_t sw = lw ? (uint32_t)kStreamerWeight : 1u;
+    const uint32_t cw = w < light ? w * lw : light * lw + (w - light) * sw;
+    const uint32_t W = light * lw + (Wl - light) * sw;
     return (uint32_t)((unsigned long long)cw * L / W);
 }
 // The warp whose piece holds chunk q (inverse of piece_start).
-__device__ __forceinline__ uint32_t piece_owner(uint32_t q, uint32_t Wl, uint32_t L, uint32_t light) {
+__device__ __forceinline__ uint32_t piece_owner(uint32_t q, uint32_t Wl, uint32_t L, uint32_t light, uint32_t lw) {
     if (light == 0) return ((q + 1) * Wl - 1) / L;
-    const uint32_t W = light + (Wl - light) * kStreamerWeight;
+    const uint32_t sw = lw ? (uint32_t)kStreamerWeight : 1u;
+    const uint32_t W = light * lw + (Wl - light) * sw;
     const uint32_t cw = (uint32_t)((((unsigned long long)q + 1) * W - 1) / L);     // largest cumulative weight that starts at or before q
-    return cw < light ? cw : light + (cw - light) / kStreamerWeight;
+    return cw < light * lw ? cw : light + (cw - light * lw) / sw;
 }
 
 // One stream inside a CTA: nblk row blocks of NC chunks each, a flat list the warps cut into
@@ -516,10 +518,14 @@ __device__ __forceinline__ void run_stream(const Ctx &x, int warp, uint32_t nblk
     const uint32_t L = nblk * NC;
     if (L == 0) return;
     const uint32_t Wl = L < (uint32_t)kFusedWarps ? L : (uint32_t)kFusedWarps;
-    if (light >= Wl || L < 4u * Wl) light = 0;
+    uint32_t lw = 1;
+    if (light >= Wl) light = 0;
+    else if (L < 4u * Wl) {               // a short stream: the few routing warps stay out, or (many of them) all share alike
+        if (2u * light <= Wl) lw = 0; else light = 0;
+    }
     if ((uint32_t)warp >= Wl) return;
-    const uint32_t qa = piece_start((uint32_t)warp, Wl, L, light);
-    const uint32_t qb = piece_start((uint32_t)warp + 1, Wl, L, light);
+    const uint32_t qa = piece_start((uint32_t)warp, Wl, L, light, lw);
+    const uint32_t qb = piece_start((uint32_t)warp + 1, Wl, L, light, lw);
     if (qa == qb) return;
     // kStreamBufs chunks per warp are in flight: the loads of chunk q + kStreamBufs - 1 are issued
     // before the MMAs of chunk q
@@ -560,8 +566,8 @@ __device__ __forceinline__ void run_stream(const Ctx &x, int warp, uint32_t nblk
             }
             if (q + 1 == blk_end || q + 1 == qb) {
                 // the warps that share block rb
-                const uint32_t first = piece_owner(rb * NC, Wl, L, light);
-                const uint32_t last = piece_owner((rb + 1) * NC - 1, Wl, L, light);
+                const uint32_t first = piece_owner(rb * NC, Wl, L, light, lw);
+                const uint32_t last = piece_owner((rb + 1) * NC - 1, Wl, L, light, lw);
                 if (first == last) {
                     finish_block<PH>(x, rb, acc);
                 } else {
@@ -575,7 +581,7 @@ __device__ __forceinline__ void run_stream(const Ctx &x, int warp, uint32_t nblk
                     if (is_last) {
                         __threadfence_block();
                         float v[4] = {0.f, 0.f, 0.f, 0.f};
-                        const uint32_t qa_first = piece_start(first, Wl, L, light);
+                        const uint32_t qa_first = piece_start(first, Wl, L, light, lw);
                         for (uint32_t w2 = first; w2 <= last; ++w2) {
                             // a warp after the first starts inside this block: it used its head slot
                             const uint32_t slot2 = 2 * w2 + ((w2 == first && rb != qa_first / NC) ? 1u : 0u);
