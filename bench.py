@@ -325,14 +325,18 @@ def run_ours(args):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    ms, _ = run_case(B, plan, wl, wsets, x, y, k, args.steps, args.warmup, False, barrier, args.min_seconds)
-    blocks = list(run_case.blocks)
-    gpu_launches = run_case.launches
-    # second pass, directly behind the first (same power state), with CUDA events at the stage
-    # boundaries (they switch the programmatic launch chaining off, so the headline above is taken
-    # without them)
-    _, stages = run_case(B, plan, wl, wsets, x, y, k, args.steps, 3, True, barrier, args.min_seconds / 2)
-    clocks = sampler.stop() if rank == 0 else {}
+    clocks = {}
+    try:
+        ms, _ = run_case(B, plan, wl, wsets, x, y, k, args.steps, args.warmup, False, barrier, args.min_seconds)
+        blocks = list(run_case.blocks)
+        gpu_launches = run_case.launches
+        # second pass, directly behind the first (same power state), with CUDA events at the stage
+        # boundaries (they switch the programmatic launch chaining off, so the headline above is taken
+        # without them)
+        _, stages = run_case(B, plan, wl, wsets, x, y, k, args.steps, 3, True, barrier, args.min_seconds / 2)
+    finally:                      # the sampler is a child process: it must not outlive a failed run
+        if rank == 0:
+            clocks = sampler.stop()
     assert plan.device_status() == 0, "device status word set during the timed region"
     ms_best, _ = replicas.aggregate(min(blocks), T * args.steps, dist, device)
     ms, tokens_done = replicas.aggregate(ms, T * args.steps, dist, device)
