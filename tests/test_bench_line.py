@@ -57,3 +57,25 @@ def test_headline_is_the_last_line_and_short(tmp_path):
     # the side file holds every line, the headline included
     kept = [json.loads(l) for l in side.read_text().splitlines() if l.strip()]
     assert kept[-1]["value"] == head["value"] and len(kept) == len(objs)
+
+
+def test_work_model_gives_the_hand_computed_figures():
+    """The roofline numerators, against figures worked out by hand for the Qwen1.5-MoE-shaped layer
+    (d 2048, E 60, I 1408, gated shared expert of 5632): 17.3 MB per routed expert and 69.2 MB for the
+    shared expert in bf16, 138.7 MB for a one-token call that touches four experts; 1.136e12 flop
+    for 8192 tokens at k = 4, of which 7.559e11 in the gate/up GEMM."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    from paper_2509_02753_b200 import synth
+    wl = synth.WORKLOADS["qwen15"]
+    per_expert = 3 * 2048 * 1408 * 2
+    shared = 3 * 2048 * 5632 * 2
+    assert per_expert == 17_301_504 and shared == 69_206_016
+    assert bench.layer_bytes(wl, 1, 4) == 4 * per_expert + shared + (2048 * 60 + 2048) * 2 + 2 * 2048 * 2 == 138_670_080
+    assert bench.layer_flops(wl, 8192, 4) == 8192 * (4 * 6 * 2048 * 1408 + 6 * 2048 * 5632 + 2 * 2048 * 60)
+    assert abs(bench.layer_flops(wl, 8192, 4) / 1.136e12 - 1) < 2e-3
+    assert abs(bench.ffn1_flops(wl, 8192, 4) / 7.559e11 - 1) < 1e-3
+    # phase 1 at 8192 tokens with all 60 experts touched: 738 MB of gate/up weights + activations = 1090 MB
+    assert abs(bench.ffn1_bytes(wl, 8192, 4, 60) / 1.0905e9 - 1) < 2e-3
