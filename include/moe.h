@@ -208,6 +208,29 @@ int moe_route(moe_plan_t *plan, const void *x, const moe_layer_weights_t *w, int
               int32_t *offsets, int32_t *perm, int32_t *inv_perm, void *cuda_stream);
 int moe_gather_rows(moe_plan_t *plan, const void *src, const int32_t *row_index, int32_t index_div,
                     int32_t n_rows, int32_t rows_f32, void *dst, void *cuda_stream);
+/*
+ * moe_send_rows_expert_major: the sending half of expert parallelism as ONE kernel of plain stores
+ * (the paper's Introduction: inter-GPU traffic grows with the number of active experts; the rows
+ * that cross are the T * k_l pairs).  The rows of this rank's pairs, taken in expert order (perm from
+ * moe_route; row p is x[perm[p] / index_div]), are written straight to their place in the OWNER's
+ * arrival buffer, which is laid out expert-major - the owner's local experts ascending, inside an
+ * expert the source ranks ascending, inside a source the pairs in their stable order - so the owner
+ * can call moe_experts_forward on it with counts[e] = sum over sources of all_counts[s][e] and needs
+ * neither an exchange call nor a regrouping copy.  all_counts (device, [world, E] int32, E = this
+ * plan's experts = all experts of the layer, E % world == 0): pairs per (source rank, expert), the
+ * same on every rank (one all-gather of each rank's counts).  peer_rows (HOST array of `world`
+ * device pointers, world <= 16): each rank's arrival buffer, rows of d elements of the plan's dtype,
+ * capacity_rows[r] (HOST array) rows long; entry `rank` is this GPU's own memory, the others memory
+ * of the peers mapped into this process (the stores are ordinary ones).  Rows of this rank's block
+ * of all_counts that do not add up to n_rows send nothing; a destination row >= capacity_rows[r]
+ * is dropped; both raise MOE_ERR_DEVICE_CHECK at the next moe_device_status.  The caller orders the
+ * ranks (a barrier or an event exchange) before the owners read.  Checked on one GPU with every
+ * rank's buffer in its memory; not run across GPUs.
+ * Errors: INVALID_ARG, ALIGN, CUDA.
+ */
+int moe_send_rows_expert_major(moe_plan_t *plan, const void *x, const int32_t *perm, int32_t index_div,
+                               int32_t n_rows, const int32_t *all_counts, int32_t rank, int32_t world,
+                               void *const *peer_rows, const int32_t *capacity_rows, void *cuda_stream);
 int moe_regroup_index(moe_plan_t *plan, const int32_t *recv_counts, int32_t world, int32_t n_rows,
                       int32_t *to_expert_major, int32_t *inverse, int32_t *per_expert, void *cuda_stream);
 int moe_experts_forward(moe_plan_t *plan, const void *x_rows, const int32_t *counts,

@@ -30,7 +30,7 @@ EXPORTS = (
     "moe_status_string", "moe_plan_set_stage_timing", "moe_plan_stage_times",
     "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts", "moe_plan_tile_stats",
     "moe_debug_fused_stamps", "moe_host_pipeline_submit", "moe_host_pipeline_wait",
-    "moe_route", "moe_gather_rows", "moe_regroup_index", "moe_experts_forward", "moe_combine",
+    "moe_route", "moe_gather_rows", "moe_regroup_index", "moe_experts_forward", "moe_combine", "moe_send_rows_expert_major",
     "moe_debug_wait_timeout", "moe_debug_barrier_timeout", "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
@@ -93,6 +93,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_route.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.moe_gather_rows.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
     lib.moe_regroup_index.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    lib.moe_send_rows_expert_major.argtypes = [vp, vp, vp, i32, i32, vp, i32, i32, P(vp), P(i32), vp]
     lib.moe_experts_forward.argtypes = [vp, vp, vp, P(moe_layer_weights_t), i32, vp, vp, vp]
     lib.moe_combine.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
     lib.moe_profile_layer.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, P(ctypes.c_double),
@@ -248,6 +249,21 @@ def moe_regroup_index(plan: int, recv_counts: torch.Tensor, n_rows: int, stream=
     _check("moe_regroup_index", load_library().moe_regroup_index(
         plan, recv_counts.data_ptr(), world, n_rows, to_em.data_ptr(), inv.data_ptr(), per.data_ptr(), _stream(stream)))
     return to_em[:n_rows], inv[:n_rows], per
+
+
+def moe_send_rows_expert_major(plan: int, x: torch.Tensor, perm: torch.Tensor, index_div: int, all_counts: torch.Tensor,
+                               rank: int, peer_rows: Sequence[torch.Tensor], stream=None) -> None:
+    """Writes the rows of this rank's pairs (expert order) to their place in every owner's
+    expert-major arrival buffer; peer_rows[r] is rank r's buffer as seen from this process."""
+    world = len(peer_rows)
+    assert all_counts.dtype == torch.int32 and all_counts.is_cuda and all_counts.is_contiguous() and all_counts.shape[0] == world
+    assert perm.dtype == torch.int32 and perm.is_cuda and x.is_contiguous()
+    caps = (ctypes.c_int32 * world)(*[int(b.shape[0]) for b in peer_rows])
+    assert all(b.is_contiguous() and b.dtype == x.dtype and b.shape[1] == x.shape[1] for b in peer_rows)
+    ptrs = (ctypes.c_void_p * world)(*[b.data_ptr() for b in peer_rows])
+    _check("moe_send_rows_expert_major", load_library().moe_send_rows_expert_major(
+        plan, x.data_ptr(), perm.data_ptr(), index_div, perm.numel(), all_counts.data_ptr(), rank, world, ptrs, caps,
+        _stream(stream)))
 
 
 def moe_experts_forward(plan: int, x_rows: torch.Tensor, counts: torch.Tensor, w: moe_layer_weights_t,

@@ -286,6 +286,74 @@ cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k,
     return e;
 }
 
+// Expert parallelism, sending side, as plain stores into the owners' memory: the rows of this
+// rank's (token, slot) pairs, taken in expert order (perm), are written straight to the place they
+// have in the OWNER's expert-major buffer - local experts ascending, inside an expert the source
+// ranks ascending, inside a source the pairs in their stable order - so that the owner can run its
+// grouped GEMMs on what arrived, with no exchange call and no regrouping copy.  all_counts
+// [world, E]: pairs per (source rank, global expert), the same on every rank.  peers: one base pointer
+// per rank (its arrival buffer: this GPU's own memory for `rank`, peer-mapped memory for the others).
+// Every block redoes the small prefix sums in shared memory.
+struct PeerRows { void *base[kMaxPeers]; int32_t capacity[kMaxPeers]; };   // arrival buffers and their sizes in rows
+
+__global__ void __launch_bounds__(256) send_rows_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ perm,
+                                                        int n_rows, int k, int vec_per_row,
+                                                        const int32_t *__restrict__ all_counts, int E, int rank, int world,
+                                                        PeerRows peers, int32_t *status) {
+    __shared__ int32_t my_off[kMaxExperts + 1];       // this rank's pairs: first packed row of each expert
+    __shared__ int32_t dest_start[kMaxExperts];       // row in the owner's buffer where this rank's rows of expert e begin
+    const int e_loc = E / world;
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int e = 0; e < E; ++e) { my_off[e] = run; run += max(all_counts[rank * E + e], 0); }
+        my_off[E] = run;
+    }
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        const int first = e / e_loc * e_loc;          // the owner's first expert
+        int start = 0;
+        for (int e2 = first; e2 < e; ++e2)
+            for (int sr = 0; sr < world; ++sr) start += max(all_counts[sr * E + e2], 0);
+        for (int sr = 0; sr < rank; ++sr) start += max(all_counts[sr * E + e], 0);
+        dest_start[e] = start;
+    }
+    __syncthreads();
+    if (my_off[E] != n_rows) {                        // the counts do not describe the rows given: nothing is sent
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(status, kStatusBadIndex);
+        return;
+    }
+    const int lane = threadIdx.x & 31;
+    const int warps = gridDim.x * 8;
+    for (int r = blockIdx.x * 8 + (threadIdx.x >> 5); r < n_rows; r += warps) {
+        int lo = 0, hi = E - 1;                       // last expert whose first row is <= r
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (my_off[mid] <= r) lo = mid; else hi = mid - 1;
+        }
+        const int e = lo;
+        const int dst_row = dest_start[e] + (r - my_off[e]);
+        if (dst_row >= peers.capacity[e / e_loc]) {   // the owner's buffer is too small: flagged, row dropped
+            if (lane == 0) atomicOr(status, kStatusBadIndex);
+            continue;
+        }
+        const uint4 *src = x + (size_t)(perm[r] / k) * vec_per_row;
+        uint4 *dst = reinterpret_cast<uint4 *>(peers.base[e / e_loc]) + (size_t)dst_row * vec_per_row;
+        for (int v = lane; v < vec_per_row; v += 32) dst[v] = src[v];
+    }
+}
+
+cudaError_t launch_send_rows(const void *x, const int32_t *perm, int n_rows, int k, int d, int dtype,
+                             const int32_t *all_counts, int E, int rank, int world, void *const *peer_rows,
+                             const int32_t *capacity_rows, int32_t *status, cudaStream_t s, uint64_t *launches) {
+    PeerRows peers{};
+    for (int r = 0; r < world; ++r) { peers.base[r] = peer_rows[r]; peers.capacity[r] = capacity_rows[r]; }
+    const int bytes_per_row = d * (dtype == MOE_BF16 ? 2 : 4);
+    const int grid = n_rows > 0 ? min((n_rows + 7) / 8, 148 * 8) : 1;
+    send_rows_kernel<<<grid, 256, 0, s>>>((const uint4 *)x, perm, n_rows, k, bytes_per_row / 16, all_counts, E, rank, world,
+                                          peers, status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
 // Expert parallelism, receiving side: rows arrive source-major (all rows of source rank 0, then
 // rank 1, ...; inside a source the local experts ascend) and the grouped GEMMs want them
 // expert-major (inside an expert the sources in rank order).  recv_counts [world, E] = rows per

@@ -187,6 +187,11 @@ cudaError_t fused_prepare(int d);    // opts the kernel in to its shared-memory 
 cudaError_t launch_decode_stack(const StackArgs &a, int sm_count, cudaStream_t s, uint64_t *launches);
 cudaError_t launch_barrier_probe(const uint32_t *bar, int32_t *status, unsigned long long limit_ns, cudaStream_t s);
 
+constexpr int kMaxPeers = 16;        // ranks an expert-parallel group may have (pointers travel as kernel parameters)
+cudaError_t launch_send_rows(const void *x, const int32_t *perm, int n_rows, int k, int d, int dtype,
+                             const int32_t *all_counts, int E, int rank, int world, void *const *peer_rows,
+                             const int32_t *capacity_rows, int32_t *status, cudaStream_t s, uint64_t *launches);
+
 cudaError_t launch_widen(const void *src, float *dst, size_t n, int dtype, cudaStream_t s,
                          uint64_t *launches);
 

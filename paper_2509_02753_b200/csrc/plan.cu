@@ -643,6 +643,26 @@ int moe_gather_rows(moe_plan_t *p, const void *src, const int32_t *row_index, in
     return MOE_OK;
 }
 
+int moe_send_rows_expert_major(moe_plan_t *p, const void *x, const int32_t *perm, int32_t index_div, int32_t n_rows,
+                               const int32_t *all_counts, int32_t rank, int32_t world, void *const *peer_rows,
+                               const int32_t *capacity_rows, void *cuda_stream) {
+    if (!p || !x || !perm || !all_counts || !peer_rows || !capacity_rows) return MOE_ERR_INVALID_ARG;
+    const moe_config_t &c = p->cfg;
+    if (world < 1 || world > kMaxPeers || rank < 0 || rank >= world || c.E % world != 0) return MOE_ERR_INVALID_ARG;
+    if (index_div < 1 || n_rows < 0) return MOE_ERR_INVALID_ARG;
+    if (!aligned16(x)) return MOE_ERR_ALIGN;
+    for (int r = 0; r < world; ++r) {
+        if (!peer_rows[r] || capacity_rows[r] < 0) return MOE_ERR_INVALID_ARG;
+        if (!aligned16(peer_rows[r])) return MOE_ERR_ALIGN;
+    }
+    if (launch_send_rows(x, perm, n_rows, index_div, c.d, c.dtype, all_counts, c.E, rank, world, peer_rows, capacity_rows,
+                         p->ws.status, (cudaStream_t)cuda_stream, &p->launches) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    return MOE_OK;
+}
+
 int moe_regroup_index(moe_plan_t *p, const int32_t *recv_counts, int32_t world, int32_t n_rows, int32_t *to_expert_major,
                       int32_t *inverse, int32_t *per_expert, void *cuda_stream) {
     if (!p || !recv_counts || !to_expert_major || !inverse || !per_expert) return MOE_ERR_INVALID_ARG;

@@ -322,3 +322,66 @@ def test_experts_forward_stores_rows_where_the_index_says(dtype, n, counts, sche
         assert bool((again[:n][~keep] == 7.0).all()) and bool((again[n:] == 7.0).all())
         B.moe_experts_forward(plan.handle, x, cnt, w, moved[:n], out_index=perm)
         assert plan.device_status() == 0 and torch.equal(moved[:n], want)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("world,dtype", [(2, torch.bfloat16), (4, torch.bfloat16), (4, torch.float32)])
+def test_rows_stored_straight_into_the_owners_buffers_arrive_expert_major(world, dtype):
+    """moe_send_rows_expert_major, with every rank's arrival buffer in this GPU's memory (the
+    pointers would be peer mappings on several GPUs): after every rank has sent, each buffer holds
+    byte for byte what the exchange by slicing followed by the regrouping copy produces, the rows
+    behind it are untouched, and a buffer that is too small or counts that do not match the rows
+    are reported, not overrun."""
+    from paper_2509_02753_b200 import binding as B
+    from paper_2509_02753_b200 import synth
+    wl = synth.Workload("send", d=256, E=16, I=256, k_base=4, L=1, router_bias_std=0.6, w_std=0.02)
+    k, renorm = 3, False
+    Ts = [37, 300, 5, 129][:world]
+    w = synth.make_layer(wl, 0, dtype, "cuda")
+    xs = [synth.make_tokens(wl, T, dtype, "cuda", seed=20 + r) for r, T in enumerate(Ts)]
+    ranks = [ep.ExpertParallelLayer(wl.d, wl.E, wl.I, max(Ts), 4, dtype, w, r, world) for r in range(world)]
+    e_loc = wl.E // world
+    try:
+        packed = [rk.pack(x, k, renorm) for rk, x in zip(ranks, xs)]
+        all_counts = torch.stack([p[2]["route"]["counts"] for p in packed]).contiguous()        # [world, E]
+        host = all_counts.cpu()
+        n_recv = [int(host[:, r * e_loc:(r + 1) * e_loc].sum()) for r in range(world)]
+        bufs = [torch.full((n + 4, wl.d), 7.0, dtype=dtype, device="cuda") for n in n_recv]
+        for s, (rk, x) in enumerate(zip(ranks, xs)):
+            B.moe_send_rows_expert_major(rk.router_plan.handle, x, packed[s][2]["route"]["perm"], k, all_counts, s, bufs)
+            assert rk.router_plan.device_status() == 0
+        torch.cuda.synchronize()
+        for r in range(world):
+            blocks, cnts = [], []
+            for s in range(world):
+                rows_s, counts_s, ctx_s = packed[s]
+                off = sum(ctx_s["send_splits"][:r])
+                blocks.append(rows_s[off:off + ctx_s["send_splits"][r]])
+                cnts.append(counts_s[r])
+            arrived = torch.cat(blocks)                                     # source-major, as an all-to-all delivers
+            to_em, _, per_expert = ep.regroup_index(torch.stack(cnts))
+            want = arrived[to_em.long()]
+            assert torch.equal(bufs[r][:n_recv[r]], want)
+            assert bool((bufs[r][n_recv[r]:] == 7.0).all())
+            assert per_expert.tolist() == host[:, r * e_loc:(r + 1) * e_loc].sum(dim=0).tolist()
+        # an arrival buffer one row short: the row that does not fit is dropped and reported
+        r_big = max(range(world), key=lambda r: n_recv[r])
+        short = [b if r != r_big else torch.full((n_recv[r] - 1, wl.d), 7.0, dtype=dtype, device="cuda")
+                 for r, b in enumerate(bufs)]
+        keep = torch.full((n_recv[r_big] + 4, wl.d), 7.0, dtype=dtype, device="cuda")
+        short_views = [b if r != r_big else keep[:n_recv[r] - 1] for r, b in enumerate(short)]
+        for s, (rk, x) in enumerate(zip(ranks, xs)):
+            B.moe_send_rows_expert_major(rk.router_plan.handle, x, packed[s][2]["route"]["perm"], k, all_counts, s, short_views)
+        statuses = [rk.router_plan.device_status() for rk in ranks]
+        assert -8 in statuses                                               # MOE_ERR_DEVICE_CHECK from the rank whose row fell off
+        assert bool((keep[n_recv[r_big] - 1:] == 7.0).all())
+        # counts that do not describe the rows given: nothing is written
+        wrong = all_counts.clone()
+        wrong[0, 0] += 1
+        fresh = [torch.full((n + 4, wl.d), 7.0, dtype=dtype, device="cuda") for n in n_recv]
+        B.moe_send_rows_expert_major(ranks[0].router_plan.handle, xs[0], packed[0][2]["route"]["perm"], k, wrong, 0, fresh)
+        assert ranks[0].router_plan.device_status() == -8
+        assert all(bool((b == 7.0).all()) for b in fresh)
+    finally:
+        for rk in ranks:
+            rk.close()
