@@ -231,6 +231,20 @@ int moe_gather_rows(moe_plan_t *plan, const void *src, const int32_t *row_index,
 int moe_send_rows_expert_major(moe_plan_t *plan, const void *x, const int32_t *perm, int32_t index_div,
                                int32_t n_rows, const int32_t *all_counts, int32_t rank, int32_t world,
                                void *const *peer_rows, const int32_t *capacity_rows, void *cuda_stream);
+/*
+ * moe_return_rows_to_sources: the way back, likewise as plain stores.  o_rows (fp32, [n_rows, d]) are
+ * this rank's expert outputs in the expert-major order of its arrival buffer (what
+ * moe_experts_forward wrote for the rows moe_send_rows_expert_major delivered); each row goes to
+ * the place its pair has in the SOURCE rank's expert order, so that the source calls moe_combine
+ * on its buffer with the inv_perm of its own moe_route.  `plan` has all E experts of the layer (the
+ * router's plan), all_counts / rank / world / peer_rows (fp32 buffers of capacity_rows[r] rows, one per
+ * source rank) as in moe_send_rows_expert_major; counts of this owner's experts that do not add up to
+ * n_rows return nothing, rows that would fall behind a buffer are dropped, both reported as
+ * MOE_ERR_DEVICE_CHECK.  Checked on one GPU; not run across GPUs.  Errors: INVALID_ARG, ALIGN, CUDA.
+ */
+int moe_return_rows_to_sources(moe_plan_t *plan, const float *o_rows, int32_t n_rows, const int32_t *all_counts,
+                               int32_t rank, int32_t world, void *const *peer_rows, const int32_t *capacity_rows,
+                               void *cuda_stream);
 int moe_regroup_index(moe_plan_t *plan, const int32_t *recv_counts, int32_t world, int32_t n_rows,
                       int32_t *to_expert_major, int32_t *inverse, int32_t *per_expert, void *cuda_stream);
 int moe_experts_forward(moe_plan_t *plan, const void *x_rows, const int32_t *counts,

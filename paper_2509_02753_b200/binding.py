@@ -31,6 +31,7 @@ EXPORTS = (
     "moe_last_residual_f32", "moe_dispatch_tables_static", "moe_plan_touched_experts", "moe_plan_tile_stats",
     "moe_debug_fused_stamps", "moe_host_pipeline_submit", "moe_host_pipeline_wait",
     "moe_route", "moe_gather_rows", "moe_regroup_index", "moe_experts_forward", "moe_combine", "moe_send_rows_expert_major",
+    "moe_return_rows_to_sources",
     "moe_debug_wait_timeout", "moe_debug_barrier_timeout", "moe_profile_layer", "moe_lexi_allocate_exact", "moe_lexi_allocate_evolutionary",
 )
 STAGE_NAMES = ("router", "dispatch", "ffn1", "ffn2", "combine")
@@ -94,6 +95,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_gather_rows.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
     lib.moe_regroup_index.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
     lib.moe_send_rows_expert_major.argtypes = [vp, vp, vp, i32, i32, vp, i32, i32, P(vp), P(i32), vp]
+    lib.moe_return_rows_to_sources.argtypes = [vp, vp, i32, vp, i32, i32, P(vp), P(i32), vp]
     lib.moe_experts_forward.argtypes = [vp, vp, vp, P(moe_layer_weights_t), i32, vp, vp, vp]
     lib.moe_combine.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]
     lib.moe_profile_layer.argtypes = [vp, vp, P(moe_layer_weights_t), i32, i32, i32, P(ctypes.c_double),
@@ -264,6 +266,20 @@ def moe_send_rows_expert_major(plan: int, x: torch.Tensor, perm: torch.Tensor, i
     _check("moe_send_rows_expert_major", load_library().moe_send_rows_expert_major(
         plan, x.data_ptr(), perm.data_ptr(), index_div, perm.numel(), all_counts.data_ptr(), rank, world, ptrs, caps,
         _stream(stream)))
+
+
+def moe_return_rows_to_sources(plan: int, o_rows: torch.Tensor, all_counts: torch.Tensor, rank: int,
+                               peer_rows: Sequence[torch.Tensor], stream=None) -> None:
+    """Writes this owner's expert outputs (fp32, expert-major arrival order) to the row each pair has in
+    its source rank's expert order; peer_rows[s] is source s's fp32 buffer as seen from this process."""
+    world = len(peer_rows)
+    assert o_rows.dtype == torch.float32 and o_rows.is_cuda and o_rows.is_contiguous()
+    assert all_counts.dtype == torch.int32 and all_counts.is_contiguous() and all_counts.shape[0] == world
+    assert all(b.is_contiguous() and b.dtype == torch.float32 and b.shape[1] == o_rows.shape[1] for b in peer_rows)
+    ptrs = (ctypes.c_void_p * world)(*[b.data_ptr() for b in peer_rows])
+    caps = (ctypes.c_int32 * world)(*[int(b.shape[0]) for b in peer_rows])
+    _check("moe_return_rows_to_sources", load_library().moe_return_rows_to_sources(
+        plan, o_rows.data_ptr(), o_rows.shape[0], all_counts.data_ptr(), rank, world, ptrs, caps, _stream(stream)))
 
 
 def moe_experts_forward(plan: int, x_rows: torch.Tensor, counts: torch.Tensor, w: moe_layer_weights_t,

@@ -294,6 +294,7 @@ cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k,
 // [world, E]: pairs per (source rank, global expert), the same on every rank.  peers: one base pointer
 // per rank (its arrival buffer: this GPU's own memory for `rank`, peer-mapped memory for the others).
 // Every block redoes the small prefix sums in shared memory.
+constexpr int kMaxRegroupBlocks = 1024;      // (local expert, source rank) blocks an expert-parallel rank may have
 struct PeerRows { void *base[kMaxPeers]; int32_t capacity[kMaxPeers]; };   // arrival buffers and their sizes in rows
 
 __global__ void __launch_bounds__(256) send_rows_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ perm,
@@ -354,13 +355,73 @@ cudaError_t launch_send_rows(const void *x, const int32_t *perm, int n_rows, int
     return cudaGetLastError();
 }
 
+// Expert parallelism, the way back, as plain stores: the owner's fp32 outputs, in the expert-major
+// order of its arrival buffer, go straight to the row each pair has in its SOURCE rank's packed
+// (expert) order, which is the order that rank's moe_combine indexes with inv_perm.  Block (local
+// expert e, source s) of the owner's rows starts at blk_start[e * world + s] and belongs at row
+// src_off = sum of all_counts[s][0 .. global e) of source s's buffer.
+__global__ void __launch_bounds__(256) return_rows_kernel(const uint4 *__restrict__ o_rows, int n_rows, int vec_per_row,
+                                                          const int32_t *__restrict__ all_counts, int E, int rank, int world,
+                                                          PeerRows peers, int32_t *status) {
+    __shared__ int32_t blk_start[kMaxRegroupBlocks + 1], src_off[kMaxRegroupBlocks];
+    const int e_loc = E / world, nb = e_loc * world;
+    for (int b = threadIdx.x; b < nb; b += blockDim.x) {      // b = local expert * world + source
+        const int el = b / world, sr = b - el * world, e = rank * e_loc + el;
+        int off = 0;
+        for (int e2 = 0; e2 < e; ++e2) off += max(all_counts[sr * E + e2], 0);
+        src_off[b] = off;
+    }
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int b = 0; b < nb; ++b) {
+            const int el = b / world, sr = b - el * world;
+            blk_start[b] = run;
+            run += max(all_counts[sr * E + rank * e_loc + el], 0);
+        }
+        blk_start[nb] = run;
+    }
+    __syncthreads();
+    if (blk_start[nb] != n_rows) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(status, kStatusBadIndex);
+        return;
+    }
+    const int lane = threadIdx.x & 31;
+    const int warps = gridDim.x * 8;
+    for (int r = blockIdx.x * 8 + (threadIdx.x >> 5); r < n_rows; r += warps) {
+        int lo = 0, hi = nb - 1;                              // last block that starts at or before r
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (blk_start[mid] <= r) lo = mid; else hi = mid - 1;
+        }
+        const int sr = lo % world;
+        const int dst_row = src_off[lo] + (r - blk_start[lo]);
+        if (dst_row >= peers.capacity[sr]) {
+            if (lane == 0) atomicOr(status, kStatusBadIndex);
+            continue;
+        }
+        const uint4 *src = o_rows + (size_t)r * vec_per_row;
+        uint4 *dst = reinterpret_cast<uint4 *>(peers.base[sr]) + (size_t)dst_row * vec_per_row;
+        for (int v = lane; v < vec_per_row; v += 32) dst[v] = src[v];
+    }
+}
+
+cudaError_t launch_return_rows(const float *o_rows, int n_rows, int d, const int32_t *all_counts, int E, int rank, int world,
+                               void *const *peer_rows, const int32_t *capacity_rows, int32_t *status, cudaStream_t s,
+                               uint64_t *launches) {
+    PeerRows peers{};
+    for (int r = 0; r < world; ++r) { peers.base[r] = peer_rows[r]; peers.capacity[r] = capacity_rows[r]; }
+    const int grid = n_rows > 0 ? min((n_rows + 7) / 8, 148 * 8) : 1;
+    return_rows_kernel<<<grid, 256, 0, s>>>((const uint4 *)o_rows, n_rows, d * 4 / 16, all_counts, E, rank, world, peers, status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
 // Expert parallelism, receiving side: rows arrive source-major (all rows of source rank 0, then
 // rank 1, ...; inside a source the local experts ascend) and the grouped GEMMs want them
 // expert-major (inside an expert the sources in rank order).  recv_counts [world, E] = rows per
 // (source, local expert).  to_em[p] = arrival index of the row at expert-major position p, inv its
 // inverse, per_expert[e] = rows of local expert e.  Every CTA redoes the two small scans over the
 // world x E blocks in shared memory and then copies index ranges of its share of the blocks.
-constexpr int kMaxRegroupBlocks = 1024;
 __global__ void __launch_bounds__(256) regroup_index_kernel(const int32_t *__restrict__ recv_counts, int world, int E,
                                                             int n_rows, int32_t *to_em, int32_t *inv,
                                                             int32_t *per_expert, int32_t *status) {

@@ -191,6 +191,9 @@ constexpr int kMaxPeers = 16;        // ranks an expert-parallel group may have 
 cudaError_t launch_send_rows(const void *x, const int32_t *perm, int n_rows, int k, int d, int dtype,
                              const int32_t *all_counts, int E, int rank, int world, void *const *peer_rows,
                              const int32_t *capacity_rows, int32_t *status, cudaStream_t s, uint64_t *launches);
+cudaError_t launch_return_rows(const float *o_rows, int n_rows, int d, const int32_t *all_counts, int E, int rank, int world,
+                               void *const *peer_rows, const int32_t *capacity_rows, int32_t *status, cudaStream_t s,
+                               uint64_t *launches);
 
 cudaError_t launch_widen(const void *src, float *dst, size_t n, int dtype, cudaStream_t s,
                          uint64_t *launches);

@@ -663,6 +663,27 @@ int moe_send_rows_expert_major(moe_plan_t *p, const void *x, const int32_t *perm
     return MOE_OK;
 }
 
+int moe_return_rows_to_sources(moe_plan_t *p, const float *o_rows, int32_t n_rows, const int32_t *all_counts, int32_t rank,
+                               int32_t world, void *const *peer_rows, const int32_t *capacity_rows, void *cuda_stream) {
+    if (p && n_rows == 0) return MOE_OK;
+    if (!p || !o_rows || !all_counts || !peer_rows || !capacity_rows) return MOE_ERR_INVALID_ARG;
+    const moe_config_t &c = p->cfg;
+    if (world < 1 || world > kMaxPeers || rank < 0 || rank >= world || c.E % world != 0 || n_rows < 0 ||
+        c.E / world * world > 1024)
+        return MOE_ERR_INVALID_ARG;
+    if (!aligned16(o_rows) || c.d % 4 != 0) return MOE_ERR_ALIGN;
+    for (int r = 0; r < world; ++r) {
+        if (!peer_rows[r] || capacity_rows[r] < 0) return MOE_ERR_INVALID_ARG;
+        if (!aligned16(peer_rows[r])) return MOE_ERR_ALIGN;
+    }
+    if (launch_return_rows(o_rows, n_rows, c.d, all_counts, c.E, rank, world, peer_rows, capacity_rows, p->ws.status,
+                           (cudaStream_t)cuda_stream, &p->launches) != cudaSuccess) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+    }
+    return MOE_OK;
+}
+
 int moe_regroup_index(moe_plan_t *p, const int32_t *recv_counts, int32_t world, int32_t n_rows, int32_t *to_expert_major,
                       int32_t *inverse, int32_t *per_expert, void *cuda_stream) {
     if (!p || !recv_counts || !to_expert_major || !inverse || !per_expert) return MOE_ERR_INVALID_ARG;

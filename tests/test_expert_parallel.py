@@ -385,3 +385,91 @@ def test_rows_stored_straight_into_the_owners_buffers_arrive_expert_major(world,
     finally:
         for rk in ranks:
             rk.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("world,dtype", [(2, torch.bfloat16), (4, torch.bfloat16), (4, torch.float32)])
+def test_whole_layer_with_plain_stores_both_ways_equals_the_exchange_path(world, dtype):
+    """The expert-parallel layer with moe_send_rows_expert_major on the way out and
+    moe_return_rows_to_sources on the way back (every rank's buffers in this GPU's memory) gives, bit
+    for bit, what the path through the exchange by slicing and the regrouping copies gives, and both
+    agree with the one-GPU layer."""
+    from paper_2509_02753_b200 import binding as B
+    from paper_2509_02753_b200 import synth
+    from parity import rel_err
+    wl = synth.Workload("both", d=256, E=16, I=256, k_base=4, L=1, I_shared=128, shared_gate=True,
+                        router_bias_std=0.4, w_std=0.02)
+    k, renorm, scale = 3, False, 1.25
+    Ts = [37, 300, 5, 129][:world]
+    w = synth.make_layer(wl, 0, dtype, "cuda")
+    xs = [synth.make_tokens(wl, T, dtype, "cuda", seed=30 + r) for r, T in enumerate(Ts)]
+    ranks = [ep.ExpertParallelLayer(wl.d, wl.E, wl.I, max(Ts), 4, dtype, w, r, world, I_shared=wl.I_shared,
+                                    shared_gate=True, routed_scale=scale) for r in range(world)]
+    e_loc = wl.E // world
+    try:
+        packed = [rk.pack(x, k, renorm) for rk, x in zip(ranks, xs)]
+        # ---- the exchange path (slicing stands in for the all-to-all)
+        recv_rows, recv_counts = [], []
+        for r in range(world):
+            blocks, cnts = [], []
+            for s in range(world):
+                rows_s, counts_s, ctx_s = packed[s]
+                off = sum(ctx_s["send_splits"][:r])
+                blocks.append(rows_s[off:off + ctx_s["send_splits"][r]])
+                cnts.append(counts_s[r])
+            recv_rows.append(torch.cat(blocks))
+            recv_counts.append(torch.stack(cnts))
+        backs = [rk.compute(rr, rc) for rk, rr, rc in zip(ranks, recv_rows, recv_counts)]
+        y_exchange = []
+        for s in range(world):
+            parts = []
+            for r in range(world):
+                splits_r = [int(v) for v in recv_counts[r].sum(dim=1).tolist()]
+                off = sum(splits_r[:s])
+                parts.append(backs[r][off:off + splits_r[s]])
+            y_exchange.append(ranks[s].finish(packed[s][2], torch.cat(parts)))
+        # ---- the same layer with plain stores both ways
+        all_counts = torch.stack([p[2]["route"]["counts"] for p in packed]).contiguous()
+        host = all_counts.cpu()
+        n_recv = [int(host[:, r * e_loc:(r + 1) * e_loc].sum()) for r in range(world)]
+        arrival = [torch.zeros((max(n, 1), wl.d), dtype=dtype, device="cuda") for n in n_recv]
+        for s, (rk, x) in enumerate(zip(ranks, xs)):
+            B.moe_send_rows_expert_major(rk.router_plan.handle, x, packed[s][2]["route"]["perm"], k, all_counts, s, arrival)
+        returned = [torch.full((T * k, wl.d), float("nan"), dtype=torch.float32, device="cuda") for T in Ts]
+        for r, rk in enumerate(ranks):
+            per_expert = all_counts[:, r * e_loc:(r + 1) * e_loc].sum(dim=0).to(torch.int32).contiguous()
+            out_em = torch.zeros((n_recv[r], wl.d), dtype=torch.float32, device="cuda")
+            if n_recv[r] > 0:
+                B.moe_experts_forward(rk.local_plan.handle, arrival[r][:n_recv[r]], per_expert, rk.w_local, out_em)
+                B.moe_return_rows_to_sources(rk.router_plan.handle, out_em, all_counts, r, returned)
+        y_stores = [ranks[s].finish(packed[s][2], returned[s]) for s in range(world)]
+        torch.cuda.synchronize()
+        with B.MoEPlan(wl.d, wl.E, wl.I, max(Ts), 4, dtype, I_shared=wl.I_shared, shared_gate=True,
+                       routed_scale=scale) as plan:
+            ws = B.make_weights(w)
+            for x, ya, yb in zip(xs, y_exchange, y_stores):
+                assert torch.equal(ya, yb)
+                one = plan.layer_forward(x, ws, k, renorm)
+                assert rel_err(yb.float().cpu().numpy(), one.double().cpu().numpy()) <= (4e-2 if dtype == torch.bfloat16 else 1e-4)
+        for rk in ranks:
+            assert rk.router_plan.device_status() == 0 and rk.local_plan.device_status() == 0
+        # a source buffer that is one row short, and counts that do not describe the owner's rows
+        r0 = max(range(world), key=lambda r: n_recv[r])
+        per_expert = all_counts[:, r0 * e_loc:(r0 + 1) * e_loc].sum(dim=0).to(torch.int32).contiguous()
+        out_em = torch.ones((n_recv[r0], wl.d), dtype=torch.float32, device="cuda")
+        s_short = max(range(world), key=lambda s: int(host[s, r0 * e_loc:(r0 + 1) * e_loc].sum()))
+        last_needed = int(host[s_short, :(r0 + 1) * e_loc].sum())           # one behind the last row owner r0 writes there
+        room = [torch.full((T * k + 2, wl.d), 7.0, dtype=torch.float32, device="cuda") for T in Ts]
+        views = [b[:Ts[s] * k] if s != s_short else b[:last_needed - 1] for s, b in enumerate(room)]
+        B.moe_return_rows_to_sources(ranks[r0].router_plan.handle, out_em, all_counts, r0, views)
+        assert ranks[r0].router_plan.device_status() == -8
+        assert bool((room[s_short][last_needed - 1:] == 7.0).all())
+        wrong = all_counts.clone()
+        wrong[0, r0 * e_loc] += 1
+        fresh = [torch.full((T * k, wl.d), 7.0, dtype=torch.float32, device="cuda") for T in Ts]
+        B.moe_return_rows_to_sources(ranks[r0].router_plan.handle, out_em, wrong, r0, fresh)
+        assert ranks[r0].router_plan.device_status() == -8
+        assert all(bool((b == 7.0).all()) for b in fresh)
+    finally:
+        for rk in ranks:
+            rk.close()
