@@ -222,6 +222,169 @@ __global__ void __launch_bounds__(1024) dispatch_block_kernel(DispatchArgs a, in
     }
 }
 
+// Cluster variant: the three passes in ONE launch for calls of any size the layer path sees.  A
+// cluster of 8 CTAs shares the pairs (CTA c the c-th eighth, warp w of it a contiguous run), the
+// per-CTA totals meet through distributed shared memory, and every CTA then knows where its first
+// row of each expert lies: expert-major, inside an expert CTA by CTA, warp by warp, pair by pair -
+// the same stable order as the other forms.  Ranks are ballot ranks (no atomics).  The loops are
+// kept rolled: a kernel this short mostly runs instructions it fetches for the first time.
+// When asked, the eight CTAs also build an eighth each of the tile lists of the tensor-core GEMMs.
+constexpr int kDispatchClusterCtas = 8;
+
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+
+__global__ void __launch_bounds__(1024) dispatch_cluster_kernel(DispatchArgs a, int n_pairs, TileBuildArgs tb, int build) {
+    __shared__ int32_t hist[32][kMaxExperts];
+    __shared__ int32_t tot_s[kMaxExperts];                       // this CTA's pairs per expert (read by the other CTAs)
+    __shared__ int32_t first_s[kMaxExperts];                     // pairs of an expert in the CTAs before this one
+    __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1];
+    __shared__ TileBuildSmem tb_sm;
+    pdl_trigger();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int n_warps = kDispatchClusterCtas * 32;
+    const int per_warp = (((n_pairs + n_warps - 1) / n_warps) + 31) / 32 * 32;
+    const int gw = (int)rank * 32 + warp;
+    const int p0 = (int)min((long long)gw * per_warp, (long long)n_pairs), p1 = min(p0 + per_warp, n_pairs);
+    for (int e = lane; e < kMaxExperts; e += 32) hist[warp][e] = 0;
+    __syncwarp();
+    pdl_wait();
+    // pass 1: histogram of the warp's run; pairs of one expert inside a step are counted by their leader
+    for (int base = p0; base < p1; base += 128) {
+        int ev[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int p = base + u * 32 + lane;
+            ev[u] = p < p1 ? a.topk_idx[p] : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            int e = ev[u];
+            if (e != -1 && (unsigned)e >= (unsigned)a.E) { atomicOr(a.status, kStatusBadIndex); e = -1; }
+            const unsigned peers = __match_any_sync(0xffffffffu, e);
+            if (e >= 0 && lane == __ffs(peers) - 1) hist[warp][e] += __popc(peers);
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < kMaxExperts) {
+        const int e = threadIdx.x;
+        int run = 0;
+#pragma unroll 8
+        for (int w = 0; w < 32; ++w) {
+            const int c = hist[w][e];
+            hist[w][e] = run;
+            run += c;
+        }
+        tot_s[e] = run;
+    }
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    if (threadIdx.x < kMaxExperts) {
+        const int e = threadIdx.x;
+        const uint32_t mine = (uint32_t)__cvta_generic_to_shared(&tot_s[e]);
+        int total = 0, before = 0;
+#pragma unroll
+        for (int c = 0; c < kDispatchClusterCtas; ++c) {
+            uint32_t remote;
+            int v;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(mine), "r"(c));
+            asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
+            total += v;
+            before += c < (int)rank ? v : 0;
+        }
+        cnt_s[e] = e < a.E ? total : 0;
+        first_s[e] = before;
+    }
+    cluster_arrive_release();      // this CTA has read the others' totals; waited for before it exits
+    __syncthreads();
+    if (warp == 0) {
+        int c[kExpertsPerLane], sum = 0;
+#pragma unroll
+        for (int j = 0; j < kExpertsPerLane; ++j) {
+            const int e = lane * kExpertsPerLane + j;
+            c[j] = e < a.E ? cnt_s[e] : 0;
+            sum += c[j];
+        }
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        int run = incl - sum;
+#pragma unroll
+        for (int j = 0; j < kExpertsPerLane; ++j) {
+            const int e = lane * kExpertsPerLane + j;
+            if (e < a.E) {
+                off_s[e] = run;
+                if (rank == 0) { a.counts[e] = c[j]; a.offsets[e] = run; }
+            }
+            run += c[j];
+        }
+        if (lane == 31) {
+            off_s[a.E] = incl;
+            if (rank == 0) a.offsets[a.E] = incl;
+        }
+    }
+    __syncthreads();
+    // pass 2: ranked placement; off_s[e] + first_s[e] + hist[warp][e] is the warp's cursor for expert e
+    for (int base = p0; base < p1; base += 128) {
+        int ev[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int p = base + u * 32 + lane;
+            ev[u] = p < p1 ? a.topk_idx[p] : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int p = base + u * 32 + lane;
+            int e = ev[u];
+            if ((unsigned)e >= (unsigned)a.E) e = -1;
+            const unsigned peers = __match_any_sync(0xffffffffu, e);
+            const int leader = __ffs(peers) - 1;
+            int first = 0;
+            if (e >= 0 && lane == leader) {
+                first = hist[warp][e];
+                hist[warp][e] = first + __popc(peers);
+                first += off_s[e] + first_s[e];
+            }
+            first = __shfl_sync(0xffffffffu, first, leader);
+            if (e >= 0) {
+                const int r = first + __popc(peers & ((1u << lane) - 1u));
+                a.perm[r] = p;
+                a.inv_perm[p] = r;
+            }
+            __syncwarp();
+        }
+    }
+    if (build) {
+        __syncthreads();
+        build_tiles_block(tb, cnt_s, off_s, tb_sm, (int)rank, kDispatchClusterCtas);
+    }
+    cluster_wait_acquire();
+}
+
+cudaError_t launch_dispatch_cluster(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained,
+                                    const TileBuildArgs *tiles) {
+    const int n_pairs = a.T * a.k;
+    if (n_pairs <= 0) return cudaSuccess;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(kDispatchClusterCtas); cfg.blockDim = dim3(1024); cfg.dynamicSmemBytes = 0; cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kDispatchClusterCtas; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = chained ? 2 : 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, dispatch_cluster_kernel, a, n_pairs,
+                                             tiles ? *tiles : TileBuildArgs{}, tiles ? 1 : 0);
+    ++*launches;
+    return e;
+}
+
 cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained,
                             const TileBuildArgs *tiles) {
     const int n_pairs = a.T * a.k;

@@ -115,6 +115,13 @@ struct DispatchArgs {
 cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained = false,
                             const TileBuildArgs *tiles = nullptr);
 constexpr int kBlockDispatchPairs = 8192;
+// The same tables from one launch of a cluster of 8 CTAs, whatever the size of the call; with tiles
+// != NULL the cluster also builds the tensor-core tile lists.
+cudaError_t launch_dispatch_cluster(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained,
+                                    const TileBuildArgs *tiles);
+// Calls of more tokens than this take the tensor-core router (one CTA per 64 tokens, about as long
+// for 100 tokens as for 9000); up to it one block per token is as fast.
+constexpr int kTcRouterMinTokens = 128;
 cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k, int d, int dtype,
                           void *x_perm, cudaStream_t s, uint64_t *launches, bool chained = false,
                           const TileBuildArgs *tiles = nullptr);   // tiles: also build the tile lists

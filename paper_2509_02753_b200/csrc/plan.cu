@@ -230,7 +230,7 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
         if ((err = launch_decode_front(fr, s, &p->launches)) != cudaSuccess) return MOE_ERR_CUDA;
         mark(1);
     } else {
-        if (T > 512 && p->use_tc_router && tc_router_supported(&p->tc, ra))
+        if (T > kTcRouterMinTokens && p->use_tc_router && tc_router_supported(&p->tc, ra))
             err = launch_router_tc(&p->tc, ra, p->sm_count, s, &p->launches);
         else
             err = launch_router(ra, s, &p->launches);
@@ -238,15 +238,15 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
         mark(1);
         DispatchArgs da{ws.topk_idx, T, k, c.E, ws.counts, ws.offsets, ws.perm, ws.inv_perm,
                         ws.part_hist, ws.status};
-        const bool fuse_tiles = sched != MOE_SCHED_SIMT && T * k <= kBlockDispatchPairs;
-        if ((err = launch_dispatch(da, s, &p->launches, chained, fuse_tiles ? &sc.tb : nullptr)) != cudaSuccess)
+        // one launch of a cluster of 8 CTAs builds the tables and, for the tensor-core schedules,
+        // the tile lists; the gather of the token rows follows
+        const bool with_tiles = sched != MOE_SCHED_SIMT;
+        if ((err = launch_dispatch_cluster(da, s, &p->launches, chained, with_tiles ? &sc.tb : nullptr)) != cudaSuccess)
             return MOE_ERR_CUDA;
-        // larger calls: the tile lists are built by a few extra blocks of the gather launch
-        const bool tiles_in_gather = sched != MOE_SCHED_SIMT && !fuse_tiles;
         if ((err = launch_gather(x, ws.perm, T * k, k, c.d, c.dtype, ws.x_perm, s, &p->launches, chained,
-                                 tiles_in_gather ? &sc.tb : nullptr)) != cudaSuccess)
+                                 nullptr)) != cudaSuccess)
             return MOE_ERR_CUDA;
-        sc.tiles_built = fuse_tiles || tiles_in_gather;
+        sc.tiles_built = with_tiles;
     }
 
     CombineArgs ca{};
@@ -614,7 +614,7 @@ int moe_route(moe_plan_t *p, const void *x, const moe_layer_weights_t *w, int32_
     RouterArgs ra{x, w->router_W, w->router_bias, gated ? w->w_s : nullptr, T, c.d, c.E, k_l, renorm ? 1 : 0, c.dtype,
                   ws.logits, ws.topk_idx, ws.topk_w, ws.gamma, ws.status, false};
     cudaError_t err;
-    if (T > 512 && p->use_tc_router && tc_router_supported(&p->tc, ra))
+    if (T > kTcRouterMinTokens && p->use_tc_router && tc_router_supported(&p->tc, ra))
         err = launch_router_tc(&p->tc, ra, p->sm_count, s, &p->launches);
     else
         err = launch_router(ra, s, &p->launches);

@@ -77,6 +77,50 @@ def test_routing_from_given_logits_is_bit_exact(T, E, k, renorm):
         np.testing.assert_allclose(wts.sum(dim=1).cpu().numpy(), 1.0, atol=1e-5)
 
 
+@pytest.mark.parametrize("T,E,k,renorm,gated", [(300, 16, 12, True, False), (200, 60, 4, False, True),
+                                                (1100, 64, 8, False, False), (129, 8, 8, True, False),
+                                                (513, 37, 3, True, False)])
+def test_tensor_core_router_selects_like_the_oracle_from_its_own_logits(T, E, k, renorm, gated):
+    """The router for more than 128 tokens (logits on the tensor cores, selection in the epilogue),
+    with duplicated rows of W_g so that many logits are exactly equal: from the logits the GPU
+    itself reports, the oracle's selection must be the GPU's on EVERY token, in order, more than
+    eight picks and k = E included; the logits themselves are held to the oracle's."""
+    d = 256
+    g = torch.Generator().manual_seed(T + 17 * E + k)
+    x = torch.randn((T, d), generator=g).to(torch.bfloat16)
+    W = (0.05 * torch.randn((E, d), generator=g)).to(torch.bfloat16)
+    W[E // 2] = W[1]                                      # equal logits on every token
+    W[E - 1] = W[0]
+    bias = 0.3 * torch.randn((E,), generator=g)
+    bias[E // 2] = bias[1]
+    bias[E - 1] = bias[0]
+    w = {"router_W": W, "router_bias": bias, "W_gate": torch.zeros((E, 64, d), dtype=torch.bfloat16),
+         "W_up": torch.zeros((E, 64, d), dtype=torch.bfloat16), "W_down": torch.zeros((E, d, 64), dtype=torch.bfloat16)}
+    if gated:
+        w.update({"Ws_gate": torch.zeros((64, d), dtype=torch.bfloat16), "Ws_up": torch.zeros((64, d), dtype=torch.bfloat16),
+                  "Ws_down": torch.zeros((d, 64), dtype=torch.bfloat16),
+                  "w_s": (0.05 * torch.randn((d,), generator=g)).to(torch.bfloat16)})
+    w_dev = {n: t.to(DEV) for n, t in w.items()}
+    with B.MoEPlan(d, E, 64, T, k, torch.bfloat16, I_shared=64 if gated else 0, shared_gate=gated) as plan:
+        r = B.moe_route(plan.handle, x.to(DEV), B.make_weights(w_dev), k, renorm, E)
+        idx, wts, counts, offsets, perm, logits = plan.last_routing(T, k)
+        assert plan.device_status() == 0
+        torch.cuda.synchronize()
+    z = logits.cpu().numpy()
+    z_ref = orc.router_logits(x, W, bias)
+    np.testing.assert_allclose(z, z_ref, rtol=0, atol=2e-4 * max(1.0, float(np.abs(z_ref).max())))
+    assert np.array_equal(z[:, E // 2], z[:, 1]) and np.array_equal(z[:, E - 1], z[:, 0])
+    idx_o, gate_o, _ = orc.topk_gates(z, k, renorm, select_f32=True)
+    assert np.array_equal(idx.cpu().numpy(), idx_o)
+    np.testing.assert_allclose(wts.cpu().numpy(), gate_o, rtol=2e-5, atol=1e-8)
+    counts_o, offsets_o, perm_o, _ = orc.dispatch(idx_o, E)
+    assert np.array_equal(counts.cpu().numpy(), counts_o) and np.array_equal(perm.cpu().numpy(), perm_o)
+    assert np.array_equal(r["topk_idx"].cpu().numpy(), idx_o)
+    if gated:
+        gamma_ref = 1.0 / (1.0 + np.exp(-(x.double().numpy() @ w["w_s"].double().numpy())))
+        np.testing.assert_allclose(r["gamma"].cpu().numpy(), gamma_ref, rtol=1e-4, atol=1e-6)
+
+
 # --------------------------------------------------------------------------- single layer
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
