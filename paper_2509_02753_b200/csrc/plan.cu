@@ -620,7 +620,7 @@ int moe_route(moe_plan_t *p, const void *x, const moe_layer_weights_t *w, int32_
         err = launch_router(ra, s, &p->launches);
     if (err != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
     DispatchArgs da{ws.topk_idx, T, k_l, c.E, ws.counts, ws.offsets, ws.perm, ws.inv_perm, ws.part_hist, ws.status};
-    if (launch_dispatch(da, s, &p->launches) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
+    if (launch_dispatch_cluster(da, s, &p->launches, false, nullptr) != cudaSuccess) { cudaGetLastError(); return MOE_ERR_CUDA; }
     p->last_T = T;
     p->last_k = k_l;
     const size_t pairs = (size_t)T * k_l;
