@@ -21,7 +21,8 @@ __global__ void __launch_bounds__(256) decode_front_kernel(FrontArgs a) {
     extern __shared__ float xs[];                 // [d] the token's row, widened
     __shared__ int32_t s_last;
     __shared__ int32_t s_idx[kFrontMaxPairs];
-    __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1], cursor_s[kMaxExperts + 1];
+    __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1];
+    __shared__ int32_t hist8[8][kMaxExperts];
     __shared__ TileBuildSmem tb_sm;
 
     pdl_trigger();
@@ -97,16 +98,36 @@ __global__ void __launch_bounds__(256) decode_front_kernel(FrontArgs a) {
     for (int i = tid; i < E * Tn; i += 256) a.pos[i] = -1;
     __syncthreads();
 
-    // ---- dispatch tables.  Counts: shared-memory atomics (order does not matter for a count).
+    // ---- dispatch tables: each of the 8 warps takes a contiguous run of pairs.  Pass 1 counts the
+    // run per expert, a scan over (expert, warp) gives every warp its first row of each expert, pass 2
+    // places the pairs: inside a step of 32 pairs those of one expert are ranked by lane (ballot),
+    // across steps by the warp's cursor - a stable counting sort.
     const int n_pairs = Tn * k;
-    for (int e = tid; e <= E; e += 256) cnt_s[e] = 0;
+    const int per_warp = ((n_pairs + 7) / 8 + 31) / 32 * 32;
+    const int p0 = min(warp * per_warp, n_pairs), p1 = min(p0 + per_warp, n_pairs);
+    for (int e = lane; e < kMaxExperts; e += 32) hist8[warp][e] = 0;
+    __syncwarp();
+    for (int base = p0; base < p1; base += 32) {
+        const int p = base + lane;
+        int e = p < p1 ? s_idx[p] : -1;
+        if ((unsigned)e >= (unsigned)E) e = -1;
+        const unsigned peers = __match_any_sync(0xffffffffu, e);
+        if (e >= 0 && lane == __ffs(peers) - 1) hist8[warp][e] += __popc(peers);
+        __syncwarp();
+    }
     __syncthreads();
-    for (int p = tid; p < n_pairs; p += 256) atomicAdd(&cnt_s[s_idx[p]], 1);
+    if (tid < kMaxExperts) {
+        int run = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            const int c = hist8[w][tid];
+            hist8[w][tid] = run;
+            run += c;
+        }
+        cnt_s[tid] = tid < E ? run : 0;
+    }
     __syncthreads();
     if (warp == 0) {
-        // exclusive scan of the counts (<= 128 experts, 4 per lane), then the ranked placement:
-        // the warp takes the pairs in order, 32 at a time; pairs of one expert inside a step are
-        // ranked by lane, across steps by a cursor - a stable counting sort
         int c[kExpertsPerLane], sum = 0;
 #pragma unroll
         for (int j = 0; j < kExpertsPerLane; ++j) {
@@ -124,31 +145,32 @@ __global__ void __launch_bounds__(256) decode_front_kernel(FrontArgs a) {
 #pragma unroll
         for (int j = 0; j < kExpertsPerLane; ++j) {
             const int e = lane * kExpertsPerLane + j;
-            if (e < E) { off_s[e] = run; a.counts[e] = c[j]; a.offsets[e] = run; cursor_s[e] = run; }
+            if (e < E) { off_s[e] = run; a.counts[e] = c[j]; a.offsets[e] = run; }
             run += c[j];
         }
         if (lane == 31) { off_s[E] = incl; a.offsets[E] = incl; }
-        __syncwarp();
-        for (int base = 0; base < n_pairs; base += 32) {
-            const int p = base + lane;
-            const int e = p < n_pairs ? s_idx[p] : -1;
-            const unsigned peers = __match_any_sync(0xffffffffu, e);
-            const int rank = __popc(peers & ((1u << lane) - 1u));
-            const int leader = __ffs(peers) - 1;
-            int first = 0;
-            if (e >= 0 && lane == leader) {
-                first = cursor_s[e];
-                cursor_s[e] = first + __popc(peers);
-            }
-            first = __shfl_sync(0xffffffffu, first, leader);
-            if (e >= 0) {
-                const int row = first + rank;
-                a.perm[row] = p;
-                a.inv_perm[p] = row;
-                a.pos[e * Tn + p / k] = row;
-            }
-            __syncwarp();
+    }
+    __syncthreads();
+    for (int base = p0; base < p1; base += 32) {
+        const int p = base + lane;
+        int e = p < p1 ? s_idx[p] : -1;
+        if ((unsigned)e >= (unsigned)E) e = -1;
+        const unsigned peers = __match_any_sync(0xffffffffu, e);
+        const int leader = __ffs(peers) - 1;
+        int first = 0;
+        if (e >= 0 && lane == leader) {
+            first = hist8[warp][e];
+            hist8[warp][e] = first + __popc(peers);
+            first += off_s[e];
         }
+        first = __shfl_sync(0xffffffffu, first, leader);
+        if (e >= 0) {
+            const int row = first + __popc(peers & ((1u << lane) - 1u));
+            a.perm[row] = p;
+            a.inv_perm[p] = row;
+            a.pos[e * Tn + p / k] = row;
+        }
+        __syncwarp();
     }
     __syncthreads();
     build_tiles_block(a.tb, cnt_s, off_s, tb_sm);

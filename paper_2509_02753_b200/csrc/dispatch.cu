@@ -114,114 +114,6 @@ __global__ void __launch_bounds__(256) dispatch_scatter_kernel(DispatchArgs a, i
     }
 }
 
-// One-block variant for calls of at most 8192 pairs (above that one SM is slower than the three
-// kernels spread over many): the three passes without leaving the block, and, when asked, the tile lists of the tensor-core GEMMs right
-// behind them (counts and offsets are still in shared memory).  Warp w owns a contiguous range of
-// pairs; it loads 32 steps of indices at once so that the global-memory latency is paid per batch,
-// not per step.  Ranks are ballot ranks over pairs taken in order, as in the three-kernel form.
-constexpr int kBlockDispatchMaxPairs = kBlockDispatchPairs;
-
-__global__ void __launch_bounds__(1024) dispatch_block_kernel(DispatchArgs a, int n_pairs, TileBuildArgs tb,
-                                                              int build) {
-    __shared__ int32_t hist[32][kMaxExperts];
-    __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1];
-    __shared__ TileBuildSmem tb_sm;
-    pdl_trigger();
-    pdl_wait();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int per_warp = (((n_pairs + 31) / 32) + 31) / 32 * 32;
-    const int p0 = min(warp * per_warp, n_pairs), p1 = min(p0 + per_warp, n_pairs);
-    for (int e = lane; e < kMaxExperts; e += 32) hist[warp][e] = 0;
-    __syncwarp();
-    // pass 1: histogram of the warp's range
-    for (int base = p0; base < p1; base += 1024) {
-        int ev[32];
-#pragma unroll
-        for (int u = 0; u < 32; ++u) {
-            const int p = base + u * 32 + lane;
-            ev[u] = p < p1 ? a.topk_idx[p] : -1;
-        }
-#pragma unroll
-        for (int u = 0; u < 32; ++u) {
-            if ((unsigned)ev[u] < (unsigned)a.E) atomicAdd(&hist[warp][ev[u]], 1);
-            else if (ev[u] != -1) atomicOr(a.status, kStatusBadIndex);
-        }
-    }
-    __syncthreads();
-    // per expert: exclusive scan over the warps, total count
-    if (threadIdx.x < a.E) {
-        const int e = threadIdx.x;
-        int run = 0;
-#pragma unroll 8
-        for (int w = 0; w < 32; ++w) {
-            const int c = hist[w][e];
-            hist[w][e] = run;
-            run += c;
-        }
-        cnt_s[e] = run;
-    }
-    __syncthreads();
-    if (warp == 0) {
-        int c[kExpertsPerLane], sum = 0;
-#pragma unroll
-        for (int j = 0; j < kExpertsPerLane; ++j) {
-            const int e = lane * kExpertsPerLane + j;
-            c[j] = e < a.E ? cnt_s[e] : 0;
-            sum += c[j];
-        }
-        int incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        int run = incl - sum;
-#pragma unroll
-        for (int j = 0; j < kExpertsPerLane; ++j) {
-            const int e = lane * kExpertsPerLane + j;
-            if (e < a.E) { off_s[e] = run; a.counts[e] = c[j]; a.offsets[e] = run; }
-            run += c[j];
-        }
-        if (lane == 31) { off_s[a.E] = incl; a.offsets[a.E] = incl; }
-    }
-    __syncthreads();
-    // pass 2: ranked placement; hist[warp][e] + off_s[e] is the warp's cursor for expert e
-    for (int base = p0; base < p1; base += 1024) {
-        int ev[32];
-#pragma unroll
-        for (int u = 0; u < 32; ++u) {
-            const int p = base + u * 32 + lane;
-            ev[u] = p < p1 ? a.topk_idx[p] : -1;
-        }
-#pragma unroll
-        for (int u = 0; u < 32; ++u) {
-            const int p = base + u * 32 + lane;
-            int e = ev[u];
-            if ((unsigned)e >= (unsigned)a.E) e = -1;
-            const unsigned peers = __match_any_sync(0xffffffffu, e);
-            const int rank = __popc(peers & ((1u << lane) - 1u));
-            const int leader = __ffs(peers) - 1;
-            int first = 0;
-            if (e >= 0 && lane == leader) {
-                first = hist[warp][e];
-                hist[warp][e] = first + __popc(peers);
-                first += off_s[e];
-            }
-            first = __shfl_sync(0xffffffffu, first, leader);
-            if (e >= 0) {
-                const int r = first + rank;
-                a.perm[r] = p;
-                a.inv_perm[p] = r;
-            }
-            __syncwarp();
-        }
-    }
-    if (build) {
-        __syncthreads();
-        build_tiles_block(tb, cnt_s, off_s, tb_sm);
-    }
-}
-
 // Cluster variant: the three passes in ONE launch for calls of any size the layer path sees.  A
 // cluster of 8 CTAs shares the pairs (CTA c the c-th eighth, warp w of it a contiguous run), the
 // per-CTA totals meet through distributed shared memory, and every CTA then knows where its first
@@ -385,16 +277,9 @@ cudaError_t launch_dispatch_cluster(const DispatchArgs &a, cudaStream_t s, uint6
     return e;
 }
 
-cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained,
-                            const TileBuildArgs *tiles) {
+cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained) {
     const int n_pairs = a.T * a.k;
     if (n_pairs <= 0) return cudaSuccess;
-    if (tiles != nullptr && n_pairs <= kBlockDispatchMaxPairs) {
-        const cudaError_t e = launch_chained(dispatch_block_kernel, dim3(1), dim3(1024), 0, s, chained, a, n_pairs,
-                                             *tiles, 1);
-        ++*launches;
-        return e;
-    }
     const int n_parts = (n_pairs + kPairsPerPart - 1) / kPairsPerPart;
     const int grid = (n_parts + 7) / 8;
     cudaError_t e = launch_chained(dispatch_count_kernel, dim3(grid), dim3(256), 0, s, chained, a, n_pairs, n_parts);
@@ -406,28 +291,16 @@ cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *lau
     return e;
 }
 
-// Gather: x_perm[r, :] = x[perm[r] / k, :], one warp per row, 16-byte loads and stores.  The first
-// tile_blocks blocks build the tile lists of the tensor-core GEMMs instead (both only need the
-// dispatch tables, so they run side by side in one launch).
-constexpr int kTileBlocks = 8;
+// Gather: x_perm[r, :] = x[perm[r] / k, :], one warp per row, 16-byte loads and stores.
 __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4 *__restrict__ x,
                                                           const int32_t *__restrict__ perm,
                                                           int n_rows, int k, int vec_per_row,
-                                                          uint4 *__restrict__ x_perm, TileBuildArgs tb,
-                                                          int tile_blocks) {
-    __shared__ TileBuildSmem tb_sm;
-    __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1];
+                                                          uint4 *__restrict__ x_perm) {
     pdl_trigger();
     pdl_wait();
-    if ((int)blockIdx.x < tile_blocks) {
-        for (int e = threadIdx.x; e < tb.E; e += blockDim.x) { cnt_s[e] = tb.counts[e]; off_s[e] = tb.offsets[e]; }
-        __syncthreads();
-        build_tiles_block(tb, cnt_s, off_s, tb_sm, blockIdx.x, tile_blocks);
-        return;
-    }
     const int lane = threadIdx.x & 31;
-    const int warps = (gridDim.x - tile_blocks) * 8;
-    for (int r = (blockIdx.x - tile_blocks) * 8 + (threadIdx.x >> 5); r < n_rows; r += warps) {
+    const int warps = gridDim.x * 8;
+    for (int r = blockIdx.x * 8 + (threadIdx.x >> 5); r < n_rows; r += warps) {
         const int t = perm[r] / k;
         const uint4 *src = x + (size_t)t * vec_per_row;
         uint4 *dst = x_perm + (size_t)r * vec_per_row;
@@ -436,15 +309,12 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const uint4 *__restric
 }
 
 cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k, int d, int dtype,
-                          void *x_perm, cudaStream_t s, uint64_t *launches, bool chained,
-                          const TileBuildArgs *tiles) {
+                          void *x_perm, cudaStream_t s, uint64_t *launches, bool chained) {
     if (n_rows <= 0) return cudaSuccess;
     const int bytes_per_row = d * (dtype == MOE_BF16 ? 2 : 4);
-    const int tile_blocks = tiles ? kTileBlocks : 0;
-    const int grid = min((n_rows + 7) / 8, 148 * 8) + tile_blocks;
+    const int grid = min((n_rows + 7) / 8, 148 * 8);
     const cudaError_t e = launch_chained(gather_rows_kernel, dim3(grid), dim3(256), 0, s, chained,
-                                         (const uint4 *)x, perm, n_rows, k, bytes_per_row / 16, (uint4 *)x_perm,
-                                         tiles ? *tiles : TileBuildArgs{}, tile_blocks);
+                                         (const uint4 *)x, perm, n_rows, k, bytes_per_row / 16, (uint4 *)x_perm);
     ++*launches;
     return e;
 }
@@ -696,5 +566,5 @@ extern "C" int moe_dispatch_tables_static(const int32_t *topk_idx, int32_t T, in
         return MOE_OK;
     }
     uint64_t launches = 0;
-    return lexi::launch_dispatch(a, s, &launches, false, nullptr) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+    return lexi::launch_dispatch(a, s, &launches, false) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

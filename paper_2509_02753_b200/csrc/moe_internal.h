@@ -110,21 +110,17 @@ struct DispatchArgs {
     const int32_t *topk_idx; int T, k, E;
     int32_t *counts, *offsets, *perm, *inv_perm, *part_hist; int32_t *status;
 };
-// tiles != NULL (and a call of at most kBlockDispatchPairs pairs): one block does the dispatch and then builds the
-// tensor-core tile lists; returns with both done.  Otherwise the three-kernel dispatch only.
-cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained = false,
-                            const TileBuildArgs *tiles = nullptr);
-constexpr int kBlockDispatchPairs = 8192;
+// The dispatch tables in three launches (per-warp histograms, one-block scan, ranked scatter).
+cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained = false);
 // The same tables from one launch of a cluster of 8 CTAs, whatever the size of the call; with tiles
 // != NULL the cluster also builds the tensor-core tile lists.
 cudaError_t launch_dispatch_cluster(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained,
                                     const TileBuildArgs *tiles);
-// Calls of more tokens than this take the tensor-core router (one CTA per 64 tokens, about as long
-// for 100 tokens as for 9000); up to it one block per token is as fast.
+// Calls of more tokens than this take the tensor-core router (a cluster of CTAs per 64 tokens); up
+// to it one block per token is as fast.
 constexpr int kTcRouterMinTokens = 128;
 cudaError_t launch_gather(const void *x, const int32_t *perm, int n_rows, int k, int d, int dtype,
-                          void *x_perm, cudaStream_t s, uint64_t *launches, bool chained = false,
-                          const TileBuildArgs *tiles = nullptr);   // tiles: also build the tile lists
+                          void *x_perm, cudaStream_t s, uint64_t *launches, bool chained = false);
 
 cudaError_t launch_regroup_index(const int32_t *recv_counts, int world, int E, int n_rows, int32_t *to_em, int32_t *inv,
                                  int32_t *per_expert, int32_t *status, cudaStream_t s, uint64_t *launches);

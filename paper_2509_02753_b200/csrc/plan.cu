@@ -243,8 +243,7 @@ int layer_impl(moe_plan *p, const void *x, const moe_layer_weights_t *w, int T, 
         const bool with_tiles = sched != MOE_SCHED_SIMT;
         if ((err = launch_dispatch_cluster(da, s, &p->launches, chained, with_tiles ? &sc.tb : nullptr)) != cudaSuccess)
             return MOE_ERR_CUDA;
-        if ((err = launch_gather(x, ws.perm, T * k, k, c.d, c.dtype, ws.x_perm, s, &p->launches, chained,
-                                 nullptr)) != cudaSuccess)
+        if ((err = launch_gather(x, ws.perm, T * k, k, c.d, c.dtype, ws.x_perm, s, &p->launches, chained)) != cudaSuccess)
             return MOE_ERR_CUDA;
         sc.tiles_built = with_tiles;
     }

@@ -111,6 +111,62 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
         a.n_tiles[0] = sm.pre1[groups];
         a.n_tiles[1] = sm.pre2[groups] + extra2;
     }
+    if (extra2 == 0) {
+        // No null tiles to weave in: every thread writes a contiguous run of each list, so that the
+        // search for the group and the divisions are paid once per run and the rest is counting up.
+        const int n_threads = n_blocks * blockDim.x, gid = rank * blockDim.x + threadIdx.x;
+        for (int phase = 0; phase < 2; ++phase) {
+            const int32_t *pre = phase == 0 ? sm.pre1 : sm.pre2;
+            const int total = pre[groups];
+            const int per = (total + n_threads - 1) / n_threads;
+            const int i0 = min(gid * per, total), i1 = min(i0 + per, total);
+            if (i0 >= i1) continue;
+            int lo = 0, hi = groups - 1;
+            while (lo < hi) {                     // last slot with pre[slot] <= i0
+                const int mid = (lo + hi + 1) >> 1;
+                if (pre[mid] <= i0) lo = mid; else hi = mid - 1;
+            }
+            int slot = lo, local = i0 - pre[lo];
+            for (int idx = i0; idx < i1; ++idx, ++local) {
+                while (local >= pre[slot + 1] - pre[slot]) { local -= pre[slot + 1] - pre[slot]; ++slot; }
+                const int g = group_of(slot);
+                const int rows = rows_of(g);
+                const int first = g == a.E ? 0 : off_s[g];
+                Tile t;
+                t.group = g;
+                if (phase == 0) {
+                    const int n1 = g == a.E ? n1_shared : n1_routed;
+                    const int m = local / n1, n = local - m * n1;
+                    if (a.direct) {
+                        t.row0 = 0;
+                        t.rows = a.T;
+                    } else {
+                        t.row0 = first + m * a.tile_rows;
+                        t.rows = min(a.tile_rows, rows - m * a.tile_rows);
+                    }
+                    t.n0 = n * a.feat1;
+                    t.k0 = 0; t.klen = a.K1; t.slot = 0;
+                    t.pad = (a.tile_rows > kTileRows && t.rows <= kTileRows) ? 1 : 0;
+                    a.tiles1[idx] = t;
+                } else {
+                    const int ks = g == a.E ? a.ksplit_shared : a.ksplit_routed;
+                    const int kchunk = g == a.E ? a.kchunk_shared : a.kchunk_routed;
+                    const int K = g == a.E ? a.K2_shared : a.K2_routed;
+                    const int m = local / (n2 * ks), rem = local - m * (n2 * ks);
+                    const int n = rem / ks, sl = rem - n * ks;
+                    t.row0 = first + m * a.tile_rows;
+                    t.rows = min(a.tile_rows, rows - m * a.tile_rows);
+                    t.n0 = n * a.bn2;
+                    t.k0 = sl * kchunk;
+                    t.klen = max(0, min(kchunk, K - sl * kchunk));
+                    t.slot = sl;
+                    t.pad = (a.tile_rows > kTileRows && t.rows <= kTileRows) ? 1 : 0;
+                    a.tiles2[idx] = t;
+                }
+            }
+        }
+        return;
+    }
     for (int phase = 0; phase < 2; ++phase) {
         const int32_t *pre = phase == 0 ? sm.pre1 : sm.pre2;
         const int logical = pre[groups];
