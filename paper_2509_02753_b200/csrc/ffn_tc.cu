@@ -25,6 +25,8 @@
 
 #include <cstdlib>
 
+#include <atomic>
+
 #include "ffn_tc.h"
 #include "tc_ptx.cuh"
 #include "tile_build.cuh"
@@ -647,15 +649,25 @@ size_t decode_row_cap(const moe_config_t &c) {
     return pairs < cap ? pairs : cap;
 }
 
+constexpr int kMaxTcDevices = 64;
+int current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxTcDevices) { cudaGetLastError(); return -1; }
+    return dev;
+}
+
 template <int PHASE, int BN, int A_ROWS, int STAGES, int MIN_CTAS, typename OutT>
 cudaError_t launch_tc(const CUtensorMap *maps, const TcParams &p, int grid, cudaStream_t s, bool chained) {
     auto kern = ffn_tc_kernel<PHASE, BN, A_ROWS, STAGES, MIN_CTAS, OutT>;
     constexpr int smem = tc_smem_bytes<A_ROWS, BN, STAGES>(tc_staged_out<PHASE, BN, OutT>());
-    static bool configured = false;
-    if (!configured) {
+    // the shared-memory opt-in belongs to the kernel on one device
+    static std::atomic<bool> configured[kMaxTcDevices];
+    const int dev = current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    if (!configured[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[dev].store(true, std::memory_order_release);
     }
     return launch_chained(kern, dim3(grid), dim3(192), smem, s, chained,
                           maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], p);
@@ -665,7 +677,10 @@ template <int PHASE, typename OutT>
 cudaError_t launch_tc_pair(const CUtensorMap *maps, const TcParams &p, int max_pairs, cudaStream_t s, bool chained) {
     auto kern = ffn_tc_pair_kernel<PHASE, OutT>;
     constexpr int smem = pair_smem_bytes<PHASE>();
-    static int max_clusters = -1;
+    static std::atomic<int> max_clusters_dev[kMaxTcDevices];     // 0: not asked yet on that device
+    const int dev = current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    int max_clusters = max_clusters_dev[dev].load(std::memory_order_acquire);
     cudaLaunchConfig_t cfg{};
     cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = smem; cfg.stream = s;
     cudaLaunchAttribute attr[2];
@@ -674,7 +689,7 @@ cudaError_t launch_tc_pair(const CUtensorMap *maps, const TcParams &p, int max_p
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    if (max_clusters < 0) {
+    if (max_clusters <= 0) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         cfg.gridDim = dim3(2 * 74);
@@ -684,6 +699,7 @@ cudaError_t launch_tc_pair(const CUtensorMap *maps, const TcParams &p, int max_p
         if (e != cudaSuccess) return e;
         if (n < 1) return cudaErrorInvalidConfiguration;
         max_clusters = n;
+        max_clusters_dev[dev].store(n, std::memory_order_release);
     }
     const int clusters = max_pairs < max_clusters ? (max_pairs < 1 ? 1 : max_pairs) : max_clusters;
     cfg.gridDim = dim3(2 * clusters);
