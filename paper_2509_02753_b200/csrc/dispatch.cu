@@ -8,6 +8,7 @@
 // Everything is deterministic: ranks come from warp ballots over pairs taken in order, never
 // from the arrival order of atomics.
 #include <atomic>
+#include <cstdlib>
 
 #include "moe_internal.h"
 #include "tile_build.cuh"
@@ -259,10 +260,32 @@ __global__ void __launch_bounds__(1024) dispatch_cluster_kernel(DispatchArgs a, 
     cluster_wait_acquire();
 }
 
+// The tile lists alone, from tables that are already in global memory (one block).
+__global__ void __launch_bounds__(1024) tile_lists_kernel(TileBuildArgs tb) {
+    __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1];
+    __shared__ TileBuildSmem tb_sm;
+    pdl_trigger();
+    pdl_wait();
+    for (int e = threadIdx.x; e <= tb.E; e += blockDim.x) {
+        cnt_s[e] = e < tb.E ? tb.counts[e] : 0;
+        off_s[e] = tb.offsets[e];
+    }
+    __syncthreads();
+    build_tiles_block(tb, cnt_s, off_s, tb_sm);
+}
+
+cudaError_t launch_dispatch(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained);
+
+// A device (or a share of one) that cannot run 8 CTAs of 1024 threads as one cluster gets the
+// three-kernel form followed by a one-block tile builder; LEXI_DISPATCH_CLUSTER=0 asks for that too.
 cudaError_t launch_dispatch_cluster(const DispatchArgs &a, cudaStream_t s, uint64_t *launches, bool chained,
                                     const TileBuildArgs *tiles) {
     const int n_pairs = a.T * a.k;
     if (n_pairs <= 0) return cudaSuccess;
+    static const bool env_off = [] { const char *v = getenv("LEXI_DISPATCH_CLUSTER"); return v && v[0] == '0'; }();
+    static std::atomic<int> usable[64];            // per device: 0 unknown, 1 yes, -1 no
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); dev = -1; }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(kDispatchClusterCtas); cfg.blockDim = dim3(1024); cfg.dynamicSmemBytes = 0; cfg.stream = s;
     cudaLaunchAttribute attr[2];
@@ -270,10 +293,27 @@ cudaError_t launch_dispatch_cluster(const DispatchArgs &a, cudaStream_t s, uint6
     attr[0].val.clusterDim.x = kDispatchClusterCtas; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = chained ? 2 : 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, dispatch_cluster_kernel, a, n_pairs,
-                                             tiles ? *tiles : TileBuildArgs{}, tiles ? 1 : 0);
-    ++*launches;
+    cfg.attrs = attr;
+    int state = env_off || dev < 0 ? -1 : usable[dev].load(std::memory_order_acquire);
+    if (state == 0) {
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, dispatch_cluster_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+        state = n >= 1 ? 1 : -1;
+        usable[dev].store(state, std::memory_order_release);
+    }
+    if (state == 1) {
+        cfg.numAttrs = chained ? 2 : 1;
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, dispatch_cluster_kernel, a, n_pairs,
+                                                 tiles ? *tiles : TileBuildArgs{}, tiles ? 1 : 0);
+        ++*launches;
+        return e;
+    }
+    cudaError_t e = launch_dispatch(a, s, launches, chained);
+    if (e == cudaSuccess && tiles) {
+        e = launch_chained(tile_lists_kernel, dim3(1), dim3(1024), 0, s, chained, *tiles);
+        ++*launches;
+    }
     return e;
 }
 

@@ -121,6 +121,41 @@ def test_tensor_core_router_selects_like_the_oracle_from_its_own_logits(T, E, k,
         np.testing.assert_allclose(r["gamma"].cpu().numpy(), gamma_ref, rtol=1e-4, atol=1e-6)
 
 
+def test_layer_without_the_dispatch_cluster_gives_the_same_bits():
+    """A device that cannot run 8 CTAs as one cluster gets the dispatch tables from three kernels
+    and the tile lists from a fourth.  LEXI_DISPATCH_CLUSTER=0 (read once per process, hence the
+    child process) takes that way; both ways must give the same bits on two prefill-sized calls
+    and one on the decode schedule."""
+    import os
+    import subprocess
+    import sys
+    import tempfile
+    code = (
+        "import sys, torch\n"
+        "sys.path.insert(0, sys.argv[1])\n"
+        "from paper_2509_02753_b200 import binding as B, synth\n"
+        "wl = synth.Workload('fb', d=256, E=24, I=192, k_base=3, L=1, I_shared=128, shared_gate=True, router_bias_std=0.5, w_std=0.02)\n"
+        "w = B.make_weights(synth.make_layer(wl, 0, torch.bfloat16, 'cuda'))\n"
+        "out = {}\n"
+        "with B.MoEPlan(wl.d, wl.E, wl.I, 1500, 3, torch.bfloat16, I_shared=wl.I_shared, shared_gate=True) as plan:\n"
+        "    for T, k in ((1500, 3), (300, 3), (150, 2)):\n"
+        "        x = synth.make_tokens(wl, T, torch.bfloat16, 'cuda')\n"
+        "        out[T] = plan.layer_forward(x, w, k, True).cpu()\n"
+        "    assert plan.device_status() == 0\n"
+        "torch.save(out, sys.argv[2])\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    results = {}
+    with tempfile.TemporaryDirectory() as tmp:
+        for flag in ("1", "0"):
+            path = os.path.join(tmp, f"y{flag}.pt")
+            env = dict(os.environ, LEXI_DISPATCH_CLUSTER=flag)
+            subprocess.run([sys.executable, "-c", code, root, path], check=True, env=env, timeout=300)
+            results[flag] = torch.load(path)
+    for T, y in results["1"].items():
+        assert torch.isfinite(y.float()).all()
+        assert torch.equal(y, results["0"][T]), f"T={T}"
+
+
 # --------------------------------------------------------------------------- single layer
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
