@@ -79,12 +79,15 @@ def test_routing_from_given_logits_is_bit_exact(T, E, k, renorm):
 
 @pytest.mark.parametrize("T,E,k,renorm,gated", [(300, 16, 12, True, False), (200, 60, 4, False, True),
                                                 (1100, 64, 8, False, False), (129, 8, 8, True, False),
-                                                (513, 37, 3, True, False)])
+                                                (513, 37, 3, True, False), (19100, 24, 5, False, True),
+                                                (3000, 16, 2, True, False)])
 def test_tensor_core_router_selects_like_the_oracle_from_its_own_logits(T, E, k, renorm, gated):
     """The router for more than 128 tokens (logits on the tensor cores, selection in the epilogue),
     with duplicated rows of W_g so that many logits are exactly equal: from the logits the GPU
     itself reports, the oracle's selection must be the GPU's on EVERY token, in order, more than
-    eight picks and k = E included; the logits themselves are held to the oracle's."""
+    eight picks and k = E included; the logits themselves are held to the oracle's.  The sizes cover
+    clusters of 4, 2 and 1 CTAs per tile, a CTA with several tiles, and the 128-token tiles of very
+    large calls."""
     d = 256
     g = torch.Generator().manual_seed(T + 17 * E + k)
     x = torch.randn((T, d), generator=g).to(torch.bfloat16)
