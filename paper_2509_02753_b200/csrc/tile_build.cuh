@@ -126,17 +126,32 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
                 const int mid = (lo + hi + 1) >> 1;
                 if (pre[mid] <= i0) lo = mid; else hi = mid - 1;
             }
-            int slot = lo, local = i0 - pre[lo];
+            int slot = lo, local = i0 - pre[lo], gsz = pre[lo + 1] - pre[lo];
+            int cur = -1, g = 0, rows = 0, first = 0, m = 0, n = 0, sl = 0;
+            int nn = 1, ks = 1, kchunk = 0, K = 0;     // feature blocks, K slabs, slab length, K of the group
             for (int idx = i0; idx < i1; ++idx, ++local) {
-                while (local >= pre[slot + 1] - pre[slot]) { local -= pre[slot + 1] - pre[slot]; ++slot; }
-                const int g = group_of(slot);
-                const int rows = rows_of(g);
-                const int first = g == a.E ? 0 : off_s[g];
+                while (local >= gsz) { local -= gsz; ++slot; gsz = pre[slot + 1] - pre[slot]; }
+                if (slot != cur) {                // first tile of the run, or a new group: divide once
+                    cur = slot;
+                    g = group_of(slot);
+                    rows = rows_of(g);
+                    first = g == a.E ? 0 : off_s[g];
+                    if (phase == 0) {
+                        nn = g == a.E ? n1_shared : n1_routed;
+                        m = local / nn; n = local - m * nn;
+                    } else {
+                        nn = n2;
+                        ks = g == a.E ? a.ksplit_shared : a.ksplit_routed;
+                        kchunk = g == a.E ? a.kchunk_shared : a.kchunk_routed;
+                        K = g == a.E ? a.K2_shared : a.K2_routed;
+                        m = local / (nn * ks);
+                        const int rem = local - m * (nn * ks);
+                        n = rem / ks; sl = rem - n * ks;
+                    }
+                }
                 Tile t;
                 t.group = g;
                 if (phase == 0) {
-                    const int n1 = g == a.E ? n1_shared : n1_routed;
-                    const int m = local / n1, n = local - m * n1;
                     if (a.direct) {
                         t.row0 = 0;
                         t.rows = a.T;
@@ -148,12 +163,8 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
                     t.k0 = 0; t.klen = a.K1; t.slot = 0;
                     t.pad = (a.tile_rows > kTileRows && t.rows <= kTileRows) ? 1 : 0;
                     a.tiles1[idx] = t;
+                    if (++n == nn) { n = 0; ++m; }
                 } else {
-                    const int ks = g == a.E ? a.ksplit_shared : a.ksplit_routed;
-                    const int kchunk = g == a.E ? a.kchunk_shared : a.kchunk_routed;
-                    const int K = g == a.E ? a.K2_shared : a.K2_routed;
-                    const int m = local / (n2 * ks), rem = local - m * (n2 * ks);
-                    const int n = rem / ks, sl = rem - n * ks;
                     t.row0 = first + m * a.tile_rows;
                     t.rows = min(a.tile_rows, rows - m * a.tile_rows);
                     t.n0 = n * a.bn2;
@@ -162,6 +173,7 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
                     t.slot = sl;
                     t.pad = (a.tile_rows > kTileRows && t.rows <= kTileRows) ? 1 : 0;
                     a.tiles2[idx] = t;
+                    if (++sl == ks) { sl = 0; if (++n == nn) { n = 0; ++m; } }
                 }
             }
         }
