@@ -119,8 +119,7 @@ __global__ void __launch_bounds__(256) dispatch_scatter_kernel(DispatchArgs a, i
 // cluster of 8 CTAs shares the pairs (CTA c the c-th eighth, warp w of it a contiguous run), the
 // per-CTA totals meet through distributed shared memory, and every CTA then knows where its first
 // row of each expert lies: expert-major, inside an expert CTA by CTA, warp by warp, pair by pair -
-// the same stable order as the other forms.  Ranks are ballot ranks (no atomics).  The loops are
-// kept rolled: a kernel this short mostly runs instructions it fetches for the first time.
+// the same stable order as the other forms.  Ranks are ballot ranks (no atomics).
 // When asked, the eight CTAs also build an eighth each of the tile lists of the tensor-core GEMMs.
 constexpr int kDispatchClusterCtas = 8;
 

@@ -14,9 +14,10 @@
 //     all CTAs read it through distributed shared memory; C is chosen so that the clusters of a
 //     call still run at once;
 //   * the selection is done by four threads per token, 16 logits each: a pick is a short tournament
-//     in registers plus two shuffle steps, and the loop over the k_l picks is not unrolled, so the
-//     code stays small (a kernel this short runs mostly on instructions it fetches for the first
-//     time); the tokens of a tile are spread over the CTAs of the cluster.
+//     in registers plus two shuffle steps (the selection is a chain of dependent instructions with
+//     few warps to hide it: one thread per token over all 64 logits, one warp per token with k_l
+//     warp-wide reductions, and ranking every logit against all others each measured 3-4 times
+//     slower); the tokens of a tile are spread over the CTAs of the cluster.
 // Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-17 move the accumulator to shared memory and
 // route.  Selection semantics equal the warp-shuffle router: fp32 logits (+ bias), larger first,
 // equal logits -> lower index.  All mbarrier waits are bounded; a wait that gives up still
