@@ -54,17 +54,32 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
     const int n1_routed = (a.N1_routed + a.feat1 - 1) / a.feat1;
     const int n1_shared = (a.N1_shared + a.feat1 - 1) / a.feat1;
     const int n2 = (a.N2 + a.bn2 - 1) / a.bn2;
+    int st_touched = 0, st_rows_r = 0, st_rows_s = 0;     // this thread's share of the call's statistics
     for (int sidx = threadIdx.x; sidx < groups; sidx += blockDim.x) {
         const int g = group_of(sidx);
         const int mblk = (rows_of(g) + a.tile_rows - 1) / a.tile_rows;
-        if (rank == 0 && a.stats && g != a.E && rows_of(g) > 0) atomicAdd(a.stats, 1);
-        if (rank == 0 && a.stats && !a.direct) {
+        if (g != a.E && rows_of(g) > 0) ++st_touched;
+        if (!a.direct) {
             const int r = rows_of(g), rem = r % a.tile_rows;
             const int small = a.tile_rows / 2;          // a last block of at most half a tile runs at half height
-            atomicAdd(a.stats + (g == a.E ? 2 : 1), r / a.tile_rows * a.tile_rows + (rem == 0 ? 0 : (rem <= small ? small : a.tile_rows)));
+            const int run = r / a.tile_rows * a.tile_rows + (rem == 0 ? 0 : (rem <= small ? small : a.tile_rows));
+            if (g == a.E) st_rows_s += run; else st_rows_r += run;
         }
         sm.pre1[sidx] = mblk1_of(g) * (g == a.E ? n1_shared : n1_routed);
         sm.pre2[sidx] = mblk * n2 * (g == a.E ? a.ksplit_shared : a.ksplit_routed);
+    }
+    if (rank == 0 && a.stats && threadIdx.x < ((groups + 31) & ~31)) {     // the warps that saw a group: one atomic each per counter
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            st_touched += __shfl_xor_sync(0xffffffffu, st_touched, o);
+            st_rows_r += __shfl_xor_sync(0xffffffffu, st_rows_r, o);
+            st_rows_s += __shfl_xor_sync(0xffffffffu, st_rows_s, o);
+        }
+        if ((threadIdx.x & 31) == 0) {
+            if (st_touched) atomicAdd(a.stats, st_touched);
+            if (st_rows_r) atomicAdd(a.stats + 1, st_rows_r);
+            if (st_rows_s) atomicAdd(a.stats + 2, st_rows_s);
+        }
     }
     __syncthreads();
     if (threadIdx.x < 32) {
