@@ -809,6 +809,12 @@ void tc_make_schedule(const moe_config_t &c, const Workspace &ws, const FfnArgs 
     tb.status = ws.status;
     tb.direct = direct ? 1 : 0;
     tb.tile_rows = sc.pair ? 2 * kTileRows : kTileRows;
+    tb.tile_shift = sc.pair ? 8 : 7;
+    static_assert(kTileRows == 128, "tile_shift");
+    tb.n1_routed_blocks = (tb.N1_routed + tb.feat1 - 1) / tb.feat1;
+    tb.n1_shared_blocks = (tb.N1_shared + tb.feat1 - 1) / tb.feat1;
+    tb.n2_blocks = (tb.N2 + tb.bn2 - 1) / tb.bn2;
+    tb.long_over_short_m1 = tb.K2_routed > 0 ? (tb.K2_shared + tb.K2_routed - 1) / tb.K2_routed - 1 : 0;
     // prefill: consumers of the phase-2 list (CTAs, or CTA pairs), for the balance of long shared tiles
     tb.rr2 = (!decode && !direct && has_shared) ? (sc.pair ? sm_count / 2 : sm_count) : 0;
     tb.stats = ws.stats;

@@ -25,6 +25,10 @@ struct TileBuildArgs {
     // reduce over a longer K than the routed ones; null tiles (rows = 0) are slipped in behind the
     // shared tiles so that every consumer ends up with the same amount of work
     int32_t rr2;
+    // quotients the host knows (an integer division on the device is a chain of ~30 instructions):
+    // feature blocks of phase 1 per routed / shared group, output blocks of phase 2, log2(tile_rows),
+    // and how many rounds of short tiles one long shared tile of phase 2 is worth, less one
+    int32_t n1_routed_blocks, n1_shared_blocks, n2_blocks, tile_shift, long_over_short_m1;
     int32_t *stats;   // stats[0] += routed experts that received at least one token; stats[1], stats[2] += token
                       // rows the MMAs of this call execute for the routed / shared groups (valid rows rounded up to
                       // the MMA heights the kernels use): executed = padded work, against T k_l and T algorithmic rows
@@ -33,6 +37,7 @@ struct TileBuildArgs {
 // Shared-memory scratch of build_tiles_block.
 struct TileBuildSmem {
     int32_t pre1[kMaxExperts + 2], pre2[kMaxExperts + 2];
+    int32_t part1[32], part2[32];
 };
 
 // Called by all threads of one block; cnt_s/off_s hold counts and offsets in shared memory.
@@ -48,21 +53,20 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
     auto rows_of = [&](int g) { return g == a.E ? a.T : cnt_s[g]; };
     auto mblk1_of = [&](int g) {
         const int r = rows_of(g);
-        return a.direct ? (r > 0 ? 1 : 0) : (r + a.tile_rows - 1) / a.tile_rows;
+        return a.direct ? (r > 0 ? 1 : 0) : (r + a.tile_rows - 1) >> a.tile_shift;
     };
     // tiles per group, then an exclusive scan over the (at most 129) groups by warp 0
-    const int n1_routed = (a.N1_routed + a.feat1 - 1) / a.feat1;
-    const int n1_shared = (a.N1_shared + a.feat1 - 1) / a.feat1;
-    const int n2 = (a.N2 + a.bn2 - 1) / a.bn2;
+    const int n1_routed = a.n1_routed_blocks, n1_shared = a.n1_shared_blocks, n2 = a.n2_blocks;
+    const int tmask = a.tile_rows - 1;            // tile_rows is 128 or 256
     int st_touched = 0, st_rows_r = 0, st_rows_s = 0;     // this thread's share of the call's statistics
     for (int sidx = threadIdx.x; sidx < groups; sidx += blockDim.x) {
         const int g = group_of(sidx);
-        const int mblk = (rows_of(g) + a.tile_rows - 1) / a.tile_rows;
+        const int mblk = (rows_of(g) + a.tile_rows - 1) >> a.tile_shift;
         if (g != a.E && rows_of(g) > 0) ++st_touched;
         if (!a.direct) {
-            const int r = rows_of(g), rem = r % a.tile_rows;
+            const int r = rows_of(g), rem = r & tmask;
             const int small = a.tile_rows / 2;          // a last block of at most half a tile runs at half height
-            const int run = r / a.tile_rows * a.tile_rows + (rem == 0 ? 0 : (rem <= small ? small : a.tile_rows));
+            const int run = (r & ~tmask) + (rem == 0 ? 0 : (rem <= small ? small : a.tile_rows));
             if (g == a.E) st_rows_s += run; else st_rows_r += run;
         }
         sm.pre1[sidx] = mblk1_of(g) * (g == a.E ? n1_shared : n1_routed);
@@ -83,30 +87,34 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
     }
     __syncthreads();
     if (threadIdx.x < 32) {
+        // exclusive scan over the (at most 129) groups: every lane sums its own stretch, then adds up
+        // the stretch sums of the lanes before it from shared memory (32 independent broadcast
+        // loads; a chain of five shuffle rounds measured 1.5 us here, a serial walk 1.2 us)
         const int lane = threadIdx.x;
         const int per = (groups + 31) / 32;
         const int base = lane * per;
         int s1 = 0, s2 = 0;
         for (int i = 0; i < per; ++i)
             if (base + i < groups) { s1 += sm.pre1[base + i]; s2 += sm.pre2[base + i]; }
-        int i1 = s1, i2 = s2;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v1 = __shfl_up_sync(0xffffffffu, i1, o), v2 = __shfl_up_sync(0xffffffffu, i2, o);
-            if (lane >= o) { i1 += v1; i2 += v2; }
+        sm.part1[lane] = s1; sm.part2[lane] = s2;
+        __syncwarp();
+        int r1 = 0, r2 = 0, t1 = 0, t2 = 0;
+#pragma unroll 8
+        for (int l = 0; l < 32; ++l) {
+            const int c1 = sm.part1[l], c2 = sm.part2[l];
+            r1 += l < lane ? c1 : 0; r2 += l < lane ? c2 : 0;
+            t1 += c1; t2 += c2;
         }
-        int r1 = i1 - s1, r2 = i2 - s2;
+        if (lane == 0) {
+            if (t1 > a.cap1 || t2 + kMaxBalanceTiles > a.cap2) { atomicOr(a.status, kStatusBadIndex); t1 = 0; t2 = 0; }
+            sm.pre1[groups] = t1; sm.pre2[groups] = t2;
+        }
         for (int i = 0; i < per; ++i)
             if (base + i < groups) {
                 const int c1 = sm.pre1[base + i], c2 = sm.pre2[base + i];
                 sm.pre1[base + i] = r1; sm.pre2[base + i] = r2;
                 r1 += c1; r2 += c2;
             }
-        if (lane == 31) {
-            int t1 = i1, t2 = i2;
-            if (t1 > a.cap1 || t2 + kMaxBalanceTiles > a.cap2) { atomicOr(a.status, kStatusBadIndex); t1 = 0; t2 = 0; }
-            sm.pre1[groups] = t1; sm.pre2[groups] = t2;
-        }
     }
     __syncthreads();
     // Balance of list 2 (see rr2): S long shared tiles come first; if S is not a multiple of the
@@ -118,7 +126,7 @@ __device__ __forceinline__ void build_tiles_block(const TileBuildArgs &a, const 
         bal_S = groups > 1 ? sm.pre2[1] : sm.pre2[groups];
         bal_C = a.rr2;
         bal_rem = bal_S % bal_C;
-        bal_rows = bal_rem > 0 ? (a.K2_shared + a.K2_routed - 1) / a.K2_routed - 1 : 0;
+        bal_rows = bal_rem > 0 ? a.long_over_short_m1 : 0;
         if (bal_rows * bal_rem > kMaxBalanceTiles) bal_rows = 0;
     }
     const int extra2 = bal_rows * bal_rem;
