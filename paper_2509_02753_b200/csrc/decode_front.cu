@@ -23,6 +23,7 @@ __global__ void __launch_bounds__(256) decode_front_kernel(FrontArgs a) {
     __shared__ int32_t s_idx[kFrontMaxPairs];
     __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1];
     __shared__ int32_t hist8[8][kMaxExperts];
+    __shared__ int32_t part_s[32];
     __shared__ TileBuildSmem tb_sm;
 
     pdl_trigger();
@@ -135,13 +136,17 @@ __global__ void __launch_bounds__(256) decode_front_kernel(FrontArgs a) {
             c[j] = e < E ? cnt_s[e] : 0;
             sum += c[j];
         }
-        int incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
+        // exclusive prefix over the lanes: the sums of the lanes before this one, read from shared
+        // memory (32 independent loads instead of a chain of five shuffle rounds)
+        part_s[lane] = sum;
+        __syncwarp();
+        int run = 0, incl = 0;
+#pragma unroll 8
+        for (int l = 0; l < 32; ++l) {
+            const int v = part_s[l];
+            run += l < lane ? v : 0;
+            incl += l <= lane ? v : 0;
         }
-        int run = incl - sum;
 #pragma unroll
         for (int j = 0; j < kExpertsPerLane; ++j) {
             const int e = lane * kExpertsPerLane + j;

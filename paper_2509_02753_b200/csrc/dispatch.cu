@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(1024) dispatch_cluster_kernel(DispatchArgs a, 
     __shared__ int32_t hist[32][kMaxExperts];
     __shared__ int32_t tot_s[kMaxExperts];                       // this CTA's pairs per expert (read by the other CTAs)
     __shared__ int32_t first_s[kMaxExperts];                     // pairs of an expert in the CTAs before this one
-    __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1];
+    __shared__ int32_t cnt_s[kMaxExperts + 1], off_s[kMaxExperts + 1], part_s[32];
     __shared__ TileBuildSmem tb_sm;
     pdl_trigger();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -200,13 +200,17 @@ __global__ void __launch_bounds__(1024) dispatch_cluster_kernel(DispatchArgs a, 
             c[j] = e < a.E ? cnt_s[e] : 0;
             sum += c[j];
         }
-        int incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
+        // exclusive prefix over the lanes: the sums of the lanes before this one, read from shared
+        // memory (32 independent loads instead of a chain of five shuffle rounds)
+        part_s[lane] = sum;
+        __syncwarp();
+        int run = 0, incl = 0;
+#pragma unroll 8
+        for (int l = 0; l < 32; ++l) {
+            const int v = part_s[l];
+            run += l < lane ? v : 0;
+            incl += l <= lane ? v : 0;
         }
-        int run = incl - sum;
 #pragma unroll
         for (int j = 0; j < kExpertsPerLane; ++j) {
             const int e = lane * kExpertsPerLane + j;
